@@ -1,0 +1,194 @@
+/*
+ * cats.h -- C ABI of libcats: the target model's tree-verification forward of
+ * CATS-style self-speculative decoding (Algorithm 1, Stage 3 "Final
+ * Verification", and the walk / roll-back that follow it), for NVIDIA B200
+ * (sm_100a).
+ *
+ * One decoding cycle hands this library a draft token tree of T nodes
+ * (1 <= T <= 128).  Node 0 is the root: the last committed token, whose K/V
+ * rows are not yet in the cache.  parent[0] == -1 and 0 <= parent[i] < i.
+ * The committed prefix has prefix_len tokens; their K/V rows are rows
+ * [0, prefix_len) of every layer's cache.  Tree node i uses cache row
+ * prefix_len + i until cats_compact_kv moves the accepted rows together.
+ *
+ * Conventions shared by every entry point
+ *   - Pointers named d_* are DEVICE pointers; the caller owns every buffer.
+ *     The library allocates no device memory and keeps no state besides
+ *     function attributes set once per process.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous,
+ *     never synchronise and never copy to the host (except the *_host entry
+ *     point, which says so).
+ *   - Weights are bf16 in nn.Linear layout [out_features][in_features],
+ *     row-major; norm gains are bf16 [hidden].  16-bit tensors are raw bf16.
+ *   - Return value: CATS_OK or a negative cats_status for problems the host
+ *     can see (null pointer, T out of range, unsupported shape, short
+ *     workspace, misaligned pointer); nothing is launched in that case.
+ *   - Problems only the device can see (malformed parent array, a bounded wait
+ *     that expired) are written with atomicMin into *d_status (an int32 the
+ *     caller zeroes once); kernels then finish without touching memory out of
+ *     bounds.  Kernels never trap.
+ *   - Rounding contract: the residual stream and the logits are fp32; GEMM
+ *     inputs (normalised hidden states, q, attention output, SwiGLU output)
+ *     and the K/V cache are bf16, each rounded once from fp32; all sums,
+ *     softmax, norms, SiLU and RoPE are computed in fp32.
+ */
+#ifndef CATS_H_
+#define CATS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CATS_MAX_TREE 128
+
+typedef enum {
+    CATS_OK = 0,
+    CATS_ERR_INVALID_ARG = -1,
+    CATS_ERR_BAD_TREE = -2,
+    CATS_ERR_UNSUPPORTED = -3,
+    CATS_ERR_WORKSPACE = -4,
+    CATS_ERR_CUDA = -5,
+    CATS_ERR_TIMEOUT = -6,
+    CATS_ERR_UNIMPLEMENTED = -7
+} cats_status;
+
+/* Decoder shape (LLaMA-2 / Vicuna family, the paper's target models): RMSNorm,
+ * rotary embeddings with rotate-half pairing, multi-head attention with
+ * n_kv_heads == n_heads, SwiGLU MLP, no biases.  head_dim must be 64 or 128,
+ * hidden and n_heads*head_dim multiples of 64, ffn a multiple of 8. */
+typedef struct {
+    int32_t hidden, n_heads, head_dim, ffn, vocab, n_layers, max_seq;
+    float rms_eps, rope_base;
+} cats_model_cfg;
+
+/* Device pointers to one layer's bf16 weights. */
+typedef struct {
+    const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
+} cats_layer_weights;
+
+/* Ancestor mask, depth and position ids of the draft tree ("tree-based
+ * attention mask encoding the main draft sequence and SV correction branches",
+ * Fig. 4; Algorithm 1, mask = T.tree_mask).
+ *   d_parent [T] int32 in.  d_mask [T][2] uint64 out: bit j of row i (word
+ *   j>>6, bit j&63) is set iff j == i or j is an ancestor of i.  d_pos [T]
+ *   int32 out = prefix_len + depth.  d_depth [T] int32 out, may be NULL.
+ * A malformed parent array sets *d_status = CATS_ERR_BAD_TREE; the outputs are
+ * then zero masks and pos = prefix_len. */
+int cats_build_tree_mask(const int32_t *d_parent, int32_t T, int32_t prefix_len, uint64_t *d_mask,
+                         int32_t *d_pos, int32_t *d_depth, int32_t *d_status, void *stream);
+
+/* Hidden states of the tree tokens from the embedding table (Algorithm 1,
+ * T.hidden_states, for a forward that starts at layer 1).
+ *   d_embed [vocab][hidden] bf16, d_tokens [T] int32 -> d_resid [T][hidden] fp32.
+ * Token ids outside [0, vocab) set CATS_ERR_INVALID_ARG in *d_status and read row 0. */
+int cats_embed_tokens(const void *d_embed, const int32_t *d_tokens, int32_t T, int32_t hidden, int32_t vocab,
+                      float *d_resid, int32_t *d_status, void *stream);
+
+/* Bytes of scratch cats_verify_layer / cats_lm_head_argmax / cats_tree_attention
+ * need for trees of up to T nodes over prefixes of up to max_prefix tokens.
+ * The workspace must be 1024-byte aligned. */
+size_t cats_workspace_bytes(const cats_model_cfg *cfg, int32_t T, int32_t max_prefix);
+
+/* One decoder layer over the T tree nodes under the tree mask (Algorithm 1,
+ * Stage 3: H_tgt <- M_{L_SV+1:L_total}(T.hidden_states, mask, KV_M); "a single
+ * batched forward pass under the corresponding tree attention mask").
+ *   d_resid [T][hidden] fp32, in/out: the residual stream.
+ *   d_kcache/d_vcache: THIS layer's caches, bf16 [max_seq][n_heads*head_dim];
+ *     rows [0,prefix_len) are read, rows prefix_len+i are written (k rotated).
+ *   d_mask, d_pos: from cats_build_tree_mask.
+ */
+int cats_verify_layer(const cats_model_cfg *cfg, const cats_layer_weights *w, float *d_resid, void *d_kcache,
+                      void *d_vcache, const uint64_t *d_mask, const int32_t *d_pos, int32_t T,
+                      int32_t prefix_len, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
+
+/* Tree-masked attention alone: node i of every head attends to cache rows
+ * [0,prefix_len) and to row prefix_len+j iff bit j of d_mask[i] is set
+ * (Fig. 4, tree attention mask; softmax(q.k * scale) v).
+ *   d_q [T][n_heads][head_dim] bf16 (already rotated); d_k/d_v bf16 with
+ *   kv_row_stride_elems elements between rows, head h at column h*head_dim;
+ *   d_out [T][n_heads][head_dim] bf16. */
+int cats_tree_attention(const void *d_q, const void *d_k, const void *d_v, const uint64_t *d_mask, int32_t T,
+                        int32_t prefix_len, int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems,
+                        float scale, void *d_out, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
+
+/* Final norm, LM head and per-node argmax (Algorithm 1: p_tgt <-
+ * softmax(H(H_tgt)); greedy acceptance needs only argmax of the logits).
+ *   d_logits [T][vocab] fp32 out, may be NULL.  d_argmax [T] int32 out: lowest
+ *   vocabulary index attaining the maximum.  d_resid [T][hidden] fp32 in. */
+int cats_lm_head_argmax(const cats_model_cfg *cfg, const void *d_final_norm, const void *d_w_lm,
+                        const float *d_resid, int32_t T, float *d_logits, int32_t *d_argmax, void *d_ws,
+                        size_t ws_bytes, int32_t *d_status, void *stream);
+
+/* Greedy longest-accepted-path walk and bonus token (Algorithm 1, "Walk the
+ * tree to find the longest accepted prefix"; y_out and the bonus token).
+ * A child is accepted iff its token equals d_argmax at its parent; among equal
+ * sibling tokens the lowest node index wins.
+ *   d_path [T] out: accepted node indices, d_path[0] = 0; *d_path_len >= 1.
+ *   d_out_tokens [T] out: accepted draft tokens, then the bonus token;
+ *   *d_n_out == *d_path_len. */
+int cats_accept_path(const int32_t *d_parent, const int32_t *d_tokens, const int32_t *d_argmax, int32_t T,
+                     int32_t *d_path, int32_t *d_path_len, int32_t *d_out_tokens, int32_t *d_n_out,
+                     int32_t *d_status, void *stream);
+
+/* KV roll-back along the accepted path (Algorithm 1, "Roll back KV_M ... to
+ * length s along the accepted path"): for every layer, K and V, row
+ * prefix_len + d_path[k] moves to row prefix_len + k, in place;
+ * *d_new_len = prefix_len + *d_path_len.  Caches are 16-bit elements laid out
+ * [n_layers][layer_stride_elems]; a row has row_elems elements (multiple of 8).
+ * d_src_rows / d_dst_rows ([T] int32, may be NULL) receive the row indices. */
+int cats_compact_kv(void *d_kcache, void *d_vcache, int32_t n_layers, int64_t layer_stride_elems,
+                    int64_t row_elems, int32_t prefix_len, const int32_t *d_path, const int32_t *d_path_len,
+                    int32_t *d_new_len, int32_t *d_src_rows, int32_t *d_dst_rows, int32_t *d_status,
+                    void *stream);
+
+/* Arguments of a whole verification forward (Stage 3 plus walk and roll-back). */
+typedef struct {
+    const cats_model_cfg *cfg;
+    const cats_layer_weights *layers; /* HOST array of cfg->n_layers structs of device pointers */
+    const void *d_embed;              /* [vocab][hidden] bf16; used when d_hidden_in == NULL */
+    const void *d_final_norm;         /* [hidden] bf16 */
+    const void *d_w_lm;               /* [vocab][hidden] bf16 */
+    void *d_kcache, *d_vcache;        /* [n_layers][max_seq][n_heads*head_dim] bf16 */
+    const float *d_hidden_in;         /* [T][hidden] fp32 or NULL */
+    int32_t T, prefix_len;
+    int32_t compact;                  /* != 0: run cats_compact_kv at the end */
+    /* device outputs, all caller-owned */
+    uint64_t *d_mask;                 /* [T][2] */
+    int32_t *d_pos, *d_depth;         /* [T] */
+    float *d_resid;                   /* [T][hidden] */
+    float *d_logits;                  /* [T][vocab] or NULL */
+    int32_t *d_argmax, *d_path, *d_out_tokens; /* [T] */
+    int32_t *d_scalars;               /* [4]: path_len, n_out, new_len, reserved */
+    void *d_ws;
+    size_t ws_bytes;
+    int32_t *d_status;
+} cats_forward_args;
+
+/* The whole path on device buffers: mask/pos, embedding (or caller's hidden
+ * states), layers [0, n_layers), head + argmax, walk, compaction.  d_parent and
+ * d_tokens are [T] int32 device arrays.  One asynchronous sequence of kernel
+ * launches on `stream`, no host round trip. */
+int cats_verify_forward(const cats_forward_args *a, const int32_t *d_parent, const int32_t *d_tokens,
+                        void *stream);
+
+/* Same, for HOST inputs and outputs: copies h_parent/h_tokens ([T] int32, host)
+ * into d_parent_stage/d_tokens_stage, runs cats_verify_forward, copies back
+ * h_scalars[4] (path_len, n_out, new_len, status), h_out_tokens[T] and
+ * h_path[T], and synchronises the stream before returning. */
+int cats_verify_forward_host(const cats_forward_args *a, const int32_t *h_parent, const int32_t *h_tokens,
+                             int32_t *d_parent_stage, int32_t *d_tokens_stage, int32_t *h_scalars,
+                             int32_t *h_out_tokens, int32_t *h_path, void *stream);
+
+/* Number of kernel launches the last call of this thread issued (for reports). */
+int cats_last_launch_count(void);
+
+const char *cats_status_string(int status);
+int cats_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CATS_H_ */

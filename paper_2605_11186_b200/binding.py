@@ -1,0 +1,227 @@
+"""Thin ctypes binding of ``libcats.so``: argument marshalling only.
+
+Every function takes torch CUDA tensors (used purely as device memory), passes their data pointers and the
+current CUDA stream to the C-ABI entry point of the same name, and raises ``CatsError`` on a negative
+status.  There is no fallback: if the library cannot be loaded, importing this module fails.
+"""
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcats.so")
+
+if not os.path.exists(LIB_PATH):
+    _build.build()
+lib = C.CDLL(LIB_PATH)
+
+MAX_TREE = 128
+
+
+class CatsError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, lib.cats_status_string(status).decode(), status))
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32), ("ffn", C.c_int32),
+                ("vocab", C.c_int32), ("n_layers", C.c_int32), ("max_seq", C.c_int32), ("rms_eps", C.c_float),
+                ("rope_base", C.c_float)]
+
+
+LAYER_FIELDS = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in LAYER_FIELDS]
+
+
+class ForwardArgs(C.Structure):
+    _fields_ = [("cfg", C.POINTER(ModelCfg)), ("layers", C.POINTER(LayerWeights)), ("d_embed", C.c_void_p),
+                ("d_final_norm", C.c_void_p), ("d_w_lm", C.c_void_p), ("d_kcache", C.c_void_p), ("d_vcache", C.c_void_p),
+                ("d_hidden_in", C.c_void_p), ("T", C.c_int32), ("prefix_len", C.c_int32), ("compact", C.c_int32),
+                ("d_mask", C.c_void_p), ("d_pos", C.c_void_p), ("d_depth", C.c_void_p), ("d_resid", C.c_void_p),
+                ("d_logits", C.c_void_p), ("d_argmax", C.c_void_p), ("d_path", C.c_void_p), ("d_out_tokens", C.c_void_p),
+                ("d_scalars", C.c_void_p), ("d_ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("d_status", C.c_void_p)]
+
+
+lib.cats_status_string.restype = C.c_char_p
+lib.cats_status_string.argtypes = [C.c_int]
+lib.cats_version.restype = C.c_int
+lib.cats_last_launch_count.restype = C.c_int
+lib.cats_workspace_bytes.restype = C.c_size_t
+lib.cats_workspace_bytes.argtypes = [C.POINTER(ModelCfg), C.c_int32, C.c_int32]
+_vp, _i32, _i64 = C.c_void_p, C.c_int32, C.c_int64
+lib.cats_build_tree_mask.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
+lib.cats_embed_tokens.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
+lib.cats_verify_layer.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp,
+                                  C.c_size_t, _vp, _vp]
+lib.cats_tree_attention.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, C.c_float, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.cats_lm_head_argmax.argtypes = [C.POINTER(ModelCfg), _vp, _vp, _vp, _i32, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.cats_accept_path.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.cats_compact_kv.argtypes = [_vp, _vp, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.cats_verify_forward.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp]
+lib.cats_verify_forward_host.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.cats_debug_use_plain_gemm.argtypes = [C.c_int]
+lib.cats_debug_use_plain_gemm.restype = None
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        assert t.is_contiguous(), "tensors handed to libcats must be contiguous"
+        return t.data_ptr()
+    return int(t)
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise CatsError(rc, where)
+
+
+def model_cfg(shape, max_seq, n_layers=None) -> ModelCfg:
+    """``shape``: any object with hidden, n_heads, head_dim, ffn, vocab, n_layers, rms_eps, rope_base."""
+    return ModelCfg(shape.hidden, shape.n_heads, shape.head_dim, shape.ffn, shape.vocab,
+                    shape.n_layers if n_layers is None else n_layers, max_seq, shape.rms_eps, shape.rope_base)
+
+
+def layer_weights(w: dict) -> LayerWeights:
+    s = LayerWeights()
+    for n in LAYER_FIELDS:
+        t = w[n]
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous(), n
+        setattr(s, n, t.data_ptr())
+    return s
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def workspace_bytes(cfg: ModelCfg, T: int, max_prefix: int) -> int:
+    return int(lib.cats_workspace_bytes(C.byref(cfg), T, max_prefix))
+
+
+def new_workspace(cfg: ModelCfg, T: int, max_prefix: int, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(cfg, T, max_prefix)
+    if n == 0:
+        raise CatsError(-3, "cats_workspace_bytes")
+    buf = torch.empty(n + 1024, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 1024
+    return buf[off:off + n]
+
+
+def use_plain_gemm(on: bool) -> None:
+    """Bring-up switch: route the projections through the plain CUDA-core GEMM."""
+    lib.cats_debug_use_plain_gemm(1 if on else 0)
+
+
+def last_launch_count() -> int:
+    return int(lib.cats_last_launch_count())
+
+
+def cats_build_tree_mask(parent, prefix_len, mask, pos, depth, status):
+    _check(lib.cats_build_tree_mask(_ptr(parent), parent.numel(), prefix_len, _ptr(mask), _ptr(pos), _ptr(depth),
+                                    _ptr(status), _stream()), "cats_build_tree_mask")
+
+
+def cats_embed_tokens(embed, tokens, resid, status):
+    _check(lib.cats_embed_tokens(_ptr(embed), _ptr(tokens), tokens.numel(), embed.shape[1], embed.shape[0], _ptr(resid),
+                                 _ptr(status), _stream()), "cats_embed_tokens")
+
+
+def cats_verify_layer(cfg, w: LayerWeights, resid, kcache, vcache, mask, pos, T, prefix_len, ws, status):
+    _check(lib.cats_verify_layer(C.byref(cfg), C.byref(w), _ptr(resid), _ptr(kcache), _ptr(vcache), _ptr(mask), _ptr(pos), T,
+                                 prefix_len, _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_verify_layer")
+
+
+def cats_tree_attention(q, k, v, mask, T, prefix_len, n_heads, head_dim, kv_row_stride, scale, out, ws, status):
+    _check(lib.cats_tree_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(mask), T, prefix_len, n_heads, head_dim, kv_row_stride,
+                                   scale, _ptr(out), _ptr(ws), 0 if ws is None else ws.numel(), _ptr(status), _stream()),
+           "cats_tree_attention")
+
+
+def cats_lm_head_argmax(cfg, final_norm, w_lm, resid, T, logits, argmax, ws, status):
+    _check(lib.cats_lm_head_argmax(C.byref(cfg), _ptr(final_norm), _ptr(w_lm), _ptr(resid), T, _ptr(logits), _ptr(argmax),
+                                   _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_lm_head_argmax")
+
+
+def cats_accept_path(parent, tokens, argmax, T, path, path_len, out_tokens, n_out, status):
+    _check(lib.cats_accept_path(_ptr(parent), _ptr(tokens), _ptr(argmax), T, _ptr(path), _ptr(path_len), _ptr(out_tokens),
+                                _ptr(n_out), _ptr(status), _stream()), "cats_accept_path")
+
+
+def cats_compact_kv(kcache, vcache, n_layers, layer_stride, row_elems, prefix_len, path, path_len, new_len, src_rows,
+                    dst_rows, status):
+    _check(lib.cats_compact_kv(_ptr(kcache), _ptr(vcache), n_layers, layer_stride, row_elems, prefix_len, _ptr(path),
+                               _ptr(path_len), _ptr(new_len), _ptr(src_rows), _ptr(dst_rows), _ptr(status), _stream()),
+           "cats_compact_kv")
+
+
+class VerifyForward:
+    """Holds the argument block of ``cats_verify_forward`` for one model / tree size: device buffers for
+    every output plus the workspace, all allocated once here (the library itself allocates nothing)."""
+
+    def __init__(self, shape, model: dict, kcache, vcache, T: int, prefix_len: int, want_logits=True, compact=True,
+                 hidden_in=None):
+        dev = kcache.device
+        self.shape = shape
+        self.T, self.prefix_len = T, prefix_len
+        max_seq = kcache.shape[1]
+        self.cfg = model_cfg(shape, max_seq, n_layers=len(model["layers"]))
+        self._layers = (LayerWeights * max(1, len(model["layers"])))()
+        for l, w in enumerate(model["layers"]):
+            self._layers[l] = layer_weights(w)
+        self.model = model
+        self.kcache, self.vcache = kcache, vcache
+        self.mask = torch.zeros((T, 2), dtype=torch.int64, device=dev)
+        self.pos = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.depth = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.resid = torch.zeros((T, shape.hidden), dtype=torch.float32, device=dev)
+        self.logits = torch.zeros((T, shape.vocab), dtype=torch.float32, device=dev) if want_logits else None
+        self.argmax = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.path = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.out_tokens = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.scalars = torch.zeros(4, dtype=torch.int32, device=dev)
+        self.status = new_status(dev)
+        self.ws = new_workspace(self.cfg, T, prefix_len, dev)
+        self.hidden_in = hidden_in
+        self.parent_stage = torch.zeros(T, dtype=torch.int32, device=dev)
+        self.tokens_stage = torch.zeros(T, dtype=torch.int32, device=dev)
+        a = ForwardArgs()
+        a.cfg = C.pointer(self.cfg)
+        a.layers = C.cast(self._layers, C.POINTER(LayerWeights))
+        a.d_embed = _ptr(model.get("embed"))
+        a.d_final_norm = _ptr(model["final_norm"])
+        a.d_w_lm = _ptr(model["w_lm"])
+        a.d_kcache, a.d_vcache = _ptr(kcache), _ptr(vcache)
+        a.d_hidden_in = _ptr(hidden_in)
+        a.T, a.prefix_len, a.compact = T, prefix_len, 1 if compact else 0
+        a.d_mask, a.d_pos, a.d_depth, a.d_resid = _ptr(self.mask), _ptr(self.pos), _ptr(self.depth), _ptr(self.resid)
+        a.d_logits, a.d_argmax, a.d_path = _ptr(self.logits), _ptr(self.argmax), _ptr(self.path)
+        a.d_out_tokens, a.d_scalars = _ptr(self.out_tokens), _ptr(self.scalars)
+        a.d_ws, a.ws_bytes, a.d_status = _ptr(self.ws), self.ws.numel(), _ptr(self.status)
+        self.args = a
+
+    def set_prefix_len(self, prefix_len: int):
+        self.prefix_len = prefix_len
+        self.args.prefix_len = prefix_len
+
+    def run(self, d_parent, d_tokens):
+        """cats_verify_forward on device inputs; asynchronous on the current stream."""
+        _check(lib.cats_verify_forward(C.byref(self.args), _ptr(d_parent), _ptr(d_tokens), _stream()), "cats_verify_forward")
+
+    def run_host(self, h_parent, h_tokens, h_scalars, h_out_tokens, h_path):
+        """cats_verify_forward_host: host (ideally pinned) int32 tensors in and out; synchronises."""
+        _check(lib.cats_verify_forward_host(C.byref(self.args), _ptr(h_parent), _ptr(h_tokens), _ptr(self.parent_stage),
+                                            _ptr(self.tokens_stage), _ptr(h_scalars), _ptr(h_out_tokens), _ptr(h_path),
+                                            _stream()), "cats_verify_forward_host")

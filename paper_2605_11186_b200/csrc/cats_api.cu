@@ -1,0 +1,366 @@
+// C-ABI layer of libcats: argument checks, workspace layout, and the launch sequence of the
+// tree-verification forward.  See include/cats.h for the contract of every entry point.
+#include <cstring>
+
+#include "cats_kernels.cuh"
+
+namespace cats {
+
+thread_local int g_launch_count = 0;
+thread_local bool g_call_boundary = true;
+
+namespace {
+
+constexpr int kMaxSplits = 8;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Workspace {
+    uint16_t *xn, *q, *o, *act;
+    float* part;
+    size_t part_stride;
+    float2* rope;
+    float *attn_o, *attn_ml;
+    float* pmax;
+    int32_t* pidx;
+    float* scratch;
+    size_t bytes;
+};
+
+int attn_split_bound(int nh) { int b = 296 / nh; return b < 1 ? 1 : b; }
+
+// Carves the workspace; with base == nullptr only the size is computed.
+Workspace carve(const cats_model_cfg* c, int T, void* base) {
+    Workspace w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return (uint8_t*)base + o; };
+    const int D = c->n_heads * c->head_dim;
+    const int tpad = (T + 15) / 16 * 16;
+    w.xn = (uint16_t*)take((size_t)T * c->hidden * 2);
+    w.q = (uint16_t*)take((size_t)T * D * 2);
+    w.o = (uint16_t*)take((size_t)T * D * 2);
+    w.act = (uint16_t*)take((size_t)T * c->ffn * 2);
+    w.part_stride = (size_t)T * c->hidden;
+    w.part = (float*)take((size_t)kMaxSplits * w.part_stride * 4);
+    w.rope = (float2*)take((size_t)T * (c->head_dim / 2) * sizeof(float2));
+    size_t ns = attn_split_bound(c->n_heads);
+    w.attn_o = (float*)take((size_t)c->n_heads * ns * tpad * c->head_dim * 4);
+    w.attn_ml = (float*)take((size_t)c->n_heads * ns * tpad * 2 * 4);
+    int vt = (c->vocab + 127) / 128;
+    w.pmax = (float*)take((size_t)vt * 128 * 4);
+    w.pidx = (int32_t*)take((size_t)vt * 128 * 4);
+    size_t widest = (size_t)3 * D;
+    if ((size_t)2 * c->ffn > widest) widest = (size_t)2 * c->ffn;
+    if ((size_t)c->vocab > widest) widest = c->vocab;
+    if ((size_t)c->hidden > widest) widest = c->hidden;
+    w.scratch = (float*)take((size_t)T * widest * 4);
+    w.bytes = off;
+    return w;
+}
+
+int check_cfg(const cats_model_cfg* c) {
+    if (!c) return CATS_ERR_INVALID_ARG;
+    if (c->hidden < 64 || c->n_heads < 1 || c->ffn < 8 || c->max_seq < 1) return CATS_ERR_INVALID_ARG;
+    if (c->head_dim != 64 && c->head_dim != 128) return CATS_ERR_UNSUPPORTED;
+    if (c->hidden % 64 || (c->n_heads * c->head_dim) % 64 || c->ffn % 8) return CATS_ERR_UNSUPPORTED;
+    if (c->hidden > 16384) return CATS_ERR_UNSUPPORTED;
+    return CATS_OK;
+}
+
+inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+
+int split_for(int n_out, int K) {
+    int tiles = (n_out + 127) / 128;
+    int n_kb = (K + 63) / 64;
+    int s = 148 / tiles;
+    if (s < 1) s = 1;
+    if (s > kMaxSplits) s = kMaxSplits;
+    if (s > n_kb) s = n_kb;
+    if (g_use_plain_gemm) s = 1;
+    int per = (n_kb + s - 1) / s;
+    return (n_kb + per - 1) / per;
+}
+
+#define CATS_CUDA(expr)                              \
+    do {                                             \
+        cudaError_t e__ = (expr);                    \
+        if (e__ != cudaSuccess) return CATS_ERR_CUDA; \
+    } while (0)
+
+cudaError_t run_gemm(const GemmProblem& p, const Workspace& ws, cudaStream_t st) {
+    if (g_use_plain_gemm) return launch_gemm_plain(p, ws.scratch, st);
+    return launch_gemm(p, st);
+}
+
+// One decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still
+// to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
+// sums this layer's down projection left pending (>0) or a negative status.
+int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
+               void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
+               int32_t* d_status, cudaStream_t st) {
+    const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
+    CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
+                             ws.rope, c->head_dim, c->rope_base, st));
+    GemmProblem g = {};
+    g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
+    g.W[0] = w->wq; g.W[1] = w->wk; g.W[2] = w->wv; g.X = ws.xn; g.n_splits = 1;
+    g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
+    g.d_status = d_status;
+    CATS_CUDA(run_gemm(g, ws, st));
+
+    AttnProblem a = {};
+    a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
+    a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.part_o = ws.attn_o; a.part_ml = ws.attn_ml;
+    a.d_status = d_status;
+    attn_plan(a);
+    CATS_CUDA(launch_tree_attention(a, st));
+
+    g = GemmProblem{};
+    g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
+    g.n_splits = split_for(H, D); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
+    CATS_CUDA(run_gemm(g, ws, st));
+    CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, g.n_splits, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
+                             nullptr, c->head_dim, c->rope_base, st));
+
+    g = GemmProblem{};
+    g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate; g.W[1] = w->w_up; g.X = ws.xn;
+    g.n_splits = 1; g.act_out = ws.act; g.d_status = d_status;
+    CATS_CUDA(run_gemm(g, ws, st));
+
+    g = GemmProblem{};
+    g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
+    g.n_splits = split_for(H, F); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
+    CATS_CUDA(run_gemm(g, ws, st));
+    return g.n_splits;
+}
+
+int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm, float* resid, const float* copy_from,
+              int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
+    const int H = c->hidden, V = c->vocab;
+    // scratch doubles as the fp32 residual when the caller's buffer is read-only
+    CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
+                             nullptr, c->head_dim, c->rope_base, st));
+    GemmProblem g = {};
+    g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn; g.n_splits = 1;
+    g.logits = logits; g.pmax = ws.pmax; g.pidx = ws.pidx; g.d_status = d_status;
+    CATS_CUDA(run_gemm(g, ws, st));
+    CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, st));
+    return CATS_OK;
+}
+
+int check_tree_args(int T, int P) {
+    if (T < 1 || T > CATS_MAX_TREE || P < 0) return CATS_ERR_INVALID_ARG;
+    return CATS_OK;
+}
+
+}  // namespace
+}  // namespace cats
+
+using namespace cats;
+
+extern "C" {
+
+int cats_version(void) { return 100; }
+
+const char* cats_status_string(int s) {
+    switch (s) {
+        case CATS_OK: return "ok";
+        case CATS_ERR_INVALID_ARG: return "invalid argument";
+        case CATS_ERR_BAD_TREE: return "malformed tree (parent array)";
+        case CATS_ERR_UNSUPPORTED: return "unsupported shape";
+        case CATS_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case CATS_ERR_CUDA: return "CUDA runtime error";
+        case CATS_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case CATS_ERR_UNIMPLEMENTED: return "not implemented";
+        default: return "unknown status";
+    }
+}
+
+int cats_last_launch_count(void) { return g_launch_count; }
+
+/* Bring-up switch, not part of the public header: 1 routes the projections through the plain
+ * CUDA-core GEMM instead of the tcgen05 kernel. */
+void cats_debug_use_plain_gemm(int on) { g_use_plain_gemm = on ? 1 : 0; }
+
+size_t cats_workspace_bytes(const cats_model_cfg* cfg, int32_t T, int32_t max_prefix) {
+    (void)max_prefix;
+    if (check_cfg(cfg) != CATS_OK || T < 1 || T > CATS_MAX_TREE) return 0;
+    return carve(cfg, T, nullptr).bytes;
+}
+
+int cats_build_tree_mask(const int32_t* d_parent, int32_t T, int32_t prefix_len, uint64_t* d_mask, int32_t* d_pos,
+                         int32_t* d_depth, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_parent || !d_mask || !d_pos || !d_status) return CATS_ERR_INVALID_ARG;
+    int rc = check_tree_args(T, prefix_len);
+    if (rc) return rc;
+    CATS_CUDA(launch_mask_pos(d_parent, T, prefix_len, d_mask, d_pos, d_depth, d_status, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
+int cats_embed_tokens(const void* d_embed, const int32_t* d_tokens, int32_t T, int32_t hidden, int32_t vocab, float* d_resid,
+                      int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_embed || !d_tokens || !d_resid || !d_status) return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE || hidden < 8 || hidden % 8 || vocab < 1) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_embed, 16) || misaligned(d_resid, 16)) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_embed(d_embed, d_tokens, T, hidden, vocab, d_resid, d_status, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
+int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, float* d_resid, void* d_kcache, void* d_vcache,
+                      const uint64_t* d_mask, const int32_t* d_pos, int32_t T, int32_t prefix_len, void* d_ws, size_t ws_bytes,
+                      int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    int rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!w || !d_resid || !d_kcache || !d_vcache || !d_mask || !d_pos || !d_ws || !d_status) return CATS_ERR_INVALID_ARG;
+    if (!w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->mlp_norm || !w->w_gate || !w->w_up || !w->w_down)
+        return CATS_ERR_INVALID_ARG;
+    rc = check_tree_args(T, prefix_len);
+    if (rc) return rc;
+    if (prefix_len + T > cfg->max_seq) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(d_resid, 16) || misaligned(d_kcache, 16) || misaligned(d_vcache, 16)) return CATS_ERR_INVALID_ARG;
+    const void* ws_ptrs[] = {w->wq, w->wk, w->wv, w->wo, w->w_gate, w->w_up, w->w_down, w->attn_norm, w->mlp_norm};
+    for (const void* p : ws_ptrs) if (misaligned(p, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, d_status, st);
+    if (pending < 0) return pending;
+    CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
+                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, st));
+    return CATS_OK;
+}
+
+int cats_tree_attention(const void* d_q, const void* d_k, const void* d_v, const uint64_t* d_mask, int32_t T, int32_t prefix_len,
+                        int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems, float scale, void* d_out, void* d_ws,
+                        size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_q || !d_k || !d_v || !d_mask || !d_out || !d_status) return CATS_ERR_INVALID_ARG;
+    int rc = check_tree_args(T, prefix_len);
+    if (rc) return rc;
+    if (n_heads < 1) return CATS_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return CATS_ERR_UNSUPPORTED;
+    if (kv_row_stride_elems < (int64_t)n_heads * head_dim || kv_row_stride_elems % 8) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_q, 16) || misaligned(d_k, 16) || misaligned(d_v, 16) || misaligned(d_out, 4)) return CATS_ERR_INVALID_ARG;
+    AttnProblem a = {};
+    a.q = d_q; a.k = d_k; a.v = d_v; a.mask = d_mask; a.T = T; a.prefix_len = prefix_len; a.nh = n_heads; a.hd = head_dim;
+    a.kv_stride = kv_row_stride_elems; a.scale = scale; a.out = d_out; a.d_status = d_status;
+    size_t need = attn_plan(a);
+    if (need > 0) {
+        if (!d_ws || misaligned(d_ws, 16) || ws_bytes < need) return CATS_ERR_WORKSPACE;
+        int tpad = (T + 15) / 16 * 16;
+        a.part_o = (float*)d_ws;
+        a.part_ml = a.part_o + (size_t)n_heads * a.n_splits * tpad * head_dim;
+    }
+    CATS_CUDA(launch_tree_attention(a, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
+int cats_lm_head_argmax(const cats_model_cfg* cfg, const void* d_final_norm, const void* d_w_lm, const float* d_resid, int32_t T,
+                        float* d_logits, int32_t* d_argmax, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    int rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!d_final_norm || !d_w_lm || !d_resid || !d_argmax || !d_ws || !d_status) return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE || cfg->vocab < 1) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(d_resid, 16) || misaligned(d_w_lm, 16) || misaligned(d_final_norm, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    // the caller's residual is read-only here: normalise a copy held in the scratch area
+    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, 0, d_logits, d_argmax, ws, d_status, (cudaStream_t)stream);
+}
+
+int cats_accept_path(const int32_t* d_parent, const int32_t* d_tokens, const int32_t* d_argmax, int32_t T, int32_t* d_path,
+                     int32_t* d_path_len, int32_t* d_out_tokens, int32_t* d_n_out, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_parent || !d_tokens || !d_argmax || !d_path || !d_path_len || !d_out_tokens || !d_n_out || !d_status)
+        return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_walk(d_parent, d_tokens, d_argmax, T, d_path, d_path_len, d_out_tokens, d_n_out, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
+int cats_compact_kv(void* d_kcache, void* d_vcache, int32_t n_layers, int64_t layer_stride_elems, int64_t row_elems,
+                    int32_t prefix_len, const int32_t* d_path, const int32_t* d_path_len, int32_t* d_new_len, int32_t* d_src_rows,
+                    int32_t* d_dst_rows, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_kcache || !d_vcache || !d_path || !d_path_len || !d_status) return CATS_ERR_INVALID_ARG;
+    if (n_layers < 1 || row_elems < 8 || row_elems % 8 || layer_stride_elems % 8 || prefix_len < 0) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_kcache, 16) || misaligned(d_vcache, 16)) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_compact(d_kcache, d_vcache, n_layers, layer_stride_elems, row_elems, prefix_len, d_path, d_path_len,
+                             d_new_len, d_src_rows, d_dst_rows, d_status, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
+int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, const int32_t* d_tokens, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!a || !d_parent || !d_tokens) return CATS_ERR_INVALID_ARG;
+    const cats_model_cfg* c = a->cfg;
+    int rc = check_cfg(c);
+    if (rc) return rc;
+    if (!a->layers || !a->d_final_norm || !a->d_w_lm || !a->d_kcache || !a->d_vcache || !a->d_mask || !a->d_pos || !a->d_resid ||
+        !a->d_argmax || !a->d_path || !a->d_out_tokens || !a->d_scalars || !a->d_ws || !a->d_status)
+        return CATS_ERR_INVALID_ARG;
+    if (!a->d_hidden_in && !a->d_embed) return CATS_ERR_INVALID_ARG;
+    rc = check_tree_args(a->T, a->prefix_len);
+    if (rc) return rc;
+    if (a->prefix_len + a->T > c->max_seq || c->n_layers < 0 || c->vocab < 1) return CATS_ERR_INVALID_ARG;
+    if (misaligned(a->d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(a->d_resid, 16) || misaligned(a->d_kcache, 16) || misaligned(a->d_vcache, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(c, a->T, a->d_ws);
+    if (ws.bytes > a->ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int T = a->T, P = a->prefix_len;
+    const size_t lstride = (size_t)c->max_seq * c->n_heads * c->head_dim;
+
+    CATS_CUDA(launch_mask_pos(d_parent, T, P, a->d_mask, a->d_pos, a->d_depth, a->d_status, st));
+    const float* copy_from = a->d_hidden_in;
+    if (!copy_from) CATS_CUDA(launch_embed(a->d_embed, d_tokens, T, c->hidden, c->vocab, a->d_resid, a->d_status, st));
+    int pending = 0;
+    for (int l = 0; l < c->n_layers; ++l) {
+        pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
+                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, a->d_status, st);
+        if (pending < 0) return pending;
+    }
+    rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T, pending, a->d_logits,
+                   a->d_argmax, ws, a->d_status, st);
+    if (rc) return rc;
+    CATS_CUDA(launch_walk(d_parent, d_tokens, a->d_argmax, T, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
+    if (a->compact)
+        CATS_CUDA(launch_compact(a->d_kcache, a->d_vcache, c->n_layers, (long long)lstride, (long long)c->n_heads * c->head_dim, P,
+                                 a->d_path, a->d_scalars + 0, a->d_scalars + 2, nullptr, nullptr, a->d_status, st));
+    return CATS_OK;
+}
+
+int cats_verify_forward_host(const cats_forward_args* a, const int32_t* h_parent, const int32_t* h_tokens, int32_t* d_parent_stage,
+                             int32_t* d_tokens_stage, int32_t* h_scalars, int32_t* h_out_tokens, int32_t* h_path, void* stream) {
+    if (!a || !h_parent || !h_tokens || !d_parent_stage || !d_tokens_stage || !h_scalars || !h_out_tokens || !h_path)
+        return CATS_ERR_INVALID_ARG;
+    if (a->T < 1 || a->T > CATS_MAX_TREE) return CATS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t nb = (size_t)a->T * sizeof(int32_t);
+    CATS_CUDA(cudaMemcpyAsync(d_parent_stage, h_parent, nb, cudaMemcpyHostToDevice, st));
+    CATS_CUDA(cudaMemcpyAsync(d_tokens_stage, h_tokens, nb, cudaMemcpyHostToDevice, st));
+    int rc = cats_verify_forward(a, d_parent_stage, d_tokens_stage, stream);
+    if (rc) return rc;
+    CATS_CUDA(cudaMemcpyAsync(h_scalars, a->d_scalars, 3 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CATS_CUDA(cudaMemcpyAsync(h_scalars + 3, a->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CATS_CUDA(cudaMemcpyAsync(h_out_tokens, a->d_out_tokens, nb, cudaMemcpyDeviceToHost, st));
+    CATS_CUDA(cudaMemcpyAsync(h_path, a->d_path, nb, cudaMemcpyDeviceToHost, st));
+    CATS_CUDA(cudaStreamSynchronize(st));
+    return CATS_OK;
+}
+
+}  // extern "C"

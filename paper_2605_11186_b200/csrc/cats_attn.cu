@@ -1,0 +1,351 @@
+// Tree-masked attention of the T draft-tree nodes against the KV prefix plus their own ancestors.
+//
+// Split-KV: CTA (split, head) streams its range of cache rows in blocks of 64 through a double
+// buffered cp.async pipeline (128-bit loads), keeps Q [T_pad][hd] in shared memory, and computes
+// S = Q K^T and O += P V with bf16 tensor-core MMAs (fp32 accumulation, online softmax in fp32 with
+// warp-shuffle row reductions).  Prefix rows need no mask; rows >= prefix_len test bit (row - prefix)
+// of the node's 128-bit ancestor mask held in shared memory.  Warps are laid out as (16-row query
+// tile) x (slice of the 64-row block), so small trees still use every warp.  Partial (m, l, O) per
+// split go to the workspace and k_attn_combine merges them by log-sum-exp; with a single split the
+// CTA writes the final bf16 output itself.
+#include "cats_kernels.cuh"
+
+namespace cats {
+
+constexpr int kAttnThreads = 256;
+constexpr int kKvBlock = 64;
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// byte offset of 16-byte chunk `chunk` of row `row` in a [rows][HD] bf16 tile with XOR swizzle
+template <int HD>
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+    return (uint32_t)(row * (HD * 2) + ((chunk ^ (row & 7)) << 4));
+}
+
+struct AttnDev {
+    const uint16_t *q, *k, *v;
+    const uint64_t* mask;
+    int T, P, nh, n_mt, kvg, n_splits, bps;
+    long long kv_stride;
+    float scale_log2;
+    uint16_t* out;
+    float* part_o;
+    float* part_ml;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) {
+    extern __shared__ __align__(128) uint8_t sm[];
+    constexpr int ROWB = HD * 2;                 // bytes per tile row
+    constexpr int NCH = HD / 8;                  // 16-byte chunks per row
+    constexpr int KS = HD / 16;                  // k-steps of Q K^T
+    constexpr int NT = HD / 8;                   // n-tiles of the output
+    uint8_t* q_s = sm;                                           // [n_mt*16][HD]
+    uint8_t* kv_s = q_s + (size_t)p.n_mt * 16 * ROWB;            // 2 buffers x (K [64][HD], V [64][HD])
+    uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + 2 * 2 * kKvBlock * ROWB);   // [n_mt*16][2]
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x, h = blockIdx.y;
+    const int S = p.P + p.T;
+    const int c_begin = split * p.bps * kKvBlock;
+    const int c_end = min(S, c_begin + p.bps * kKvBlock);
+    const int nb = (c_end - c_begin + kKvBlock - 1) / kKvBlock;
+    const int mt = warp % p.n_mt, g = warp / p.n_mt;
+    const bool active = g < p.kvg;
+    const int R = kKvBlock / p.kvg;              // rows of each block this warp's group handles
+    const int Tpad = p.n_mt * 16;
+
+    auto load_kv = [&](int b, int buf) {
+        uint8_t* ks = kv_s + (size_t)buf * 2 * kKvBlock * ROWB;
+        uint8_t* vs = ks + kKvBlock * ROWB;
+        int r0 = c_begin + b * kKvBlock;
+        for (int e = threadIdx.x; e < kKvBlock * NCH; e += kAttnThreads) {
+            int r = e / NCH, ch = e % NCH;
+            int row = r0 + r;
+            uint32_t off = tile_off<HD>(r, ch);
+            if (row < c_end) {
+                size_t gofs = (size_t)row * p.kv_stride + (size_t)h * HD + ch * 8;
+                cp_async16(ks + off, p.k + gofs);
+                cp_async16(vs + off, p.v + gofs);
+            } else {
+                *reinterpret_cast<uint4*>(ks + off) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vs + off) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+
+    pdl_launch_dependents();
+    // the first block can be requested before the previous kernel has finished if it lies in the prefix
+    const bool early = (c_begin + kKvBlock <= p.P);
+    if (early) load_kv(0, 0);
+    pdl_wait();
+    for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
+        int r = e / NCH, ch = e % NCH;
+        uint32_t off = tile_off<HD>(r, ch);
+        if (r < p.T) cp_async16(q_s + off, p.q + ((size_t)r * p.nh + h) * HD + ch * 8);
+        else *reinterpret_cast<uint4*>(q_s + off) = make_uint4(0, 0, 0, 0);
+    }
+    for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) mask_s[e] = (e < p.T * 2) ? p.mask[e] : 0ull;
+    if (!early && nb > 0) load_kv(0, 0);
+    cp_async_commit();
+
+    uint32_t qf[KS][4];
+    float o[NT][4];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const int row_a = mt * 16 + (lane >> 2), row_b = row_a + 8;   // the two query rows this thread owns
+
+    for (int b = 0; b < nb; ++b) {
+        if (b + 1 < nb) {
+            load_kv(b + 1, (b + 1) & 1);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        if (b == 0 && active) {
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                int r = mt * 16 + (lane & 15), ch = ks * 2 + (lane >> 4);
+                ldmatrix_x4(smem_u32(q_s + tile_off<HD>(r, ch)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
+            }
+        }
+        if (active) {
+            const uint8_t* ks_s = kv_s + (size_t)(b & 1) * 2 * kKvBlock * ROWB;
+            const uint8_t* vs_s = ks_s + kKvBlock * ROWB;
+            const int rbase = g * R;                              // first row of this warp's slice in the block
+            const int cbase = c_begin + b * kKvBlock + rbase;     // its global cache row
+            // 16 rows of the slice at a time: S = Q K^T (16 x 16), mask, online softmax, O += P V
+            for (int sub = 0; sub < R; sub += 16) {
+                if (cbase + sub >= c_end) break;
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    uint32_t b0, b1, b2, b3;
+                    int r = rbase + sub + (lane & 7) + ((lane >> 4) << 3), ch = ks * 2 + ((lane >> 3) & 1);
+                    ldmatrix_x4(smem_u32(ks_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
+                    mma_bf16_16816(s0, qf[ks], b0, b1);
+                    mma_bf16_16816(s1, qf[ks], b2, b3);
+                }
+                // visibility of the 4+4 scores this thread holds
+                float sc[8];
+                {
+                    const uint64_t ma0 = mask_s[row_a * 2], ma1 = mask_s[row_a * 2 + 1];
+                    const uint64_t mb0 = mask_s[row_b * 2], mb1 = mask_s[row_b * 2 + 1];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        int nt = e >> 2, ee = e & 3;
+                        int col = cbase + sub + nt * 8 + (lane & 3) * 2 + (ee & 1);
+                        bool rowb = (ee >> 1) != 0;
+                        bool vis;
+                        if (col < p.P) vis = true;
+                        else if (col >= S) vis = false;
+                        else {
+                            int j = col - p.P;
+                            uint64_t w = rowb ? (j < 64 ? mb0 : mb1) : (j < 64 ? ma0 : ma1);
+                            vis = (w >> (j & 63)) & 1ull;
+                        }
+                        float v = (nt ? s1[ee] : s0[ee]) * p.scale_log2;
+                        sc[e] = vis ? v : -INFINITY;
+                    }
+                }
+                float mx_a = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[4], sc[5]));
+                float mx_b = fmaxf(fmaxf(sc[2], sc[3]), fmaxf(sc[6], sc[7]));
+                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+                mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+                mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+                float mn_a = fmaxf(m_run[0], mx_a), mn_b = fmaxf(m_run[1], mx_b);
+                float ref_a = (mn_a == -INFINITY) ? 0.f : mn_a, ref_b = (mn_b == -INFINITY) ? 0.f : mn_b;
+                float corr_a = exp2f(m_run[0] - ref_a), corr_b = exp2f(m_run[1] - ref_b);
+                m_run[0] = mn_a; m_run[1] = mn_b;
+                float pr[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) pr[e] = exp2f(sc[e] - (((e & 3) >> 1) ? ref_b : ref_a));
+                l_run[0] = l_run[0] * corr_a + pr[0] + pr[1] + pr[4] + pr[5];
+                l_run[1] = l_run[1] * corr_b + pr[2] + pr[3] + pr[6] + pr[7];
+#pragma unroll
+                for (int j = 0; j < NT; ++j) { o[j][0] *= corr_a; o[j][1] *= corr_a; o[j][2] *= corr_b; o[j][3] *= corr_b; }
+                uint32_t pa[4] = {pack_bf16x2(pr[0], pr[1]), pack_bf16x2(pr[2], pr[3]), pack_bf16x2(pr[4], pr[5]),
+                                  pack_bf16x2(pr[6], pr[7])};
+#pragma unroll
+                for (int j = 0; j < NT; j += 2) {
+                    uint32_t b0, b1, b2, b3;
+                    int r = rbase + sub + (lane & 15), ch = j + (lane >> 4);
+                    ldmatrix_x4_trans(smem_u32(vs_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
+                    mma_bf16_16816(o[j], pa, b0, b1);
+                    mma_bf16_16816(o[j + 1], pa, b2, b3);
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- merge the warps that share a query tile, then write the split's partial (or final) result ----
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
+    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
+    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
+    float* mrg_o = reinterpret_cast<float*>(kv_s);              // [8 warps][16][HD], aliases the KV buffers
+    float* mrg_ml = reinterpret_cast<float*>(q_s);              // [8 warps][16][2], aliases Q (no longer needed)
+    if (active && g > 0) {
+        float* wo = mrg_o + (size_t)warp * 16 * HD;
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+            int col = j * 8 + (lane & 3) * 2;
+            *reinterpret_cast<float2*>(wo + (lane >> 2) * HD + col) = make_float2(o[j][0], o[j][1]);
+            *reinterpret_cast<float2*>(wo + ((lane >> 2) + 8) * HD + col) = make_float2(o[j][2], o[j][3]);
+        }
+        if ((lane & 3) == 0) {
+            float* wm = mrg_ml + (size_t)warp * 32;
+            wm[(lane >> 2) * 2] = m_run[0]; wm[(lane >> 2) * 2 + 1] = l_run[0];
+            wm[((lane >> 2) + 8) * 2] = m_run[1]; wm[((lane >> 2) + 8) * 2 + 1] = l_run[1];
+        }
+    }
+    __syncthreads();
+    if (active && g == 0) {
+        float M[2] = {m_run[0], m_run[1]};
+        for (int gg = 1; gg < p.kvg; ++gg) {
+            const float* wm = mrg_ml + (size_t)(gg * p.n_mt + mt) * 32;
+            M[0] = fmaxf(M[0], wm[(lane >> 2) * 2]);
+            M[1] = fmaxf(M[1], wm[((lane >> 2) + 8) * 2]);
+        }
+        float ref[2] = {M[0] == -INFINITY ? 0.f : M[0], M[1] == -INFINITY ? 0.f : M[1]};
+        float w0[2] = {exp2f(m_run[0] - ref[0]), exp2f(m_run[1] - ref[1])};
+        float L[2] = {l_run[0] * w0[0], l_run[1] * w0[1]};
+#pragma unroll
+        for (int j = 0; j < NT; ++j) { o[j][0] *= w0[0]; o[j][1] *= w0[0]; o[j][2] *= w0[1]; o[j][3] *= w0[1]; }
+        for (int gg = 1; gg < p.kvg; ++gg) {
+            int ow = gg * p.n_mt + mt;
+            const float* wm = mrg_ml + (size_t)ow * 32;
+            const float* wo = mrg_o + (size_t)ow * 16 * HD;
+            float wa = exp2f(wm[(lane >> 2) * 2] - ref[0]), wb = exp2f(wm[((lane >> 2) + 8) * 2] - ref[1]);
+            L[0] += wm[(lane >> 2) * 2 + 1] * wa;
+            L[1] += wm[((lane >> 2) + 8) * 2 + 1] * wb;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                int col = j * 8 + (lane & 3) * 2;
+                float2 va = *reinterpret_cast<const float2*>(wo + (lane >> 2) * HD + col);
+                float2 vb = *reinterpret_cast<const float2*>(wo + ((lane >> 2) + 8) * HD + col);
+                o[j][0] += va.x * wa; o[j][1] += va.y * wa; o[j][2] += vb.x * wb; o[j][3] += vb.y * wb;
+            }
+        }
+        if (p.n_splits == 1) {
+            float ia = 1.f / L[0], ib = 1.f / L[1];
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                int col = j * 8 + (lane & 3) * 2;
+                if (row_a < p.T)
+                    *reinterpret_cast<uint32_t*>(p.out + ((size_t)row_a * p.nh + h) * HD + col) = pack_bf16x2(o[j][0] * ia, o[j][1] * ia);
+                if (row_b < p.T)
+                    *reinterpret_cast<uint32_t*>(p.out + ((size_t)row_b * p.nh + h) * HD + col) = pack_bf16x2(o[j][2] * ib, o[j][3] * ib);
+            }
+        } else {
+            float* po = p.part_o + ((size_t)h * p.n_splits + split) * Tpad * HD;
+            float* pml = p.part_ml + ((size_t)h * p.n_splits + split) * Tpad * 2;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+                int col = j * 8 + (lane & 3) * 2;
+                *reinterpret_cast<float2*>(po + (size_t)row_a * HD + col) = make_float2(o[j][0], o[j][1]);
+                *reinterpret_cast<float2*>(po + (size_t)row_b * HD + col) = make_float2(o[j][2], o[j][3]);
+            }
+            if ((lane & 3) == 0) {
+                pml[row_a * 2] = M[0]; pml[row_a * 2 + 1] = L[0];
+                pml[row_b * 2] = M[1]; pml[row_b * 2 + 1] = L[1];
+            }
+        }
+    }
+}
+
+// out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One CTA per (node, head), hd threads.
+__global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                                      int n_splits, int Tpad, int nh, int hd, uint16_t* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
+    float M = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[(((size_t)h * n_splits + s) * Tpad + t) * 2]);
+    float L = 0.f, acc = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        size_t base = ((size_t)h * n_splits + s) * Tpad + t;
+        float w = exp2f(part_ml[base * 2] - M);
+        L += part_ml[base * 2 + 1] * w;
+        if (d < hd) acc += part_o[base * hd + d] * w;
+    }
+    if (d < hd) out[((size_t)t * nh + h) * hd + d] = float_to_bf16_bits(acc / L);
+}
+
+size_t attn_plan(AttnProblem& p) {
+    int S = p.prefix_len + p.T;
+    int blocks = (S + kKvBlock - 1) / kKvBlock;
+    int tpad = ((p.T + 15) / 16) * 16;
+    int by_ctas = 296 / p.nh;
+    if (by_ctas < 1) by_ctas = 1;
+    int min_bps = tpad / kKvBlock;
+    if (min_bps < 1) min_bps = 1;
+    int by_traffic = (blocks + min_bps - 1) / min_bps;
+    int ns = by_ctas < by_traffic ? by_ctas : by_traffic;
+    if (ns < 1) ns = 1;
+    int bps = (blocks + ns - 1) / ns;
+    ns = (blocks + bps - 1) / bps;
+    p.n_splits = ns;
+    p.blocks_per_split = bps;
+    return ns > 1 ? (size_t)p.nh * ns * tpad * (p.hd + 2) * sizeof(float) : 0;
+}
+
+cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 120 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 120 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    AttnDev d;
+    d.q = (const uint16_t*)p.q; d.k = (const uint16_t*)p.k; d.v = (const uint16_t*)p.v;
+    d.mask = p.mask;
+    d.T = p.T; d.P = p.prefix_len; d.nh = p.nh;
+    d.n_mt = (p.T + 15) / 16;
+    d.kvg = 8 / d.n_mt;
+    if (d.kvg > 4) d.kvg = 4;
+    if (d.kvg == 3) d.kvg = 2;
+    d.n_splits = p.n_splits; d.bps = p.blocks_per_split;
+    d.kv_stride = p.kv_stride;
+    d.scale_log2 = p.scale * 1.4426950408889634f;
+    d.out = (uint16_t*)p.out;
+    d.part_o = p.part_o; d.part_ml = p.part_ml;
+    int tpad = d.n_mt * 16;
+    size_t merge = (size_t)8 * 16 * p.hd * 4;                       // aliases the KV buffers
+    size_t kv = (size_t)2 * 2 * kKvBlock * p.hd * 2;
+    size_t qbytes = (size_t)tpad * p.hd * 2;
+    if (qbytes < 8 * 32 * 4) qbytes = 8 * 32 * 4;                   // the (m, l) merge area aliases Q
+    size_t smem = qbytes + (kv > merge ? kv : merge) + (size_t)tpad * 16;
+    cudaError_t e;
+    if (p.hd == 128) e = launch_pdl(k_tree_attn<128>, dim3(p.n_splits, p.nh), dim3(kAttnThreads), smem, st, d);
+    else e = launch_pdl(k_tree_attn<64>, dim3(p.n_splits, p.nh), dim3(kAttnThreads), smem, st, d);
+    if (e != cudaSuccess || p.n_splits == 1) return e;
+    return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
+                      p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out);
+}
+
+}  // namespace cats

@@ -1,0 +1,114 @@
+// Internal interface between the C-ABI layer (cats_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda.h>
+
+#include "cats_common.cuh"
+
+namespace cats {
+
+// Counts launches issued by the calling thread (reported through cats_last_launch_count).
+extern thread_local int g_launch_count;
+// Set at the top of every public entry point: the first kernel of a call is launched with full
+// stream ordering, so nothing a call does before its griddepcontrol.wait (weight and KV-prefix
+// prefetch) can overlap work issued by earlier calls.
+extern thread_local bool g_call_boundary;
+
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the
+// stream is still draining; every kernel calls griddepcontrol.wait before touching dependent data.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_call_boundary ? 0 : 1;
+    g_call_boundary = false;
+    ++g_launch_count;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---- small kernels ---------------------------------------------------------------------------
+cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64_t* mask, int32_t* pos, int32_t* depth,
+                            int32_t* d_status, cudaStream_t st);
+cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int vocab, float* resid, int32_t* d_status,
+                         cudaStream_t st);
+cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
+                           const void* gain, int T, int H, float eps, void* xn, const int32_t* pos, float2* rope, int hd,
+                           float rope_base, cudaStream_t st);
+cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
+                                 cudaStream_t st);
+cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
+                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, cudaStream_t st);
+cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_stride, long long row_elems, int prefix_len,
+                           const int32_t* path, const int32_t* path_len, int32_t* new_len, int32_t* src_rows,
+                           int32_t* dst_rows, int32_t* d_status, cudaStream_t st);
+
+// ---- skinny weight-streaming GEMM ----------------------------------------------------------------
+// Y^T[n_out, T] = W[n_out, K] * X^T[K, T]: weight rows are the MMA's M dimension (128 per tile), the
+// tree nodes its N dimension (T padded to a multiple of 16).
+enum GemmEpilogue : int {
+    EPI_PARTIAL = 0,  // fp32 split-K partial sums  part[split][t][n_out]
+    EPI_QKV = 1,      // RoPE on q and k, bf16 q out, k/v appended to the cache rows prefix_len + t
+    EPI_SWIGLU = 2,   // tile = 64 gate rows + 64 up rows -> a[t][f] = bf16(silu(gate) * up)
+    EPI_LMHEAD = 3    // optional fp32 logits, per-tile (max, lowest index) per node
+};
+
+struct GemmProblem {
+    int epi;
+    int T;            // tree nodes
+    int K;            // reduction length (in_features)
+    int n_out;        // output features of ONE weight matrix (QKV: n_heads*head_dim; SwiGLU: ffn)
+    int n_mats;       // 1, or 3 for QKV, or 2 for SwiGLU
+    const void* W[3]; // device weight matrices [n_out][K] bf16
+    const void* X;    // device activations [T][K] bf16
+    int n_splits;     // split-K factor (EPI_PARTIAL only)
+    // epilogue operands
+    float* part;           // EPI_PARTIAL: [n_splits][T][n_out]
+    size_t part_stride;    //   elements between splits
+    void* q_out;           // EPI_QKV: [T][n_out] bf16
+    void* kcache;          //   [max_seq][n_out] bf16 (this layer)
+    void* vcache;
+    const float2* rope;    //   [T][head_dim/2] (cos, sin)
+    int head_dim;
+    int prefix_len;
+    void* act_out;         // EPI_SWIGLU: [T][n_out] bf16
+    float* logits;         // EPI_LMHEAD: [T][n_out] fp32 or null
+    float* pmax;           //   [n_tiles][128]
+    int32_t* pidx;
+    int32_t* d_status;
+};
+
+// Number of 128-row tiles the problem has (SwiGLU: tiles of 64 gate + 64 up rows).
+int gemm_num_tiles(const GemmProblem& p);
+cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st);
+// Plain CUDA-core implementation of the same problems, kept for bring-up and cross-checks.
+cudaError_t launch_gemm_plain(const GemmProblem& p, float* scratch, cudaStream_t st);
+extern int g_use_plain_gemm;
+
+// ---- tree attention --------------------------------------------------------------------------------
+struct AttnProblem {
+    const void* q;      // [T][nh][hd] bf16
+    const void* k;      // rows of kv_stride elements, head h at h*hd
+    const void* v;
+    const uint64_t* mask;
+    int T, prefix_len, nh, hd;
+    long long kv_stride;
+    float scale;
+    void* out;          // [T][nh][hd] bf16
+    float* part_o;      // [nh][n_splits][T_pad][hd] fp32
+    float* part_ml;     // [nh][n_splits][T_pad][2]
+    int n_splits;       // filled by attn_plan
+    int blocks_per_split;
+    int32_t* d_status;
+};
+// Chooses the KV split; returns bytes of partial storage needed.
+size_t attn_plan(AttnProblem& p);
+cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st);
+
+}  // namespace cats

@@ -1,0 +1,306 @@
+// Latency-bound kernels of the tree-verification forward: ancestor mask / position ids, embedding
+// gather, RMSNorm (fused with the split-K reduction of the preceding projection and with the RoPE
+// table), argmax reduction, the greedy accepted-path walk and KV compaction.
+#include "cats_kernels.cuh"
+
+namespace cats {
+
+// ---------------------------------------------------------------------------------------------
+// Ancestor mask, depth, position ids.  One CTA of 128 threads; thread i walks from node i to the
+// root, OR-ing one bit per node met.  A malformed parent array (parent[0] != -1, parent[i] outside
+// [0, i)) reports CATS_ERR_BAD_TREE and produces zero masks; the walk is bounded by T steps.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMaxTree) k_mask_pos(const int32_t* __restrict__ parent, int T, int prefix_len,
+                                                        uint64_t* __restrict__ mask, int32_t* __restrict__ pos,
+                                                        int32_t* __restrict__ depth, int32_t* d_status) {
+    __shared__ int32_t sp[kMaxTree];
+    __shared__ int bad;
+    pdl_launch_dependents();
+    pdl_wait();
+    int i = threadIdx.x;
+    if (i == 0) bad = 0;
+    __syncthreads();
+    if (i < T) {
+        int p = parent[i];
+        sp[i] = p;
+        if ((i == 0 && p != -1) || (i > 0 && (p < 0 || p >= i))) bad = 1;
+    }
+    __syncthreads();
+    if (i >= T) return;
+    if (bad) {
+        if (i == 0) report(d_status, CATS_ERR_BAD_TREE);
+        mask[2 * i] = 0;
+        mask[2 * i + 1] = 0;
+        pos[i] = prefix_len;
+        if (depth) depth[i] = 0;
+        return;
+    }
+    uint64_t m0 = 0, m1 = 0;
+    int d = 0, j = i;
+    for (int step = 0; step < T && j >= 0; ++step) {
+        if (j < 64) m0 |= 1ull << j; else m1 |= 1ull << (j - 64);
+        j = sp[j];
+        if (j >= 0) ++d;
+    }
+    mask[2 * i] = m0;
+    mask[2 * i + 1] = m1;
+    pos[i] = prefix_len + d;
+    if (depth) depth[i] = d;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Embedding gather: resid[t][:] = float(E[tokens[t]][:]).  One CTA per token.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_embed(const uint16_t* __restrict__ E, const int32_t* __restrict__ tokens, int H,
+                                               int vocab, float* __restrict__ resid, int32_t* d_status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int t = blockIdx.x;
+    int tok = tokens[t];
+    if (tok < 0 || tok >= vocab) {
+        if (threadIdx.x == 0) report(d_status, CATS_ERR_INVALID_ARG);
+        tok = 0;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(E + (size_t)tok * H);
+    float4* dst = reinterpret_cast<float4*>(resid + (size_t)t * H);
+    for (int c = threadIdx.x; c < H / 8; c += blockDim.x) {
+        uint4 v = src[c];
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float f[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            f[2 * q] = __uint_as_float(w[q] << 16);
+            f[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+        }
+        dst[2 * c] = make_float4(f[0], f[1], f[2], f[3]);
+        dst[2 * c + 1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm, one CTA per tree node.  Before normalising it folds n_part split-K partial sums of the
+// preceding projection into the fp32 residual stream (fixed order, so results are reproducible):
+//   resid[t] (+)= part[0][t] + part[1][t] + ...;   xn[t] = bf16(g * resid[t] * rsqrt(mean(resid[t]^2) + eps)).
+// copy_from (optional): resid[t] starts from copy_from[t] instead of its own contents.
+// rope (optional): also fills the rotary table rope[t][i] = (cos, sin)(pos[t] * base^(-2i/hd)), i < hd/2,
+// evaluated in fp64 so that large positions lose no accuracy.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, const float* __restrict__ copy_from,
+                                                 const float* __restrict__ part, int n_part, size_t part_stride,
+                                                 const uint16_t* __restrict__ gain, int H, float eps,
+                                                 uint16_t* __restrict__ xn, const int32_t* __restrict__ pos,
+                                                 float2* __restrict__ rope, int hd, float rope_base) {
+    extern __shared__ float srow[];  // H floats
+    __shared__ float red[8];
+    pdl_launch_dependents();
+    int t = blockIdx.x;
+    pdl_wait();
+    if (rope != nullptr) {
+        int half = hd / 2;
+        int p = pos[t];
+        for (int i = threadIdx.x; i < half; i += blockDim.x) {
+            double inv_freq = pow((double)rope_base, -2.0 * (double)i / (double)hd);
+            double s, c;
+            sincos((double)p * inv_freq, &s, &c);
+            rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
+        }
+    }
+    const float4* r4 = reinterpret_cast<const float4*>((copy_from ? copy_from : resid) + (size_t)t * H);
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < H / 4; c += blockDim.x) {
+        float4 v = r4[c];
+        for (int s = 0; s < n_part; ++s) {
+            float4 pv = reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H)[c];
+            v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
+        }
+        reinterpret_cast<float4*>(srow)[c] = v;
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    float rs = rsqrtf(tot / (float)H + eps);
+    float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
+    for (int c = threadIdx.x; c < H / 4; c += blockDim.x) {
+        float4 v = reinterpret_cast<float4*>(srow)[c];
+        if (n_part > 0 || copy_from) out4[c] = v;
+        if (xn != nullptr) {
+            uint2 g2 = reinterpret_cast<const uint2*>(gain)[c];
+            float g0 = __uint_as_float(g2.x << 16), g1 = __uint_as_float(g2.x & 0xFFFF0000u);
+            float g2f = __uint_as_float(g2.y << 16), g3 = __uint_as_float(g2.y & 0xFFFF0000u);
+            uint2 o;
+            o.x = pack_bf16x2(g0 * (v.x * rs), g1 * (v.y * rs));
+            o.y = pack_bf16x2(g2f * (v.z * rs), g3 * (v.w * rs));
+            reinterpret_cast<uint2*>(xn + (size_t)t * H)[c] = o;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Argmax over vocabulary tiles: the LM-head GEMM leaves, per 128-row vocabulary tile and node, the
+// tile's maximum and the lowest index attaining it; one warp per node picks the overall winner
+// (lowest index among equal maxima).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_argmax_reduce(const float* __restrict__ pmax, const int32_t* __restrict__ pidx,
+                                                       int n_tiles, int t_stride, int T, int32_t* __restrict__ amax) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int t = blockIdx.x * 4 + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (t >= T) return;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int k = lane; k < n_tiles; k += 32) {
+        float v = pmax[(size_t)k * t_stride + t];
+        int ix = pidx[(size_t)k * t_stride + t];
+        if (v > best || (v == best && ix < bi)) { best = v; bi = ix; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if (lane == 0) amax[t] = bi;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Greedy longest-accepted-path walk, one warp.  At node cur the target wants token argmax[cur];
+// each lane tests four nodes, a ballot plus find-first-set gives the lowest matching child.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) k_walk(const int32_t* __restrict__ parent, const int32_t* __restrict__ tokens,
+                                             const int32_t* __restrict__ amax, int T, int32_t* __restrict__ path,
+                                             int32_t* __restrict__ path_len, int32_t* __restrict__ out_tokens,
+                                             int32_t* __restrict__ n_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int lane = threadIdx.x;
+    int par[4], tok[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        int j = q * 32 + lane;
+        par[q] = j < T ? parent[j] : -2;
+        tok[q] = j < T ? tokens[j] : -1;
+    }
+    int cur = 0, len = 1, no = 0;
+    if (lane == 0) path[0] = 0;
+    for (int step = 0; step < T; ++step) {   // a path has at most T nodes
+        int want = amax[cur];
+        int next = -1;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            unsigned b = __ballot_sync(0xffffffffu, par[q] == cur && tok[q] == want);
+            if (next < 0 && b) next = q * 32 + __ffs(b) - 1;
+        }
+        if (next < 0) break;
+        if (lane == 0) { out_tokens[no] = want; path[len] = next; }
+        ++no; ++len;
+        cur = next;
+    }
+    if (lane == 0) {
+        out_tokens[no] = amax[cur];
+        *path_len = len;
+        *n_out = no + 1;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV compaction.  Each thread owns one 16-byte column slice of one cache (layer, K or V) and moves
+// it for k = 0, 1, ... in order: row prefix+path[k] -> row prefix+k.  path[k] >= k and path is
+// increasing, so a slice never reads a row it has already overwritten, and slices do not interact.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_compact(uint16_t* __restrict__ kc, uint16_t* __restrict__ vc, int n_layers,
+                                                 long long layer_stride, long long row_elems, int prefix_len,
+                                                 const int32_t* __restrict__ path, const int32_t* __restrict__ path_len,
+                                                 int32_t* __restrict__ new_len, int32_t* __restrict__ src_rows,
+                                                 int32_t* __restrict__ dst_rows, int32_t* d_status) {
+    __shared__ int32_t sp[kMaxTree];
+    __shared__ int bad;
+    pdl_launch_dependents();
+    pdl_wait();
+    int n = *path_len;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    if (n < 1 || n > kMaxTree) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) report(d_status, CATS_ERR_INVALID_ARG);
+        return;
+    }
+    for (int k = threadIdx.x; k < n; k += blockDim.x) {
+        int p = path[k];
+        sp[k] = p;
+        if (p < k || p >= kMaxTree || (k > 0 && p <= path[k - 1])) bad = 1;
+    }
+    __syncthreads();
+    if (bad) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) report(d_status, CATS_ERR_INVALID_ARG);
+        return;
+    }
+    if (blockIdx.x == 0) {
+        if (threadIdx.x == 0 && new_len) *new_len = prefix_len + n;
+        for (int k = threadIdx.x; k < n; k += blockDim.x) {
+            if (src_rows) src_rows[k] = prefix_len + sp[k];
+            if (dst_rows) dst_rows[k] = prefix_len + k;
+        }
+    }
+    long long slices_per_row = row_elems / 8;
+    long long total = 2ll * n_layers * slices_per_row;
+    for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < total; s += (long long)gridDim.x * blockDim.x) {
+        long long col = s % slices_per_row;
+        long long lw = s / slices_per_row;
+        int layer = (int)(lw >> 1);
+        uint16_t* base = ((lw & 1) ? vc : kc) + (size_t)layer * layer_stride + (size_t)col * 8;
+        for (int k = 0; k < n; ++k) {
+            int p = sp[k];
+            if (p == k) continue;
+            uint4 v = *reinterpret_cast<const uint4*>(base + (size_t)(prefix_len + p) * row_elems);
+            *reinterpret_cast<uint4*>(base + (size_t)(prefix_len + k) * row_elems) = v;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64_t* mask, int32_t* pos, int32_t* depth,
+                            int32_t* d_status, cudaStream_t st) {
+    return launch_pdl(k_mask_pos, dim3(1), dim3(kMaxTree), 0, st, parent, T, prefix_len, mask, pos, depth, d_status);
+}
+
+cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int vocab, float* resid, int32_t* d_status,
+                         cudaStream_t st) {
+    return launch_pdl(k_embed, dim3(T), dim3(256), 0, st, (const uint16_t*)E, tokens, H, vocab, resid, d_status);
+}
+
+cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
+                           const void* gain, int T, int H, float eps, void* xn, const int32_t* pos, float2* rope, int hd,
+                           float rope_base, cudaStream_t st) {
+    return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
+                      part_stride, (const uint16_t*)gain, H, eps, (uint16_t*)xn, pos, rope, hd, rope_base);
+}
+
+cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
+                                 cudaStream_t st) {
+    return launch_pdl(k_argmax_reduce, dim3((T + 3) / 4), dim3(128), 0, st, pmax, pidx, n_tiles, t_stride, T, amax);
+}
+
+cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
+                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, cudaStream_t st) {
+    return launch_pdl(k_walk, dim3(1), dim3(32), 0, st, parent, tokens, amax, T, path, path_len, out_tokens, n_out);
+}
+
+cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_stride, long long row_elems, int prefix_len,
+                           const int32_t* path, const int32_t* path_len, int32_t* new_len, int32_t* src_rows,
+                           int32_t* dst_rows, int32_t* d_status, cudaStream_t st) {
+    long long total = 2ll * n_layers * (row_elems / 8);
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks < 1) blocks = 1;
+    return launch_pdl(k_compact, dim3(blocks), dim3(256), 0, st, (uint16_t*)kc, (uint16_t*)vc, n_layers, layer_stride,
+                      row_elems, prefix_len, path, path_len, new_len, src_rows, dst_rows, d_status);
+}
+
+}  // namespace cats
