@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the CATS tree-verification forward on B200.
+
+A step is one pass of the whole hot path (ancestor mask / position ids, embedding, 32 decoder layers with
+tree-masked attention, final norm + LM head + argmax, accepted-path walk, KV compaction) over one draft tree
+of T nodes, on a 7B-shaped random-init model with a 512-token KV prefix.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--tree-size T] [--impl ours|reference]
+
+N > 1 (launched under torchrun) runs N independent replicas, one per GPU: the path has no exchange step.
+``--impl reference`` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_11186_b200 import inputs as gen  # noqa: E402
+from paper_2605_11186_b200 import roofline  # noqa: E402
+
+METRIC = "verified tree tokens/sec per forward (7B-shape)"
+UNIT = "tree tokens/s"
+PREFIX = 512
+SWEEP = (16, 32, 64, 128)
+
+
+# --------------------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------------------
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 7:
+                continue
+            try:
+                sm.append(float(c[0]))
+                mx.append(float(c[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def make_device_model(shape, tag, device):
+    """Random-init weights N(0, 0.02) in bf16, generated on the device from the seeded sub-streams."""
+    return gen.make_model(shape, tag, device=device)
+
+
+def plant_tokens(cats, fwd, parent, rank, vocab, seed_key, p_keep=0.7):
+    """Top-k draft tree for the benchmark: child tokens are taken from the model's own top-k logits at each node,
+    level by level (what a top-K drafter produces), with the top-1 withheld with probability 1 - p_keep, so the
+    accepted path has a realistic, varying length.  Input preparation only; runs before the timed region."""
+    T = len(parent)
+    rng = np.random.Generator(np.random.Philox(gen.substream("bench_plant", T, *seed_key)))
+    depth = np.zeros(T, np.int64)
+    for i in range(1, T):
+        depth[i] = depth[parent[i]] + 1
+    tokens = gen.uniform_tokens(T, vocab, "bench_tokens", T)
+    d_parent = torch.from_numpy(parent).cuda()
+    for d in range(int(depth.max())):
+        fwd.run(d_parent, torch.from_numpy(tokens).cuda())
+        torch.cuda.synchronize()
+        for n in np.nonzero(depth == d)[0]:
+            kids = np.nonzero(parent == n)[0]
+            if len(kids) == 0:
+                continue
+            top = torch.topk(fwd.logits[n], len(kids) + 1).indices.cpu().numpy()
+            start = 0 if rng.random() < p_keep else 1
+            for r, c in enumerate(kids):
+                tokens[c] = top[start + r]
+    return tokens
+
+
+def time_steps(fn, steps, warmup, stream):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True)
+    e1 = torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / 1e3
+
+
+# --------------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------------
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2605_11186_b200 import binding as cats
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    shape = gen.LLAMA_7B
+    T = args.tree_size
+    model = make_device_model(shape, ("bench", rank), dev)
+    max_seq = PREFIX + 128
+    kc, vc = gen.make_kv_prefix(shape, shape.n_layers, max_seq, PREFIX, ("bench", rank), device=dev)
+    stream = torch.cuda.current_stream()
+
+    def setup(T_):
+        parent, srank = gen.tree_topk_shape(T_, gen.topk_k_for(T_))
+        fwd = cats.VerifyForward(shape, model, kc, vc, T_, PREFIX, want_logits=True, compact=True)
+        tokens = plant_tokens(cats, fwd, parent, srank, shape.vocab, (rank,))
+        fwd_t = cats.VerifyForward(shape, model, kc, vc, T_, PREFIX, want_logits=False, compact=True)
+        return parent, tokens, fwd_t
+
+    def graph_of(fwd, d_parent, d_tokens):
+        g = torch.cuda.CUDAGraph()
+        fwd.run(d_parent, d_tokens)           # warm: sets function attributes outside the capture
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g):
+            fwd.run(d_parent, d_tokens)
+        return g
+
+    def measure(T_, steps, warmup, with_breakdown):
+        parent, tokens, fwd = setup(T_)
+        d_parent, d_tokens = torch.from_numpy(parent).cuda(), torch.from_numpy(tokens).cuda()
+        launches = None
+        if args.no_graph:
+            def step():
+                fwd.run(d_parent, d_tokens)
+        else:
+            g = graph_of(fwd, d_parent, d_tokens)
+            step = g.replay
+        fwd.run(d_parent, d_tokens)
+        launches = cats.last_launch_count()
+        torch.cuda.synchronize()
+        sec = time_steps(step, steps, warmup, stream)
+        status = int(fwd.status.item())
+        n_out = int(fwd.scalars[1].item())
+        res = dict(T=T_, sec_per_step=sec / steps, launches=launches, status=status, accepted=n_out)
+        if with_breakdown:
+            # per-stage device time: the same forward with only some stages enabled (GEMM time is data independent)
+            bd = {}
+            for name, mask in (("gemm_only", 0b1101010), ("attention_only", 0b0000100), ("norms_only", 0b0010001)):
+                cats.stage_mask(mask)
+                try:
+                    bd[name] = time_steps(lambda: fwd.run(d_parent, d_tokens), max(3, steps // 4), 2, stream) / max(3, steps // 4)
+                finally:
+                    cats.stage_mask(0x7f)
+            res["breakdown"] = bd
+        return res, fwd, parent, tokens
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    main, fwd, parent, tokens = measure(T, args.steps, args.warmup, with_breakdown=(rank == 0))
+    if world > 1:
+        torch.distributed.barrier()
+    clocks = sampler.stop() if sampler else None
+    if main["status"] != 0:
+        raise RuntimeError("device status %d" % main["status"])
+
+    # e2e: the host entry point, pinned host buffers in and out, every step
+    hp = torch.from_numpy(parent).pin_memory()
+    ht = torch.from_numpy(tokens).pin_memory()
+    hs = torch.zeros(4, dtype=torch.int32).pin_memory()
+    ho = torch.zeros(T, dtype=torch.int32).pin_memory()
+    hpath = torch.zeros(T, dtype=torch.int32).pin_memory()
+    for _ in range(args.warmup):
+        fwd.run_host(hp, ht, hs, ho, hpath)
+    if world > 1:
+        torch.distributed.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        fwd.run_host(hp, ht, hs, ho, hpath)
+    e2e_sec = time.perf_counter() - t0
+
+    sweep = {}
+    if rank == 0 and not args.no_sweep:
+        for T_ in SWEEP:
+            if T_ == T:
+                r = main
+            else:
+                r, _, _, _ = measure(T_, max(5, args.steps // 2), 3, with_breakdown=False)
+            b = roofline.forward_bytes(shape, PREFIX, T_)
+            sweep[str(T_)] = {"tok_s": T_ / r["sec_per_step"], "ms": r["sec_per_step"] * 1e3,
+                              "gbs": b / r["sec_per_step"] / 1e9, "accepted": r["accepted"]}
+
+    sec = torch.tensor([main["sec_per_step"], e2e_sec / args.steps], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(sec, op=torch.distributed.ReduceOp.MAX)
+    sec_step, sec_e2e = float(sec[0]), float(sec[1])
+    if rank != 0:
+        return None
+    peak, peak_kind = measured_peaks()
+    fb = roofline.forward_bytes(shape, PREFIX, T)
+    wb = roofline.gemm_weight_bytes(shape)
+    gemm_sec = main["breakdown"]["gemm_only"]
+    n_gemm = roofline.gemm_launches(shape)
+    out = {
+        "metric": METRIC, "value": world * T / sec_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "cfg3: 32-layer 7B-shaped verification forward + LM head (vocab 32000), prefix 512, "
+                               "top-k draft tree of T=%d nodes, greedy walk + KV compaction" % T,
+                   "tree_nodes": T, "prefix_len": PREFIX, "replicas": world, "cuda_graph": not args.no_graph,
+                   "l2": "inputs_larger_than_l2 (13.5 GB of weights per step)", "accepted_tokens_per_step": main["accepted"]},
+        "e2e": {"value": world * T / sec_e2e, "unit": UNIT, "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 16 + 2 * T * 4},
+        "gpu_launches": main["launches"] * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "k_gemm_tc (all %d projection launches of a forward)" % n_gemm,
+                     "achieved": wb / n_gemm / (gemm_sec / n_gemm) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": wb / gemm_sec / 1e9 / peak, "peak_kind": peak_kind, "traffic": None,
+                     "bytes_per_launch": wb / n_gemm, "us_per_launch": gemm_sec / n_gemm * 1e6,
+                     "forward_achieved": fb / sec_step / 1e9, "forward_frac": fb / sec_step / 1e9 / peak,
+                     "forward_frac_of_8TBs": fb / sec_step / 8e12},
+        "breakdown_ms": {k: v * 1e3 for k, v in main["breakdown"].items()},
+        "sweep": sweep,
+    }
+    return out
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------------------------------
+
+def oracle_sample(T, n_layers_sample, repeats=1):
+    """Times the oracle, as it stands, on a bounded sample of the workload: the first n_layers_sample layers plus the
+    LM head; the layer time is scaled to 32 layers.  Returns (seconds per full forward, cores, description)."""
+    import oracle
+    shape = gen.LLAMA_7B
+    m = shape.replace(n_layers=n_layers_sample)
+    model = gen.make_model(m, ("bench", 0), device="cpu")
+    max_seq = PREFIX + 128
+    kc, vc = gen.make_kv_prefix(m, n_layers_sample, max_seq, PREFIX, ("bench", 0))
+    parent, _ = gen.tree_topk_shape(T, gen.topk_k_for(T))
+    tokens = gen.uniform_tokens(T, m.vocab, "bench_tokens", T)
+    layers = [{k: gen.bf16_bits(v) for k, v in w.items()} for w in model["layers"]]
+    cfg = oracle.RefCfg(m.hidden, m.n_heads, m.head_dim, m.ffn, m.vocab, n_layers_sample, max_seq, m.rms_eps, m.rope_base)
+    cfg0 = oracle.RefCfg(m.hidden, m.n_heads, m.head_dim, m.ffn, m.vocab, 0, max_seq, m.rms_eps, m.rope_base)
+    emb, fn, wl = gen.bf16_bits(model["embed"]), gen.bf16_bits(model["final_norm"]), gen.bf16_bits(model["w_lm"])
+    r_k, r_v = kc.float().numpy(), vc.float().numpy()
+    best_full, best_head = None, None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        _, amax, _, _ = oracle.verify_forward(cfg, layers, emb, fn, wl, parent, tokens, PREFIX, r_k, r_v, want_logits=False)
+        path, _ = oracle.accept_path(parent, tokens, amax)
+        oracle.compact_kv(r_k.copy(), r_v.copy(), PREFIX, path)
+        t_full = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        oracle.verify_forward(cfg0, [], emb, fn, wl, parent, tokens, PREFIX, r_k[:0], r_v[:0], want_logits=False)
+        t_head = time.perf_counter() - t0
+        best_full = t_full if best_full is None else min(best_full, t_full)
+        best_head = t_head if best_head is None else min(best_head, t_head)
+    t_layers = max(best_full - best_head, 1e-9)
+    sec = t_layers * (shape.n_layers / n_layers_sample) + best_head
+    desc = ("oracle timed on %d of 32 layers + LM head + walk + compaction at T=%d, layer time scaled x%d"
+            % (n_layers_sample, T, shape.n_layers // n_layers_sample))
+    return sec, oracle.n_threads(), desc
+
+
+def run_reference(args):
+    T = args.tree_size
+    secs = []
+    cores, desc = None, None
+    for i in range(args.warmup + args.steps):
+        sec, cores, desc = oracle_sample(T, 1)
+        if i >= args.warmup:
+            secs.append(sec)
+    sec = float(np.mean(secs))
+    val = T / sec
+    return {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "cfg3: 32-layer 7B-shaped verification forward + LM head (vocab 32000), prefix 512, "
+                                   "top-k draft tree of T=%d nodes, greedy walk + KV compaction" % T, "tree_nodes": T,
+                       "prefix_len": PREFIX},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--tree-size", type=int, default=64)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="launch every step directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the T in {16,32,64,128} sweep")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    out = run_ours(args, rank, world, local_rank)
+    if rank == 0:
+        if not args.no_cpu_baseline:
+            sec, cores, desc = oracle_sample(args.tree_size, 2)
+            out["cpu_baseline"] = {"value": args.tree_size / sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -125,6 +125,19 @@ def use_plain_gemm(on: bool) -> None:
     lib.cats_debug_use_plain_gemm(1 if on else 0)
 
 
+def stage_mask(mask: int) -> None:
+    """Measurement / bring-up hook: bit i enables stage i of every decoder layer (0 norm1, 1 qkv, 2 attention,
+    3 o-proj, 4 norm2, 5 gate/up, 6 down).  0x7f is normal operation."""
+    lib.cats_debug_stage_mask(C.c_uint(mask))
+
+
+def workspace_layout(cfg: ModelCfg, T: int) -> dict:
+    """Byte offsets of the intermediate buffers inside the workspace (for tests that inspect them)."""
+    out = (C.c_size_t * 6)()
+    _check(lib.cats_debug_workspace_layout(C.byref(cfg), T, out), "cats_debug_workspace_layout")
+    return dict(xn=out[0], q=out[1], o=out[2], act=out[3], part=out[4], part_stride=out[5])
+
+
 def last_launch_count() -> int:
     return int(lib.cats_last_launch_count())
 

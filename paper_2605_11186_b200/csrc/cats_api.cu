@@ -13,6 +13,11 @@ namespace {
 
 constexpr int kMaxSplits = 8;
 
+// Bring-up / measurement hook: bit i enables stage i of a decoder layer (0 norm1, 1 qkv, 2 attention,
+// 3 o-proj, 4 norm2, 5 gate/up, 6 down).  All stages run by default.
+unsigned g_stage_mask = 0x7f;
+inline bool stage_on(int i) { return (g_stage_mask >> i) & 1u; }
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Workspace {
@@ -99,38 +104,40 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
                int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
-    CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                             ws.rope, c->head_dim, c->rope_base, st));
+    if (stage_on(0))
+        CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
+                                 ws.rope, c->head_dim, c->rope_base, st));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wq; g.W[1] = w->wk; g.W[2] = w->wv; g.X = ws.xn; g.n_splits = 1;
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
     g.d_status = d_status;
-    CATS_CUDA(run_gemm(g, ws, st));
+    if (stage_on(1)) CATS_CUDA(run_gemm(g, ws, st));
 
     AttnProblem a = {};
     a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
     a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.part_o = ws.attn_o; a.part_ml = ws.attn_ml;
     a.d_status = d_status;
     attn_plan(a);
-    CATS_CUDA(launch_tree_attention(a, st));
+    if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
     g = GemmProblem{};
     g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
     g.n_splits = split_for(H, D); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    CATS_CUDA(run_gemm(g, ws, st));
-    CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, g.n_splits, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, c->head_dim, c->rope_base, st));
+    if (stage_on(3)) CATS_CUDA(run_gemm(g, ws, st));
+    if (stage_on(4))
+        CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, g.n_splits, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
+                                 nullptr, c->head_dim, c->rope_base, st));
 
     g = GemmProblem{};
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate; g.W[1] = w->w_up; g.X = ws.xn;
     g.n_splits = 1; g.act_out = ws.act; g.d_status = d_status;
-    CATS_CUDA(run_gemm(g, ws, st));
+    if (stage_on(5)) CATS_CUDA(run_gemm(g, ws, st));
 
     g = GemmProblem{};
     g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
     g.n_splits = split_for(H, F); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    CATS_CUDA(run_gemm(g, ws, st));
+    if (stage_on(6)) CATS_CUDA(run_gemm(g, ws, st));
     return g.n_splits;
 }
 
@@ -181,6 +188,24 @@ int cats_last_launch_count(void) { return g_launch_count; }
 /* Bring-up switch, not part of the public header: 1 routes the projections through the plain
  * CUDA-core GEMM instead of the tcgen05 kernel. */
 void cats_debug_use_plain_gemm(int on) { g_use_plain_gemm = on ? 1 : 0; }
+
+/* Bring-up / measurement hooks, not part of the public header.  cats_debug_stage_mask: bit i enables
+ * stage i of every decoder layer (0 norm1, 1 qkv, 2 attention, 3 o-proj, 4 norm2, 5 gate/up, 6 down);
+ * 0x7f restores normal operation.  cats_debug_workspace_layout: byte offsets of the intermediate
+ * buffers inside the workspace: xn, q, o, act, part (fp32 split-K partial sums), and in out[5] the
+ * number of fp32 elements between two partial sums. */
+void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
+int cats_debug_workspace_layout(const cats_model_cfg* cfg, int32_t T, size_t* out) {
+    if (check_cfg(cfg) != CATS_OK || T < 1 || T > CATS_MAX_TREE || !out) return CATS_ERR_INVALID_ARG;
+    Workspace w = carve(cfg, T, nullptr);
+    out[0] = (size_t)((uint8_t*)w.xn - (uint8_t*)nullptr);
+    out[1] = (size_t)((uint8_t*)w.q - (uint8_t*)nullptr);
+    out[2] = (size_t)((uint8_t*)w.o - (uint8_t*)nullptr);
+    out[3] = (size_t)((uint8_t*)w.act - (uint8_t*)nullptr);
+    out[4] = (size_t)((uint8_t*)w.part - (uint8_t*)nullptr);
+    out[5] = w.part_stride;
+    return CATS_OK;
+}
 
 size_t cats_workspace_bytes(const cats_model_cfg* cfg, int32_t T, int32_t max_prefix) {
     (void)max_prefix;

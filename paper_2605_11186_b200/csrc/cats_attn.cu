@@ -186,15 +186,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
                 l_run[1] = l_run[1] * corr_b + pr[2] + pr[3] + pr[6] + pr[7];
 #pragma unroll
                 for (int j = 0; j < NT; ++j) { o[j][0] *= corr_a; o[j][1] *= corr_a; o[j][2] *= corr_b; o[j][3] *= corr_b; }
-                uint32_t pa[4] = {pack_bf16x2(pr[0], pr[1]), pack_bf16x2(pr[2], pr[3]), pack_bf16x2(pr[4], pr[5]),
-                                  pack_bf16x2(pr[6], pr[7])};
+                // The probabilities enter the P V product as bf16 pairs hi + lo (hi = bf16(p), lo = bf16(p - hi)),
+                // so the product carries ~16 mantissa bits of p instead of 8; V is bf16 exactly.
+                uint32_t pa[4], pl[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float h0 = bf16_bits_to_float(float_to_bf16_bits(pr[2 * e]));
+                    float h1 = bf16_bits_to_float(float_to_bf16_bits(pr[2 * e + 1]));
+                    pa[e] = pack_bf16x2(h0, h1);
+                    pl[e] = pack_bf16x2(pr[2 * e] - h0, pr[2 * e + 1] - h1);
+                }
 #pragma unroll
                 for (int j = 0; j < NT; j += 2) {
                     uint32_t b0, b1, b2, b3;
                     int r = rbase + sub + (lane & 15), ch = j + (lane >> 4);
                     ldmatrix_x4_trans(smem_u32(vs_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
                     mma_bf16_16816(o[j], pa, b0, b1);
+                    mma_bf16_16816(o[j], pl, b0, b1);
                     mma_bf16_16816(o[j + 1], pa, b2, b3);
+                    mma_bf16_16816(o[j + 1], pl, b2, b3);
                 }
             }
         }

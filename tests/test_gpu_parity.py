@@ -49,12 +49,13 @@ def dev_model(model):
 
 
 def bf16_ulp_close(got_bf16: torch.Tensor, want_f32: np.ndarray):
-    """Every element within one bf16 ulp (at the larger magnitude) of the oracle's bf16 value."""
+    """Every element within one bf16 ulp (at the larger magnitude) of the oracle's bf16 value, plus 1e-3 absolute
+    for sums that cancel to nearly zero (fp32 accumulation error is absolute, not relative)."""
     g = got_bf16.float().cpu().numpy().astype(np.float64)
     w = want_f32.astype(np.float64)
     mag = np.maximum(np.abs(g), np.abs(w))
     ulp = 2.0 ** (np.floor(np.log2(np.maximum(mag, 1e-30))) - 7)
-    bad = np.abs(g - w) > ulp * 1.001
+    bad = np.abs(g - w) > ulp * 1.001 + 1e-3
     return int(bad.sum()), float(np.abs(g - w).max())
 
 
@@ -358,16 +359,20 @@ def test_config1_planted_trees_accept_paths(cats, cfg1, T, k, seed):
 def test_fused_forward_with_compaction_and_host_entry(cats, cfg1):
     c = cfg1
     m = c["m"]
-    parent, tokens = planted_tree(c["rcfg"], c["nm"], 16, 4, c["root"], c["P"], c["kc"], c["vc"], (0,))
+    nm = c["nm"]
+    for seed in range(20):      # a planted tree whose accepted path has no near-tie, so both sides must agree on it
+        parent, tokens = planted_tree(c["rcfg"], nm, 16, 4, c["root"], c["P"], c["kc"], c["vc"], (seed,))
+        r_k, r_v = c["kc"].copy(), c["vc"].copy()
+        _, amax, margin, _ = oracle.verify_forward(c["rcfg"], nm["layers"], nm["embed"], nm["final_norm"], nm["w_lm"], parent,
+                                                   tokens, c["P"], r_k, r_v)
+        r_path, r_out = oracle.accept_path(parent, tokens, amax)
+        if np.all(margin[r_path] > 2 * TOL) and len(r_path) >= 3:
+            break
+    else:
+        pytest.fail("no planted tree with a clear accepted path")
     dm = dev_model(c["model"])
     kc = torch.from_numpy(c["kc"]).to(torch.bfloat16)
     vc = torch.from_numpy(c["vc"]).to(torch.bfloat16)
-    r_k, r_v = c["kc"].copy(), c["vc"].copy()
-    nm = c["nm"]
-    _, amax, margin, _ = oracle.verify_forward(c["rcfg"], nm["layers"], nm["embed"], nm["final_norm"], nm["w_lm"], parent, tokens,
-                                               c["P"], r_k, r_v)
-    r_path, r_out = oracle.accept_path(parent, tokens, amax)
-    assert np.all(margin[r_path] > TOL)
     rc, r_new, _, _ = oracle.compact_kv(r_k, r_v, c["P"], r_path)
     d_k, d_v = kc.cuda(), vc.cuda()
     fwd = cats.VerifyForward(m, dm, d_k, d_v, 16, c["P"], want_logits=False, compact=True)
