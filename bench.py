@@ -146,7 +146,8 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.set_device(dev)
     shape = gen.LLAMA_7B
     T = args.tree_size
-    model = make_device_model(shape, ("bench", rank), dev)
+    model = cats.pack_model(make_device_model(shape, ("bench", rank), dev), free_source=True)
+    torch.cuda.empty_cache()
     max_seq = PREFIX + 128
     kc, vc = gen.make_kv_prefix(shape, shape.n_layers, max_seq, PREFIX, ("bench", rank), device=dev)
     stream = torch.cuda.current_stream()

@@ -18,8 +18,10 @@
  *   - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous,
  *     never synchronise and never copy to the host (except the *_host entry
  *     point, which says so).
- *   - Weights are bf16 in nn.Linear layout [out_features][in_features],
- *     row-major; norm gains are bf16 [hidden].  16-bit tensors are raw bf16.
+ *   - Projection weights are bf16, handed over in the library's packed layout:
+ *     cats_pack_weights converts nn.Linear matrices [out_features][in_features]
+ *     (row-major) once, at load time.  Norm gains are bf16 [hidden].  16-bit
+ *     tensors are raw bf16.
  *   - Return value: CATS_OK or a negative cats_status for problems the host
  *     can see (null pointer, T out of range, unsupported shape, short
  *     workspace, misaligned pointer); nothing is launched in that case.
@@ -64,10 +66,31 @@ typedef struct {
     float rms_eps, rope_base;
 } cats_model_cfg;
 
-/* Device pointers to one layer's bf16 weights. */
+/* Device pointers to one layer's weights.  attn_norm, mlp_norm: bf16 [hidden].
+ * wqkv: cats_pack_weights of {Wq, Wk, Wv} (layout 0, three matrices [n_heads*head_dim][hidden]);
+ * wo: layout 0 of Wo [hidden][n_heads*head_dim]; w_gate_up: layout 1 of {W_gate, W_up}
+ * ([ffn][hidden] each); w_down: layout 0 of W_down [hidden][ffn]. */
 typedef struct {
-    const void *attn_norm, *wq, *wk, *wv, *wo, *mlp_norm, *w_gate, *w_up, *w_down;
+    const void *attn_norm, *wqkv, *wo, *mlp_norm, *w_gate_up, *w_down;
 } cats_layer_weights;
+
+/* Weight packing.  The projections are bound by reading every weight once per
+ * forward ("every generation step loads the model weights"; Eq. 3-4 count
+ * exactly those bytes), so the library keeps each matrix as a sequence of
+ * 16 KB chunks -- (128-row tile, 64-column block), already in the layout the
+ * tensor cores read from shared memory -- that one SM can stream with plain
+ * contiguous bulk copies.
+ *   layout 0: n_src (1..3) matrices of identical shape [rows][cols] stacked, each
+ *             padded to whole 128-row tiles.
+ *   layout 1: n_src == 2 matrices (gate, up) interleaved as tiles of 64 + 64 rows,
+ *             so that silu(gate)*up is computed inside one tile.
+ * cols must be a multiple of 8; rows/cols beyond the matrix are stored as zeros.
+ * d_src: HOST array of n_src device pointers (bf16, row-major, 16-byte aligned);
+ * d_dst: device buffer of cats_packed_weight_bytes bytes, 1024-byte aligned.
+ * cats_packed_weight_bytes returns 0 for invalid arguments. */
+size_t cats_packed_weight_bytes(int32_t n_src, int32_t layout, int32_t rows, int32_t cols);
+int cats_pack_weights(const void *const *d_src, int32_t n_src, int32_t layout, int32_t rows, int32_t cols,
+                      void *d_dst, void *stream);
 
 /* Ancestor mask, depth and position ids of the draft tree ("tree-based
  * attention mask encoding the main draft sequence and SV correction branches",
@@ -117,7 +140,8 @@ int cats_tree_attention(const void *d_q, const void *d_k, const void *d_v, const
 /* Final norm, LM head and per-node argmax (Algorithm 1: p_tgt <-
  * softmax(H(H_tgt)); greedy acceptance needs only argmax of the logits).
  *   d_logits [T][vocab] fp32 out, may be NULL.  d_argmax [T] int32 out: lowest
- *   vocabulary index attaining the maximum.  d_resid [T][hidden] fp32 in. */
+ *   vocabulary index attaining the maximum.  d_resid [T][hidden] fp32 in.
+ *   d_w_lm: cats_pack_weights (layout 0) of the LM head [vocab][hidden]. */
 int cats_lm_head_argmax(const cats_model_cfg *cfg, const void *d_final_norm, const void *d_w_lm,
                         const float *d_resid, int32_t T, float *d_logits, int32_t *d_argmax, void *d_ws,
                         size_t ws_bytes, int32_t *d_status, void *stream);
@@ -150,7 +174,7 @@ typedef struct {
     const cats_layer_weights *layers; /* HOST array of cfg->n_layers structs of device pointers */
     const void *d_embed;              /* [vocab][hidden] bf16; used when d_hidden_in == NULL */
     const void *d_final_norm;         /* [hidden] bf16 */
-    const void *d_w_lm;               /* [vocab][hidden] bf16 */
+    const void *d_w_lm;               /* packed LM head (layout 0 of [vocab][hidden]) */
     void *d_kcache, *d_vcache;        /* [n_layers][max_seq][n_heads*head_dim] bf16 */
     const float *d_hidden_in;         /* [T][hidden] fp32 or NULL */
     int32_t T, prefix_len;

@@ -46,9 +46,18 @@ typedef struct {
 } cats_ref_layer_weights;
 
 static int g_contract = 1;
+static int g_accum32 = 0;
 
 void cats_ref_set_contract(int on) { g_contract = on ? 1 : 0; }
 int cats_ref_get_contract(void) { return g_contract; }
+
+/* Sensitivity probe, off by default: accumulate the projections' dot products in fp32 (sequential,
+ * ascending k) instead of fp64.  Every bf16 rounding point of the contract is a discontinuity: two
+ * evaluations whose sums differ in the last fp32 bits round a small fraction of the activations to
+ * neighbouring bf16 values, and those one-ulp flips spread through attention and the MLPs.  Running
+ * the oracle both ways measures how far two equally valid evaluations of the same contract drift
+ * apart -- the floor below which no GPU-vs-oracle deviation can be expected to fall. */
+void cats_ref_set_accum32(int on) { g_accum32 = on ? 1 : 0; }
 
 /* ---- bf16 <-> fp32 (round to nearest even) ---------------------------- */
 
@@ -122,6 +131,18 @@ void cats_ref_rmsnorm(const float *x, const uint16_t *g, int32_t T, int32_t H, f
  * in ascending k.  linear_row is compiled for a few vector widths; the order
  * of additions inside each acc[t] is the same in all of them. */
 __attribute__((target_clones("avx512f", "avx2", "default")))
+static void linear_row_f32(const uint16_t *w, int32_t n_in, const double *xT, int32_t T, double *acc) {
+    float facc[CATS_REF_MAX_T];
+    for (int t = 0; t < T; ++t) facc[t] = 0.0f;
+    for (int k = 0; k < n_in; ++k) {
+        float wk = cats_ref_bf16_to_f32(w[k]);
+        const double *xk = xT + (size_t)k * T;
+        for (int t = 0; t < T; ++t) facc[t] += wk * (float)xk[t];
+    }
+    for (int t = 0; t < T; ++t) acc[t] = (double)facc[t];
+}
+
+__attribute__((target_clones("avx512f", "avx2", "default")))
 static void linear_row(const uint16_t *w, int32_t n_in, const double *xT, int32_t T, double *acc) {
     for (int t = 0; t < T; ++t) acc[t] = 0.0;
     for (int k = 0; k < n_in; ++k) {
@@ -139,7 +160,8 @@ void cats_ref_linear(const uint16_t *W, int32_t n_out, int32_t n_in, const doubl
 #pragma omp parallel for schedule(static)
     for (int o = 0; o < n_out; ++o) {
         double acc[CATS_REF_MAX_T];
-        linear_row(W + (size_t)o * n_in, n_in, xT, T, acc);
+        if (g_accum32) linear_row_f32(W + (size_t)o * n_in, n_in, xT, T, acc);
+        else linear_row(W + (size_t)o * n_in, n_in, xT, T, acc);
         for (int t = 0; t < T; ++t) y[(size_t)t * n_out + o] = acc[t];
     }
     free(xT);

@@ -12,7 +12,7 @@ import numpy as np
 from .build import build as _build
 
 __all__ = [
-    "RefCfg", "set_contract", "to_bf16", "from_bf16", "build_tree_mask", "rmsnorm", "linear",
+    "RefCfg", "set_contract", "set_accum32", "to_bf16", "from_bf16", "build_tree_mask", "rmsnorm", "linear",
     "rope_head", "tree_attention", "verify_layer", "embed", "lm_head_argmax", "accept_path",
     "compact_kv", "verify_forward", "n_threads",
 ]
@@ -54,6 +54,11 @@ def n_threads() -> int:
 def set_contract(on: bool) -> None:
     """True: mirror the GPU path's bf16 rounding points.  False: no intermediate rounding."""
     _lib.cats_ref_set_contract(C.c_int(1 if on else 0))
+
+
+def set_accum32(on: bool) -> None:
+    """Sensitivity probe: accumulate the projections in fp32 instead of fp64 (see cats_ref.c)."""
+    _lib.cats_ref_set_accum32(C.c_int(1 if on else 0))
 
 
 _lib.cats_ref_bf16_to_f32.restype = C.c_float

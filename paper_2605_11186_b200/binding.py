@@ -33,7 +33,7 @@ class ModelCfg(C.Structure):
                 ("rope_base", C.c_float)]
 
 
-LAYER_FIELDS = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")
+LAYER_FIELDS = ("attn_norm", "wqkv", "wo", "mlp_norm", "w_gate_up", "w_down")
 
 
 class LayerWeights(C.Structure):
@@ -66,8 +66,9 @@ lib.cats_accept_path.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _
 lib.cats_compact_kv.argtypes = [_vp, _vp, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.cats_verify_forward.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp]
 lib.cats_verify_forward_host.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
-lib.cats_debug_use_plain_gemm.argtypes = [C.c_int]
-lib.cats_debug_use_plain_gemm.restype = None
+lib.cats_packed_weight_bytes.restype = C.c_size_t
+lib.cats_packed_weight_bytes.argtypes = [_i32, _i32, _i32, _i32]
+lib.cats_pack_weights.argtypes = [C.POINTER(C.c_void_p), _i32, _i32, _i32, _i32, _vp, _vp]
 
 
 def _ptr(t):
@@ -94,11 +95,55 @@ def model_cfg(shape, max_seq, n_layers=None) -> ModelCfg:
                     shape.n_layers if n_layers is None else n_layers, max_seq, shape.rms_eps, shape.rope_base)
 
 
+def pack_weights(mats, layout: int) -> torch.Tensor:
+    """cats_pack_weights: ``mats`` is a list of 1-3 bf16 CUDA matrices of identical shape [rows][cols]
+    (nn.Linear layout).  Returns the packed buffer (uint8 CUDA tensor, 1024-byte aligned)."""
+    rows, cols = mats[0].shape
+    for m in mats:
+        assert m.is_cuda and m.dtype == torch.bfloat16 and m.is_contiguous() and tuple(m.shape) == (rows, cols)
+    n = int(lib.cats_packed_weight_bytes(len(mats), layout, rows, cols))
+    if n == 0:
+        raise CatsError(-1, "cats_packed_weight_bytes")
+    buf = torch.empty(n + 1024, dtype=torch.uint8, device=mats[0].device)
+    off = (-buf.data_ptr()) % 1024
+    out = buf[off:off + n]
+    ptrs = (C.c_void_p * len(mats))(*[m.data_ptr() for m in mats])
+    _check(lib.cats_pack_weights(ptrs, len(mats), layout, rows, cols, out.data_ptr(), _stream()), "cats_pack_weights")
+    return out
+
+
+def pack_layer(w: dict) -> dict:
+    """nn.Linear-layout layer weights (wq, wk, wv, wo, w_gate, w_up, w_down, attn_norm, mlp_norm) -> packed layer."""
+    return {"attn_norm": w["attn_norm"].contiguous(), "mlp_norm": w["mlp_norm"].contiguous(),
+            "wqkv": pack_weights([w["wq"], w["wk"], w["wv"]], 0), "wo": pack_weights([w["wo"]], 0),
+            "w_gate_up": pack_weights([w["w_gate"], w["w_up"]], 1), "w_down": pack_weights([w["w_down"]], 0)}
+
+
+def pack_model(model: dict, free_source: bool = False) -> dict:
+    """Packs every projection of a model dict (layers, w_lm); embed and final_norm are kept as they are."""
+    out = {"layers": []}
+    for w in model["layers"]:
+        out["layers"].append(pack_layer(w))
+        if free_source:
+            for k in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down"):
+                w.pop(k, None)
+    for k in ("embed", "final_norm", "shape"):
+        if k in model:
+            out[k] = model[k]
+    if "w_lm" in model:
+        out["w_lm"] = pack_weights([model["w_lm"]], 0)
+        if free_source:
+            model.pop("w_lm")
+    torch.cuda.synchronize()
+    return out
+
+
 def layer_weights(w: dict) -> LayerWeights:
+    """``w``: a packed layer (see pack_layer)."""
     s = LayerWeights()
     for n in LAYER_FIELDS:
         t = w[n]
-        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous(), n
+        assert t.is_cuda and t.is_contiguous(), n
         setattr(s, n, t.data_ptr())
     return s
 
@@ -120,11 +165,6 @@ def new_workspace(cfg: ModelCfg, T: int, max_prefix: int, device="cuda") -> torc
     return buf[off:off + n]
 
 
-def use_plain_gemm(on: bool) -> None:
-    """Bring-up switch: route the projections through the plain CUDA-core GEMM."""
-    lib.cats_debug_use_plain_gemm(1 if on else 0)
-
-
 def stage_mask(mask: int) -> None:
     """Measurement / bring-up hook: bit i enables stage i of every decoder layer (0 norm1, 1 qkv, 2 attention,
     3 o-proj, 4 norm2, 5 gate/up, 6 down).  0x7f is normal operation."""
@@ -133,9 +173,23 @@ def stage_mask(mask: int) -> None:
 
 def workspace_layout(cfg: ModelCfg, T: int) -> dict:
     """Byte offsets of the intermediate buffers inside the workspace (for tests that inspect them)."""
-    out = (C.c_size_t * 6)()
+    out = (C.c_size_t * 8)()
     _check(lib.cats_debug_workspace_layout(C.byref(cfg), T, out), "cats_debug_workspace_layout")
-    return dict(xn=out[0], q=out[1], o=out[2], act=out[3], part=out[4], part_stride=out[5])
+    return dict(xn=out[0], q=out[1], o=out[2], act=out[3], part=out[4], part_stride=out[5], pieces_o=out[6],
+                pieces_down=out[7])
+
+
+def unpack_activation(buf: torch.Tensor, T: int, K: int) -> torch.Tensor:
+    """Reads a packed activation buffer (uint8 view of the workspace) back as a [T][K] bf16 tensor (tests only)."""
+    n_pad = (T + 15) // 16 * 16
+    n_kb = (K + 63) // 64
+    x = buf[:n_kb * n_pad * 128].view(torch.bfloat16).view(n_kb, n_pad // 8, 8, 8, 8)   # kb, row group, row, chunk, elem
+    r = torch.arange(8, device=buf.device)
+    c = torch.arange(8, device=buf.device)
+    phys = (c[None, :] ^ r[:, None])                                                  # [row][logical chunk] -> physical
+    x = torch.gather(x, 3, phys[None, None, :, :, None].expand(n_kb, n_pad // 8, 8, 8, 8))
+    x = x.permute(1, 2, 0, 3, 4).reshape(n_pad, n_kb * 64)
+    return x[:T, :K].contiguous()
 
 
 def last_launch_count() -> int:
@@ -194,7 +248,7 @@ class VerifyForward:
         self._layers = (LayerWeights * max(1, len(model["layers"])))()
         for l, w in enumerate(model["layers"]):
             self._layers[l] = layer_weights(w)
-        self.model = model
+        self.model = model    # packed (see pack_model)
         self.kcache, self.vcache = kcache, vcache
         self.mask = torch.zeros((T, 2), dtype=torch.int64, device=dev)
         self.pos = torch.zeros(T, dtype=torch.int32, device=dev)

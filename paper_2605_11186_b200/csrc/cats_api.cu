@@ -11,7 +11,6 @@ thread_local bool g_call_boundary = true;
 
 namespace {
 
-constexpr int kMaxSplits = 8;
 
 // Bring-up / measurement hook: bit i enables stage i of a decoder layer (0 norm1, 1 qkv, 2 attention,
 // 3 o-proj, 4 norm2, 5 gate/up, 6 down).  All stages run by default.
@@ -21,14 +20,17 @@ inline bool stage_on(int i) { return (g_stage_mask >> i) & 1u; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Workspace {
-    uint16_t *xn, *q, *o, *act;
+    uint8_t *xn, *o, *act;      // packed activation layout
+    uint16_t* q;                // [T][D] row-major
     float* part;
     size_t part_stride;
     float2* rope;
     float *attn_o, *attn_ml;
     float* pmax;
     int32_t* pidx;
-    float* scratch;
+    float* fix_part;
+    int* fix_flags;
+    float* scratch;             // [T][hidden] fp32
     size_t bytes;
 };
 
@@ -41,12 +43,13 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return (uint8_t*)base + o; };
     const int D = c->n_heads * c->head_dim;
     const int tpad = (T + 15) / 16 * 16;
-    w.xn = (uint16_t*)take((size_t)T * c->hidden * 2);
+    auto packed = [&](int K) { return (size_t)((K + 63) / 64) * tpad * 128; };
+    w.xn = take(packed(c->hidden));
     w.q = (uint16_t*)take((size_t)T * D * 2);
-    w.o = (uint16_t*)take((size_t)T * D * 2);
-    w.act = (uint16_t*)take((size_t)T * c->ffn * 2);
+    w.o = take(packed(D));
+    w.act = take(packed(c->ffn));
     w.part_stride = (size_t)T * c->hidden;
-    w.part = (float*)take((size_t)kMaxSplits * w.part_stride * 4);
+    w.part = (float*)take((size_t)kMaxPartSlots * w.part_stride * 4);
     w.rope = (float2*)take((size_t)T * (c->head_dim / 2) * sizeof(float2));
     size_t ns = attn_split_bound(c->n_heads);
     w.attn_o = (float*)take((size_t)c->n_heads * ns * tpad * c->head_dim * 4);
@@ -54,11 +57,9 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     int vt = (c->vocab + 127) / 128;
     w.pmax = (float*)take((size_t)vt * 128 * 4);
     w.pidx = (int32_t*)take((size_t)vt * 128 * 4);
-    size_t widest = (size_t)3 * D;
-    if ((size_t)2 * c->ffn > widest) widest = (size_t)2 * c->ffn;
-    if ((size_t)c->vocab > widest) widest = c->vocab;
-    if ((size_t)c->hidden > widest) widest = c->hidden;
-    w.scratch = (float*)take((size_t)T * widest * 4);
+    w.fix_part = (float*)take((size_t)kGemmCtas * tpad * 128 * 4);
+    w.fix_flags = (int*)take((size_t)kGemmCtas * sizeof(int));
+    w.scratch = (float*)take((size_t)T * c->hidden * 4);
     w.bytes = off;
     return w;
 }
@@ -74,28 +75,11 @@ int check_cfg(const cats_model_cfg* c) {
 
 inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
-int split_for(int n_out, int K) {
-    int tiles = (n_out + 127) / 128;
-    int n_kb = (K + 63) / 64;
-    int s = 148 / tiles;
-    if (s < 1) s = 1;
-    if (s > kMaxSplits) s = kMaxSplits;
-    if (s > n_kb) s = n_kb;
-    if (g_use_plain_gemm) s = 1;
-    int per = (n_kb + s - 1) / s;
-    return (n_kb + per - 1) / per;
-}
-
 #define CATS_CUDA(expr)                              \
     do {                                             \
         cudaError_t e__ = (expr);                    \
         if (e__ != cudaSuccess) return CATS_ERR_CUDA; \
     } while (0)
-
-cudaError_t run_gemm(const GemmProblem& p, const Workspace& ws, cudaStream_t st) {
-    if (g_use_plain_gemm) return launch_gemm_plain(p, ws.scratch, st);
-    return launch_gemm(p, st);
-}
 
 // One decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still
 // to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
@@ -104,53 +88,56 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
                int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
+    const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 ws.rope, c->head_dim, c->rope_base, st));
+                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
-    g.W[0] = w->wq; g.W[1] = w->wk; g.W[2] = w->wv; g.X = ws.xn; g.n_splits = 1;
+    g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
     g.d_status = d_status;
-    if (stage_on(1)) CATS_CUDA(run_gemm(g, ws, st));
+    if (stage_on(1)) CATS_CUDA(launch_gemm(g, st));
 
     AttnProblem a = {};
     a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
-    a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.part_o = ws.attn_o; a.part_ml = ws.attn_ml;
-    a.d_status = d_status;
+    a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.out_packed_npad = tpad;
+    a.part_o = ws.attn_o; a.part_ml = ws.attn_ml; a.d_status = d_status;
     attn_plan(a);
     if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
     g = GemmProblem{};
     g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
-    g.n_splits = split_for(H, D); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    if (stage_on(3)) CATS_CUDA(run_gemm(g, ws, st));
+    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
+    int pieces_o = gemm_plan(g).max_pieces;
+    if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
-        CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, g.n_splits, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                                 nullptr, c->head_dim, c->rope_base, st));
+        CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
+                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
 
     g = GemmProblem{};
-    g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate; g.W[1] = w->w_up; g.X = ws.xn;
-    g.n_splits = 1; g.act_out = ws.act; g.d_status = d_status;
-    if (stage_on(5)) CATS_CUDA(run_gemm(g, ws, st));
+    g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
+    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.act_out = ws.act; g.d_status = d_status;
+    if (stage_on(5)) CATS_CUDA(launch_gemm(g, st));
 
     g = GemmProblem{};
     g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
-    g.n_splits = split_for(H, F); g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    if (stage_on(6)) CATS_CUDA(run_gemm(g, ws, st));
-    return g.n_splits;
+    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
+    int pieces_d = gemm_plan(g).max_pieces;
+    if (stage_on(6)) CATS_CUDA(launch_gemm(g, st));
+    return pieces_d;
 }
 
 int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm, float* resid, const float* copy_from,
               int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, V = c->vocab;
-    // scratch doubles as the fp32 residual when the caller's buffer is read-only
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, c->head_dim, c->rope_base, st));
+                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
-    g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn; g.n_splits = 1;
+    g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
+    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.logits = logits; g.pmax = ws.pmax; g.pidx = ws.pidx; g.d_status = d_status;
-    CATS_CUDA(run_gemm(g, ws, st));
+    CATS_CUDA(launch_gemm(g, st));
     CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, st));
     return CATS_OK;
 }
@@ -185,10 +172,6 @@ const char* cats_status_string(int s) {
 
 int cats_last_launch_count(void) { return g_launch_count; }
 
-/* Bring-up switch, not part of the public header: 1 routes the projections through the plain
- * CUDA-core GEMM instead of the tcgen05 kernel. */
-void cats_debug_use_plain_gemm(int on) { g_use_plain_gemm = on ? 1 : 0; }
-
 /* Bring-up / measurement hooks, not part of the public header.  cats_debug_stage_mask: bit i enables
  * stage i of every decoder layer (0 norm1, 1 qkv, 2 attention, 3 o-proj, 4 norm2, 5 gate/up, 6 down);
  * 0x7f restores normal operation.  cats_debug_workspace_layout: byte offsets of the intermediate
@@ -204,6 +187,11 @@ int cats_debug_workspace_layout(const cats_model_cfg* cfg, int32_t T, size_t* ou
     out[3] = (size_t)((uint8_t*)w.act - (uint8_t*)nullptr);
     out[4] = (size_t)((uint8_t*)w.part - (uint8_t*)nullptr);
     out[5] = w.part_stride;
+    GemmProblem g = {};
+    g.epi = EPI_PARTIAL; g.T = T; g.K = cfg->n_heads * cfg->head_dim; g.n_out = cfg->hidden; g.n_mats = 1;
+    out[6] = (size_t)gemm_plan(g).max_pieces;
+    g.K = cfg->ffn;
+    out[7] = (size_t)gemm_plan(g).max_pieces;
     return CATS_OK;
 }
 
@@ -211,6 +199,24 @@ size_t cats_workspace_bytes(const cats_model_cfg* cfg, int32_t T, int32_t max_pr
     (void)max_prefix;
     if (check_cfg(cfg) != CATS_OK || T < 1 || T > CATS_MAX_TREE) return 0;
     return carve(cfg, T, nullptr).bytes;
+}
+
+size_t cats_packed_weight_bytes(int32_t n_src, int32_t layout, int32_t rows, int32_t cols) {
+    if (n_src < 1 || n_src > 3 || rows < 1 || cols < 1 || (layout != 0 && layout != 1) || (layout == 1 && n_src != 2)) return 0;
+    return packed_weight_bytes(n_src, layout, rows, cols);
+}
+
+int cats_pack_weights(const void* const* d_src, int32_t n_src, int32_t layout, int32_t rows, int32_t cols, void* d_dst,
+                      void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_src || !d_dst || cats_packed_weight_bytes(n_src, layout, rows, cols) == 0) return CATS_ERR_INVALID_ARG;
+    for (int i = 0; i < n_src; ++i)
+        if (!d_src[i] || misaligned(d_src[i], 16)) return CATS_ERR_INVALID_ARG;
+    if (cols % 8 || misaligned(d_dst, 1024)) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_pack_weights(d_src, n_src, layout, rows, cols, d_dst, (cudaStream_t)stream));
+    g_call_boundary = true;
+    return CATS_OK;
 }
 
 int cats_build_tree_mask(const int32_t* d_parent, int32_t T, int32_t prefix_len, uint64_t* d_mask, int32_t* d_pos,
@@ -243,22 +249,22 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     int rc = check_cfg(cfg);
     if (rc) return rc;
     if (!w || !d_resid || !d_kcache || !d_vcache || !d_mask || !d_pos || !d_ws || !d_status) return CATS_ERR_INVALID_ARG;
-    if (!w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->mlp_norm || !w->w_gate || !w->w_up || !w->w_down)
-        return CATS_ERR_INVALID_ARG;
+    if (!w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm || !w->w_gate_up || !w->w_down) return CATS_ERR_INVALID_ARG;
     rc = check_tree_args(T, prefix_len);
     if (rc) return rc;
     if (prefix_len + T > cfg->max_seq) return CATS_ERR_INVALID_ARG;
     if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
     if (misaligned(d_resid, 16) || misaligned(d_kcache, 16) || misaligned(d_vcache, 16)) return CATS_ERR_INVALID_ARG;
-    const void* ws_ptrs[] = {w->wq, w->wk, w->wv, w->wo, w->w_gate, w->w_up, w->w_down, w->attn_norm, w->mlp_norm};
+    const void* ws_ptrs[] = {w->wqkv, w->wo, w->w_gate_up, w->w_down, w->attn_norm, w->mlp_norm};
     for (const void* p : ws_ptrs) if (misaligned(p, 16)) return CATS_ERR_INVALID_ARG;
     Workspace ws = carve(cfg, T, d_ws);
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, d_status, st);
     if (pending < 0) return pending;
-    CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, st));
+    if (stage_on(6))
+        CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
+                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
     return CATS_OK;
 }
 

@@ -46,6 +46,7 @@ struct AttnDev {
     int T, P, nh, n_mt, kvg, n_splits, bps;
     long long kv_stride;
     float scale_log2;
+    int out_npad;        // > 0: out is in the packed activation layout with this many rows per K block
     uint16_t* out;
     float* part_o;
     float* part_ml;
@@ -265,10 +266,17 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 #pragma unroll
             for (int j = 0; j < NT; ++j) {
                 int col = j * 8 + (lane & 3) * 2;
-                if (row_a < p.T)
-                    *reinterpret_cast<uint32_t*>(p.out + ((size_t)row_a * p.nh + h) * HD + col) = pack_bf16x2(o[j][0] * ia, o[j][1] * ia);
-                if (row_b < p.T)
-                    *reinterpret_cast<uint32_t*>(p.out + ((size_t)row_b * p.nh + h) * HD + col) = pack_bf16x2(o[j][2] * ib, o[j][3] * ib);
+                uint8_t* ob = reinterpret_cast<uint8_t*>(p.out);
+                size_t off_a, off_b;
+                if (p.out_npad > 0) {
+                    off_a = packed_act_offset(row_a, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2;
+                    off_b = packed_act_offset(row_b, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2;
+                } else {
+                    off_a = (((size_t)row_a * p.nh + h) * HD + col) * 2;
+                    off_b = (((size_t)row_b * p.nh + h) * HD + col) * 2;
+                }
+                if (row_a < p.T) *reinterpret_cast<uint32_t*>(ob + off_a) = pack_bf16x2(o[j][0] * ia, o[j][1] * ia);
+                if (row_b < p.T) *reinterpret_cast<uint32_t*>(ob + off_b) = pack_bf16x2(o[j][2] * ib, o[j][3] * ib);
             }
         } else {
             float* po = p.part_o + ((size_t)h * p.n_splits + split) * Tpad * HD;
@@ -289,7 +297,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One CTA per (node, head), hd threads.
 __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                      int n_splits, int Tpad, int nh, int hd, uint16_t* __restrict__ out) {
+                                                      int n_splits, int Tpad, int nh, int hd, uint16_t* __restrict__ out,
+                                                      int out_npad) {
     pdl_launch_dependents();
     pdl_wait();
     const int t = blockIdx.x, h = blockIdx.y, d = threadIdx.x;
@@ -302,7 +311,14 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
         L += part_ml[base * 2 + 1] * w;
         if (d < hd) acc += part_o[base * hd + d] * w;
     }
-    if (d < hd) out[((size_t)t * nh + h) * hd + d] = float_to_bf16_bits(acc / L);
+    if (d < hd) {
+        uint16_t v = float_to_bf16_bits(acc / L);
+        if (out_npad > 0)
+            *reinterpret_cast<uint16_t*>(reinterpret_cast<uint8_t*>(out) + packed_act_offset(t, (h * hd + d) >> 3, out_npad) +
+                                         (size_t)(d & 7) * 2) = v;
+        else
+            out[((size_t)t * nh + h) * hd + d] = v;
+    }
 }
 
 size_t attn_plan(AttnProblem& p) {
@@ -343,6 +359,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.kv_stride = p.kv_stride;
     d.scale_log2 = p.scale * 1.4426950408889634f;
     d.out = (uint16_t*)p.out;
+    d.out_npad = p.out_packed_npad;
     d.part_o = p.part_o; d.part_ml = p.part_ml;
     int tpad = d.n_mt * 16;
     size_t merge = (size_t)8 * 16 * p.hd * 4;                       // aliases the KV buffers
@@ -355,7 +372,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     else e = launch_pdl(k_tree_attn<64>, dim3(p.n_splits, p.nh), dim3(kAttnThreads), smem, st, d);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
-                      p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out);
+                      p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
 }
 
 }  // namespace cats

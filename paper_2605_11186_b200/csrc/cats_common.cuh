@@ -38,6 +38,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return (uint32_t)float_to_bf16_bits(lo) | ((uint32_t)float_to_bf16_bits(hi) << 16);
 }
 
+// Byte offset of the 16-byte group holding elements k8*8 .. k8*8+7 of row t inside a packed activation
+// buffer: one chunk of n_pad rows x 64 columns per K block, rows of 128 bytes with the 128-byte swizzle
+// (the shared-memory layout tcgen05.mma reads).  Every producer of a GEMM input writes this layout.
+__host__ __device__ __forceinline__ size_t packed_act_offset(int t, int k8, int n_pad) {
+    int kb = k8 >> 3, c = k8 & 7;
+    return (size_t)kb * n_pad * 128 + (size_t)(t >> 3) * 1024 + (size_t)(t & 7) * 128 + (size_t)((c ^ (t & 7)) << 4);
+}
+
 // ---- programmatic dependent launch ------------------------------------------------------------
 // wait: blocks until every kernel this launch depends on has completed and its writes are visible.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

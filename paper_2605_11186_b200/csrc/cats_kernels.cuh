@@ -39,8 +39,8 @@ cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64
 cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int vocab, float* resid, int32_t* d_status,
                          cudaStream_t st);
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
-                           const void* gain, int T, int H, float eps, void* xn, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, cudaStream_t st);
+                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
+                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
@@ -51,13 +51,17 @@ cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_str
 
 // ---- skinny weight-streaming GEMM ----------------------------------------------------------------
 // Y^T[n_out, T] = W[n_out, K] * X^T[K, T]: weight rows are the MMA's M dimension (128 per tile), the
-// tree nodes its N dimension (T padded to a multiple of 16).
+// tree nodes its N dimension (T padded to a multiple of 16).  W is packed by launch_pack_weights, X is
+// in the packed activation layout (packed_act_offset).
 enum GemmEpilogue : int {
-    EPI_PARTIAL = 0,  // fp32 split-K partial sums  part[split][t][n_out]
+    EPI_PARTIAL = 0,  // fp32 split-K partial sums  part[piece][t][n_out]
     EPI_QKV = 1,      // RoPE on q and k, bf16 q out, k/v appended to the cache rows prefix_len + t
-    EPI_SWIGLU = 2,   // tile = 64 gate rows + 64 up rows -> a[t][f] = bf16(silu(gate) * up)
+    EPI_SWIGLU = 2,   // tile = 64 gate rows + 64 up rows -> a[t][f] = bf16(silu(gate) * up), packed layout
     EPI_LMHEAD = 3    // optional fp32 logits, per-tile (max, lowest index) per node
 };
+
+constexpr int kGemmCtas = 148;      // one persistent CTA per SM
+constexpr int kMaxPartSlots = 8;    // partial-sum slots of EPI_PARTIAL
 
 struct GemmProblem {
     int epi;
@@ -65,31 +69,38 @@ struct GemmProblem {
     int K;            // reduction length (in_features)
     int n_out;        // output features of ONE weight matrix (QKV: n_heads*head_dim; SwiGLU: ffn)
     int n_mats;       // 1, or 3 for QKV, or 2 for SwiGLU
-    const void* W[3]; // device weight matrices [n_out][K] bf16
-    const void* X;    // device activations [T][K] bf16
-    int n_splits;     // split-K factor (EPI_PARTIAL only)
+    const void* W[3]; // W[0]: packed weights (all matrices of the problem in one buffer)
+    const void* X;    // packed activations
+    float* fix_part;  // [kGemmCtas][n_pad][128] fp32: partial tiles of tiles shared by several CTAs
+    int* fix_flags;   // [kGemmCtas], zero between launches
     // epilogue operands
-    float* part;           // EPI_PARTIAL: [n_splits][T][n_out]
-    size_t part_stride;    //   elements between splits
+    float* part;           // EPI_PARTIAL: [pieces][T][n_out]
+    size_t part_stride;    //   elements between slots
     void* q_out;           // EPI_QKV: [T][n_out] bf16
     void* kcache;          //   [max_seq][n_out] bf16 (this layer)
     void* vcache;
     const float2* rope;    //   [T][head_dim/2] (cos, sin)
     int head_dim;
     int prefix_len;
-    void* act_out;         // EPI_SWIGLU: [T][n_out] bf16
+    void* act_out;         // EPI_SWIGLU: packed activations, ceil(n_out/64) K blocks
     float* logits;         // EPI_LMHEAD: [T][n_out] fp32 or null
     float* pmax;           //   [n_tiles][128]
     int32_t* pidx;
     int32_t* d_status;
 };
 
+struct GemmPlan {
+    int units_per_cta;   // (tile, K block) pairs per CTA, contiguous
+    int n_ctas;
+    int max_pieces;      // EPI_PARTIAL: number of partial-sum slots the following reduction must fold
+};
+
 // Number of 128-row tiles the problem has (SwiGLU: tiles of 64 gate + 64 up rows).
 int gemm_num_tiles(const GemmProblem& p);
+GemmPlan gemm_plan(const GemmProblem& p);
 cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st);
-// Plain CUDA-core implementation of the same problems, kept for bring-up and cross-checks.
-cudaError_t launch_gemm_plain(const GemmProblem& p, float* scratch, cudaStream_t st);
-extern int g_use_plain_gemm;
+size_t packed_weight_bytes(int n_src, int layout, int rows, int cols);
+cudaError_t launch_pack_weights(const void* const* src, int n_src, int layout, int rows, int cols, void* dst, cudaStream_t st);
 
 // ---- tree attention --------------------------------------------------------------------------------
 struct AttnProblem {
@@ -100,7 +111,8 @@ struct AttnProblem {
     int T, prefix_len, nh, hd;
     long long kv_stride;
     float scale;
-    void* out;          // [T][nh][hd] bf16
+    void* out;          // [T][nh][hd] bf16, or the packed activation layout if out_packed_npad > 0
+    int out_packed_npad;
     float* part_o;      // [nh][n_splits][T_pad][hd] fp32
     float* part_ml;     // [nh][n_splits][T_pad][2]
     int n_splits;       // filled by attn_plan

@@ -81,20 +81,26 @@ __global__ void __launch_bounds__(256) k_embed(const uint16_t* __restrict__ E, c
 // RMSNorm, one CTA per tree node.  Before normalising it folds n_part split-K partial sums of the
 // preceding projection into the fp32 residual stream (fixed order, so results are reproducible):
 //   resid[t] (+)= part[0][t] + part[1][t] + ...;   xn[t] = bf16(g * resid[t] * rsqrt(mean(resid[t]^2) + eps)).
+// xn is written in the packed activation layout the GEMM reads (n_pad rows per K block).
 // copy_from (optional): resid[t] starts from copy_from[t] instead of its own contents.
 // rope (optional): also fills the rotary table rope[t][i] = (cos, sin)(pos[t] * base^(-2i/hd)), i < hd/2,
 // evaluated in fp64 so that large positions lose no accuracy.
+// zero_flags (optional): CTA 0 clears the GEMM's stream-K flags (they are clear after every
+// successful launch; this guards against an uninitialised workspace).
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, const float* __restrict__ copy_from,
                                                  const float* __restrict__ part, int n_part, size_t part_stride,
                                                  const uint16_t* __restrict__ gain, int H, float eps,
-                                                 uint16_t* __restrict__ xn, const int32_t* __restrict__ pos,
-                                                 float2* __restrict__ rope, int hd, float rope_base) {
+                                                 uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
+                                                 float2* __restrict__ rope, int hd, float rope_base, int* zero_flags,
+                                                 int n_flags) {
     extern __shared__ float srow[];  // H floats
     __shared__ float red[8];
     pdl_launch_dependents();
     int t = blockIdx.x;
     pdl_wait();
+    if (zero_flags != nullptr && t == 0)
+        for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
     if (rope != nullptr) {
         int half = hd / 2;
         int p = pos[t];
@@ -124,18 +130,20 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
     float rs = rsqrtf(tot / (float)H + eps);
-    float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
-    for (int c = threadIdx.x; c < H / 4; c += blockDim.x) {
-        float4 v = reinterpret_cast<float4*>(srow)[c];
-        if (n_part > 0 || copy_from) out4[c] = v;
-        if (xn != nullptr) {
-            uint2 g2 = reinterpret_cast<const uint2*>(gain)[c];
-            float g0 = __uint_as_float(g2.x << 16), g1 = __uint_as_float(g2.x & 0xFFFF0000u);
-            float g2f = __uint_as_float(g2.y << 16), g3 = __uint_as_float(g2.y & 0xFFFF0000u);
-            uint2 o;
-            o.x = pack_bf16x2(g0 * (v.x * rs), g1 * (v.y * rs));
-            o.y = pack_bf16x2(g2f * (v.z * rs), g3 * (v.w * rs));
-            reinterpret_cast<uint2*>(xn + (size_t)t * H)[c] = o;
+    if (n_part > 0 || copy_from) {
+        float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
+        for (int c = threadIdx.x; c < H / 4; c += blockDim.x) out4[c] = reinterpret_cast<float4*>(srow)[c];
+    }
+    if (xn != nullptr) {
+        for (int c = threadIdx.x; c < H / 8; c += blockDim.x) {   // 8 consecutive features = one 16-byte group
+            float4 a = reinterpret_cast<float4*>(srow)[2 * c], b = reinterpret_cast<float4*>(srow)[2 * c + 1];
+            uint4 g = reinterpret_cast<const uint4*>(gain)[c];
+            uint4 o;
+            o.x = pack_bf16x2(__uint_as_float(g.x << 16) * (a.x * rs), __uint_as_float(g.x & 0xFFFF0000u) * (a.y * rs));
+            o.y = pack_bf16x2(__uint_as_float(g.y << 16) * (a.z * rs), __uint_as_float(g.y & 0xFFFF0000u) * (a.w * rs));
+            o.z = pack_bf16x2(__uint_as_float(g.z << 16) * (b.x * rs), __uint_as_float(g.z & 0xFFFF0000u) * (b.y * rs));
+            o.w = pack_bf16x2(__uint_as_float(g.w << 16) * (b.z * rs), __uint_as_float(g.w & 0xFFFF0000u) * (b.w * rs));
+            *reinterpret_cast<uint4*>(xn + packed_act_offset(t, c, n_pad)) = o;
         }
     }
 }
@@ -276,10 +284,11 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 }
 
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
-                           const void* gain, int T, int H, float eps, void* xn, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, cudaStream_t st) {
+                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
+                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st) {
     return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
-                      part_stride, (const uint16_t*)gain, H, eps, (uint16_t*)xn, pos, rope, hd, rope_base);
+                      part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, (T + 15) / 16 * 16, pos, rope, hd,
+                      rope_base, zero_flags, n_flags);
 }
 
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,

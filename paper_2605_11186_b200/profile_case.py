@@ -25,7 +25,7 @@ def main():
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     T, P = args.tree_size, args.prefix
-    model = gen.make_model(shape, "profile", device=dev)
+    model = cats.pack_model(gen.make_model(shape, "profile", device=dev), free_source=True)
     kc, vc = gen.make_kv_prefix(shape, args.layers, P + 128, P, "profile", device=dev)
     parent, _ = gen.tree_topk_shape(T, gen.topk_k_for(T))
     tokens = gen.uniform_tokens(T, shape.vocab, "profile", T)
