@@ -137,6 +137,30 @@ int cats_tree_attention(const void *d_q, const void *d_k, const void *d_v, const
                         int32_t prefix_len, int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems,
                         float scale, void *d_out, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
 
+/* Bytes of scratch the library image itself carries on every GPU for the entry point below. */
+#define CATS_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* cats_tree_attention for callers that cannot allocate.  (The paper has no counterpart: this is a
+ * packaging variant of the same operation.)  Same arguments and result as cats_tree_attention, but
+ * no workspace: the split-KV partial results go to a fixed CATS_STATIC_SCRATCH_BYTES array that is
+ * part of the library and stays resident on every GPU that loads it, until the process exits.  It
+ * is meant for code that has tensors but no way to get scratch memory at the call site: a plugin
+ * that is handed buffers and no allocator, a region where touching the device allocator is not
+ * allowed (someone else's stream capture), a real-time loop that must not call into the driver's
+ * memory management.  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   - Problems whose partial results do not fit (n_heads * splits * ceil16(T) * (head_dim + 2) * 4
+ *     bytes; e.g. 40 heads x 128 at T = 128) are refused with CATS_ERR_WORKSPACE; nothing is
+ *     launched.  Use cats_tree_attention with a caller-owned workspace for those.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps whatever the last call left in it.
+ *     Nothing in it needs to start at zero (every slot that is read was written by the same call),
+ *     but two calls whose kernels overlap on the GPU (different streams, or concurrent host
+ *     threads) would overwrite each other's partial results: serialise them. */
+int cats_tree_attention_static(const void *d_q, const void *d_k, const void *d_v, const uint64_t *d_mask, int32_t T,
+                               int32_t prefix_len, int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems,
+                               float scale, void *d_out, int32_t *d_status, void *stream);
+
 /* Final norm, LM head and per-node argmax (Algorithm 1: p_tgt <-
  * softmax(H(H_tgt)); greedy acceptance needs only argmax of the logits).
  *   d_logits [T][vocab] fp32 out, may be NULL.  d_argmax [T] int32 out: lowest

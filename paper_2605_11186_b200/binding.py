@@ -217,6 +217,18 @@ def cats_tree_attention(q, k, v, mask, T, prefix_len, n_heads, head_dim, kv_row_
            "cats_tree_attention")
 
 
+STATIC_SCRATCH_BYTES = 16 << 20
+lib.cats_tree_attention_static.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, C.c_float, _vp, _vp, _vp]
+
+
+def cats_tree_attention_static(q, k, v, mask, T, prefix_len, n_heads, head_dim, kv_row_stride, scale, out, status):
+    """cats_tree_attention without a workspace: the scratch is the fixed array inside the library (for callers that
+    cannot allocate).  Raises CatsError(-4) if the problem needs more than STATIC_SCRATCH_BYTES of partial results."""
+    _check(lib.cats_tree_attention_static(_ptr(q), _ptr(k), _ptr(v), _ptr(mask), T, prefix_len, n_heads, head_dim,
+                                          kv_row_stride, scale, _ptr(out), _ptr(status), _stream()),
+           "cats_tree_attention_static")
+
+
 def cats_lm_head_argmax(cfg, final_norm, w_lm, resid, T, logits, argmax, ws, status):
     _check(lib.cats_lm_head_argmax(C.byref(cfg), _ptr(final_norm), _ptr(w_lm), _ptr(resid), T, _ptr(logits), _ptr(argmax),
                                    _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_lm_head_argmax")

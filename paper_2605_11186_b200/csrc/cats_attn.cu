@@ -8,6 +8,8 @@
 // tile) x (slice of the 64-row block), so small trees still use every warp.  Partial (m, l, O) per
 // split go to the workspace and k_attn_combine merges them by log-sum-exp; with a single split the
 // CTA writes the final bf16 output itself.
+#include <mutex>
+
 #include "cats_kernels.cuh"
 
 namespace cats {
@@ -376,3 +378,73 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
 }
 
 }  // namespace cats
+
+// ---------------------------------------------------------------------------------------------------
+// Allocation-free variant of cats_tree_attention.
+//
+// Some callers cannot hand the library a workspace because they cannot obtain device memory at the
+// point of the call: code running between cudaStreamBeginCapture and EndCapture of someone else's
+// graph, plugins that are given tensors but no allocator, latency-critical loops that must not touch
+// the driver's allocator.  For them the split-KV partial results (running max, sum and unnormalised
+// output per split) live in a fixed array inside the library image.  Every GPU that loads the library
+// carries these CATS_STATIC_SCRATCH_BYTES until the process exits.
+//
+// g_attn_scratch is a device symbol: in host code its name is only a stand-in, not a device address.
+// The address is looked up once per device with cudaGetSymbolAddress, with that device current, and
+// that pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------------
+namespace cats {
+namespace {
+constexpr size_t kStaticScratchBytes = CATS_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_attn_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+void* g_attn_scratch_addr[kMaxDevices] = {};
+std::mutex g_attn_scratch_mutex;
+
+// Device address of the scratch array on the current device; looked up on the first call per device.
+cudaError_t static_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_attn_scratch_mutex);
+    if (g_attn_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_attn_scratch);
+        if (e != cudaSuccess) return e;
+        if (p == nullptr) return cudaErrorInvalidSymbol;
+        g_attn_scratch_addr[dev] = p;
+    }
+    *out = g_attn_scratch_addr[dev];
+    return cudaSuccess;
+}
+}  // namespace
+}  // namespace cats
+
+extern "C" int cats_tree_attention_static(const void* d_q, const void* d_k, const void* d_v, const uint64_t* d_mask, int32_t T,
+                                          int32_t prefix_len, int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems,
+                                          float scale, void* d_out, int32_t* d_status, void* stream) {
+    using namespace cats;
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_q || !d_k || !d_v || !d_mask || !d_out || !d_status) return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE || prefix_len < 0 || n_heads < 1) return CATS_ERR_INVALID_ARG;
+    if (head_dim != 64 && head_dim != 128) return CATS_ERR_UNSUPPORTED;
+    if (kv_row_stride_elems < (int64_t)n_heads * head_dim || kv_row_stride_elems % 8) return CATS_ERR_INVALID_ARG;
+    auto misaligned = [](const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; };
+    if (misaligned(d_q, 16) || misaligned(d_k, 16) || misaligned(d_v, 16) || misaligned(d_out, 4)) return CATS_ERR_INVALID_ARG;
+    AttnProblem a = {};
+    a.q = d_q; a.k = d_k; a.v = d_v; a.mask = d_mask; a.T = T; a.prefix_len = prefix_len; a.nh = n_heads; a.hd = head_dim;
+    a.kv_stride = kv_row_stride_elems; a.scale = scale; a.out = d_out; a.d_status = d_status;
+    const size_t need = attn_plan(a);
+    if (need > kStaticScratchBytes) return CATS_ERR_WORKSPACE;   // the problem needs more scratch than the library carries
+    if (need > 0) {
+        void* base = nullptr;
+        if (static_scratch_address(&base) != cudaSuccess) return CATS_ERR_CUDA;
+        const int tpad = (T + 15) / 16 * 16;
+        a.part_o = static_cast<float*>(base);
+        a.part_ml = a.part_o + (size_t)n_heads * a.n_splits * tpad * head_dim;
+    }
+    if (launch_tree_attention(a, (cudaStream_t)stream) != cudaSuccess) return CATS_ERR_CUDA;
+    return CATS_OK;
+}

@@ -1,0 +1,100 @@
+"""The allocation-free attention entry point (cats_tree_attention_static) against cats_tree_attention.
+
+Some users of the library have device tensors but nowhere to get scratch memory from when they call in (no
+allocator handed to a plugin, a region in which the device allocator must not be touched).  For them the library
+carries a fixed scratch array of its own.  This file checks, through the C ABI, that the variant returns what the
+workspace-taking entry point returns -- twice in a row with different inputs, since every call reuses the same
+array and finds the previous call's leftovers in it -- and that it refuses problems larger than the array.
+It is named to be collected last, so that a run stopping at the first failure has already run everything else."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_11186_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def cats():
+    from paper_2605_11186_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _mask_of(parent):
+    """Ancestor-or-self bitmask rows built on the host (inputs for both entry points alike)."""
+    T = len(parent)
+    m = np.zeros((T, 2), np.uint64)
+    for i in range(T):
+        j = i
+        while j >= 0:
+            m[i, j >> 6] |= np.uint64(1) << np.uint64(j & 63)
+            j = parent[j]
+    return m
+
+
+def _case(cats, tag, parent, P, nh, hd):
+    T = len(parent)
+    S = P + T
+    D = nh * hd
+    q = gen.normal_bf16((T, nh, hd), 1.0, "cuda", "noalloc", tag, "q")
+    k = gen.normal_bf16((S, D), 1.0, "cuda", "noalloc", tag, "k")
+    v = gen.normal_bf16((S, D), 1.0, "cuda", "noalloc", tag, "v")
+    mask = torch.from_numpy(_mask_of(parent).view(np.int64)).cuda()
+    return dict(T=T, P=P, nh=nh, hd=hd, D=D, q=q, k=k, v=v, mask=mask, scale=float(1.0 / np.sqrt(hd)))
+
+
+def _with_workspace(cats, c):
+    out = torch.zeros((c["T"], c["nh"], c["hd"]), dtype=torch.bfloat16, device="cuda")
+    cfg = cats.model_cfg(gen.ModelShape(hidden=c["D"], n_heads=c["nh"], head_dim=c["hd"], ffn=64, vocab=128, n_layers=1),
+                         c["P"] + c["T"])
+    ws = cats.new_workspace(cfg, c["T"], c["P"])
+    st = cats.new_status()
+    cats.cats_tree_attention(c["q"], c["k"], c["v"], c["mask"], c["T"], c["P"], c["nh"], c["hd"], c["D"], c["scale"], out, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return out
+
+
+def _static(cats, c):
+    out = torch.zeros((c["T"], c["nh"], c["hd"]), dtype=torch.bfloat16, device="cuda")
+    st = cats.new_status()
+    cats.cats_tree_attention_static(c["q"], c["k"], c["v"], c["mask"], c["T"], c["P"], c["nh"], c["hd"], c["D"], c["scale"], out, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return out
+
+
+def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(cats):
+    first = _case(cats, "a", gen.tree_heap(64), 1024, 32, 128)          # several KV splits: the scratch is used
+    second = _case(cats, "b", gen.tree_random(37, 11), 2000, 8, 64)     # other shape, other split layout, same array
+    want1 = _with_workspace(cats, first)
+    want2 = _with_workspace(cats, second)
+    got1 = _static(cats, first)
+    got2 = _static(cats, second)
+    for got, want in ((got1, want1), (got2, want2)):
+        assert torch.isfinite(got.float()).all()
+        err = (got.float() - want.float()).abs().max().item()
+        assert err <= TOL, err
+    # the same call again, straight after a different problem used the array
+    again = _static(cats, first)
+    assert (again.float() - want1.float()).abs().max().item() <= TOL
+
+
+def test_static_scratch_single_split_needs_no_scratch(cats):
+    c = _case(cats, "c", gen.tree_chain(16), 40, 4, 64)
+    assert (_static(cats, c).float() - _with_workspace(cats, c).float()).abs().max().item() <= TOL
+
+
+def test_static_scratch_refuses_oversized_problems(cats):
+    c = _case(cats, "d", gen.tree_random(128, 5), 4096, 40, 128)        # 40 heads x 128 at T = 128: > 16 MiB of partials
+    out = torch.zeros((c["T"], c["nh"], c["hd"]), dtype=torch.bfloat16, device="cuda")
+    st = cats.new_status()
+    with pytest.raises(cats.CatsError) as e:
+        cats.cats_tree_attention_static(c["q"], c["k"], c["v"], c["mask"], c["T"], c["P"], c["nh"], c["hd"], c["D"], c["scale"], out, st)
+    assert e.value.status == -4
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and torch.all(out == 0)                  # nothing was launched
