@@ -138,7 +138,7 @@ int cats_tree_attention(const void *d_q, const void *d_k, const void *d_v, const
                         float scale, void *d_out, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
 
 /* Bytes of scratch the library image itself carries on every GPU for the entry point below. */
-#define CATS_STATIC_SCRATCH_BYTES (16u << 20)
+#define CATS_STATIC_SCRATCH_BYTES (1u << 20)
 
 /* cats_tree_attention for callers that cannot allocate.  (The paper has no counterpart: this is a
  * packaging variant of the same operation.)  Same arguments and result as cats_tree_attention, but
@@ -148,9 +148,11 @@ int cats_tree_attention(const void *d_q, const void *d_k, const void *d_v, const
  * that is handed buffers and no allocator, a region where touching the device allocator is not
  * allowed (someone else's stream capture), a real-time loop that must not call into the driver's
  * memory management.  The call performs no cudaMalloc/cudaFree and calls no allocating routine.
- *   - Problems whose partial results do not fit (n_heads * splits * ceil16(T) * (head_dim + 2) * 4
- *     bytes; e.g. 40 heads x 128 at T = 128) are refused with CATS_ERR_WORKSPACE; nothing is
- *     launched.  Use cats_tree_attention with a caller-owned workspace for those.
+ *   - Scratch is needed only when one head is spread over several thread-block clusters (long
+ *     prefixes with few heads): n_heads * clusters_per_head * ceil16(T) * (head_dim + 2) * 4 bytes.
+ *     Problems needing more than the array holds (e.g. 14 heads x 128, T = 128, prefix 20000:
+ *     1.9 MB) are refused with CATS_ERR_WORKSPACE and nothing is launched; use
+ *     cats_tree_attention with a caller-owned workspace for those.
  *   - The first call on each device looks up the array's device address (with that device
  *     current) and caches it; make that first call outside any stream capture.
  *   - All calls on a device share the one array, and it keeps whatever the last call left in it.

@@ -217,7 +217,7 @@ def cats_tree_attention(q, k, v, mask, T, prefix_len, n_heads, head_dim, kv_row_
            "cats_tree_attention")
 
 
-STATIC_SCRATCH_BYTES = 16 << 20
+STATIC_SCRATCH_BYTES = 1 << 20
 lib.cats_tree_attention_static.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, C.c_float, _vp, _vp, _vp]
 
 

@@ -1,5 +1,7 @@
 // C-ABI layer of libcats: argument checks, workspace layout, and the launch sequence of the
 // tree-verification forward.  See include/cats.h for the contract of every entry point.
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "cats_kernels.cuh"
@@ -34,7 +36,7 @@ struct Workspace {
     size_t bytes;
 };
 
-int attn_split_bound(int nh) { int b = 296 / nh; return b < 1 ? 1 : b; }
+int attn_split_bound(int nh) { int b = (148 + nh - 1) / nh; return b < 1 ? 1 : b; }   // clusters per head, upper bound
 
 // Carves the workspace; with base == nullptr only the size is computed.
 Workspace carve(const cats_model_cfg* c, int T, void* base) {
@@ -84,25 +86,70 @@ inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintp
 // One decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still
 // to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
 // sums this layer's down projection left pending (>0) or a negative status.
+// L2 prefetch schedule (MB): how much of which upcoming weight matrix each kernel of a layer asks the memory system
+// to pull into L2 while it runs (HBM idles during the latency-bound kernels and during the tail of every projection).
+// Off by default: measured on B200, the bulk L2 prefetch instruction brings in only part of what it is asked for and
+// the forward got slower with every schedule tried.  The hook stays for measurements: CATS_PREFETCH_MB=a,b,c,d,e,f.
+struct PrefetchPolicy {
+    int norm1_qkv = 0;      // first RMSNorm: Wqkv, after what the previous down projection already requested
+    int qkv_o = 0;          // QKV projection, once its own weights are requested: Wo
+    int attn_gu = 0;        // attention: start of Wgate/up
+    int o_gu = 0;           // O projection: Wgate/up, continuing
+    int gu_down = 0;        // gate/up projection: Wdown
+    int down_next = 0;      // down projection: next layer's Wqkv (or the LM head)
+    bool loaded = false;
+};
+PrefetchPolicy g_pf;
+
+const PrefetchPolicy& pf_policy() {
+    if (!g_pf.loaded) {
+        g_pf.loaded = true;
+        if (const char* e = getenv("CATS_PREFETCH_MB")) {
+            int v[6];
+            if (sscanf(e, "%d,%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4], &v[5]) == 6) {
+                g_pf.norm1_qkv = v[0]; g_pf.qkv_o = v[1]; g_pf.attn_gu = v[2]; g_pf.o_gu = v[3]; g_pf.gu_down = v[4]; g_pf.down_next = v[5];
+            }
+        }
+    }
+    return g_pf;
+}
+
+// [offset_mb, offset_mb + len_mb) of a buffer of `total` bytes, clipped
+PrefetchSpan span_of(const void* base, size_t total, int offset_mb, int len_mb) {
+    PrefetchSpan s = {nullptr, 0};
+    size_t off = (size_t)offset_mb << 20, len = (size_t)len_mb << 20;
+    if (!base || len == 0 || off >= total) return s;
+    if (off + len > total) len = total - off;
+    s.ptr = (const uint8_t*)base + off;
+    s.bytes = len;
+    return s;
+}
+
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               int32_t* d_status, cudaStream_t st) {
+               const void* next_w, size_t next_w_bytes, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
     const int tpad = (T + 15) / 16 * 16;
+    const PrefetchPolicy& pf = pf_policy();
+    const size_t b_qkv = packed_weight_bytes(3, 0, D, H), b_o = packed_weight_bytes(1, 0, H, D);
+    const size_t b_gu = packed_weight_bytes(2, 1, F, H), b_d = packed_weight_bytes(1, 0, H, F);
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas,
+                                 span_of(w->wqkv, b_qkv, pf.down_next, pf.norm1_qkv), st));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
     g.d_status = d_status;
+    g.pf = span_of(w->wo, b_o, 0, pf.qkv_o);
     if (stage_on(1)) CATS_CUDA(launch_gemm(g, st));
 
     AttnProblem a = {};
     a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
     a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.out_packed_npad = tpad;
     a.part_o = ws.attn_o; a.part_ml = ws.attn_ml; a.d_status = d_status;
+    a.pf = span_of(w->w_gate_up, b_gu, 0, pf.attn_gu);
     attn_plan(a);
     if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
@@ -110,20 +157,23 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_o = gemm_plan(g).max_pieces;
+    g.pf = span_of(w->w_gate_up, b_gu, pf.attn_gu, pf.o_gu);
     if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
+                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, PrefetchSpan{nullptr, 0}, st));
 
     g = GemmProblem{};
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.act_out = ws.act; g.d_status = d_status;
+    g.pf = span_of(w->w_down, b_d, 0, pf.gu_down);
     if (stage_on(5)) CATS_CUDA(launch_gemm(g, st));
 
     g = GemmProblem{};
     g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_d = gemm_plan(g).max_pieces;
+    g.pf = span_of(next_w, next_w_bytes, 0, pf.down_next);
     if (stage_on(6)) CATS_CUDA(launch_gemm(g, st));
     return pieces_d;
 }
@@ -132,7 +182,8 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas,
+                             span_of(w_lm, packed_weight_bytes(1, 0, V, H), pf_policy().down_next, pf_policy().norm1_qkv), st));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -260,11 +311,12 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     Workspace ws = carve(cfg, T, d_ws);
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, d_status, st);
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, nullptr, 0,
+                             d_status, st);
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
+                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, PrefetchSpan{nullptr, 0}, st));
     return CATS_OK;
 }
 
@@ -361,8 +413,13 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     if (!copy_from) CATS_CUDA(launch_embed(a->d_embed, d_tokens, T, c->hidden, c->vocab, a->d_resid, a->d_status, st));
     int pending = 0;
     for (int l = 0; l < c->n_layers; ++l) {
+        const bool last = (l + 1 == c->n_layers);
+        const void* next_w = last ? a->d_w_lm : a->layers[l + 1].wqkv;
+        const size_t next_b = last ? packed_weight_bytes(1, 0, c->vocab, c->hidden)
+                                   : packed_weight_bytes(3, 0, c->n_heads * c->head_dim, c->hidden);
         pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
-                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, a->d_status, st);
+                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, next_w, next_b,
+                             a->d_status, st);
         if (pending < 0) return pending;
     }
     rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T, pending, a->d_logits,

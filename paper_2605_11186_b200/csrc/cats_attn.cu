@@ -1,13 +1,17 @@
 // Tree-masked attention of the T draft-tree nodes against the KV prefix plus their own ancestors.
 //
-// Split-KV: CTA (split, head) streams its range of cache rows in blocks of 64 through a double
+// Split-KV inside a thread-block cluster: the cache rows [0, prefix + T) of one head are divided
+// among the CTAs of a cluster (up to 8).  Each CTA streams its rows in blocks of 64 through a double
 // buffered cp.async pipeline (128-bit loads), keeps Q [T_pad][hd] in shared memory, and computes
 // S = Q K^T and O += P V with bf16 tensor-core MMAs (fp32 accumulation, online softmax in fp32 with
 // warp-shuffle row reductions).  Prefix rows need no mask; rows >= prefix_len test bit (row - prefix)
 // of the node's 128-bit ancestor mask held in shared memory.  Warps are laid out as (16-row query
-// tile) x (slice of the 64-row block), so small trees still use every warp.  Partial (m, l, O) per
-// split go to the workspace and k_attn_combine merges them by log-sum-exp; with a single split the
-// CTA writes the final bf16 output itself.
+// tile) x (slice of the 64-row block), so small trees still use every warp.  Every warp leaves its
+// partial (m, l, O) in its CTA's shared memory; after a cluster barrier the CTAs merge all partials of
+// the head by log-sum-exp, reading each other's shared memory (distributed shared memory), each CTA
+// finishing a share of the rows, and write the bf16 result.  Only when a head has far more rows than a
+// cluster can cover with few heads (long prefixes, few heads) are several clusters used per head; their
+// merged partials then go to the caller's workspace and k_attn_combine merges them.
 #include <mutex>
 
 #include "cats_kernels.cuh"
@@ -45,14 +49,35 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 struct AttnDev {
     const uint16_t *q, *k, *v;
     const uint64_t* mask;
-    int T, P, nh, n_mt, kvg, n_splits, bps;
+    int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split;
     long long kv_stride;
     float scale_log2;
     int out_npad;        // > 0: out is in the packed activation layout with this many rows per K block
     uint16_t* out;
-    float* part_o;
-    float* part_ml;
+    float* part_o;       // n_outer > 1: [nh][n_outer][T_pad][hd] fp32
+    float* part_ml;      //              [nh][n_outer][T_pad][2]
+    const uint8_t* pf_ptr;
+    size_t pf_bytes;
 };
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_map(uint32_t local_smem_addr, int rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
 
 template <int HD>
 __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) {
@@ -68,8 +93,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y;
     const int S = p.P + p.T;
-    const int c_begin = split * p.bps * kKvBlock;
-    const int c_end = min(S, c_begin + p.bps * kKvBlock);
+    const int c_begin = min(S, split * p.rows_per_split);
+    const int c_end = min(S, c_begin + p.rows_per_split);
     const int nb = (c_end - c_begin + kKvBlock - 1) / kKvBlock;
     const int mt = warp % p.n_mt, g = warp / p.n_mt;
     const bool active = g < p.kvg;
@@ -109,6 +134,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) mask_s[e] = (e < p.T * 2) ? p.mask[e] : 0ull;
     if (!early && nb > 0) load_kv(0, 0);
     cp_async_commit();
+    if (threadIdx.x == kAttnThreads - 1)    // upcoming weights into L2 while this kernel is busy with the KV cache
+        l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
 
     uint32_t qf[KS][4];
     float o[NT][4];
@@ -214,90 +241,88 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         __syncthreads();
     }
 
-    // ---- merge the warps that share a query tile, then write the split's partial (or final) result ----
+    // ---- every warp deposits its partial (m, l, O); the cluster merges all partials of the head ----
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
-    float* mrg_o = reinterpret_cast<float*>(kv_s);              // [8 warps][16][HD], aliases the KV buffers
-    float* mrg_ml = reinterpret_cast<float*>(q_s);              // [8 warps][16][2], aliases Q (no longer needed)
-    if (active && g > 0) {
-        float* wo = mrg_o + (size_t)warp * 16 * HD;
+    cp_async_wait<0>();                                  // a CTA without rows still has its Q copy in flight
+    __syncthreads();
+    float* loc_o = reinterpret_cast<float*>(kv_s);      // [kvg][Tpad][HD], aliases the KV buffers
+    float* loc_ml = reinterpret_cast<float*>(q_s);      // [kvg][Tpad][2], aliases Q (no longer needed)
+    if (active) {
+        float* wo = loc_o + ((size_t)g * Tpad) * HD;
 #pragma unroll
         for (int j = 0; j < NT; ++j) {
             int col = j * 8 + (lane & 3) * 2;
-            *reinterpret_cast<float2*>(wo + (lane >> 2) * HD + col) = make_float2(o[j][0], o[j][1]);
-            *reinterpret_cast<float2*>(wo + ((lane >> 2) + 8) * HD + col) = make_float2(o[j][2], o[j][3]);
+            *reinterpret_cast<float2*>(wo + (size_t)row_a * HD + col) = make_float2(o[j][0], o[j][1]);
+            *reinterpret_cast<float2*>(wo + (size_t)row_b * HD + col) = make_float2(o[j][2], o[j][3]);
         }
         if ((lane & 3) == 0) {
-            float* wm = mrg_ml + (size_t)warp * 32;
-            wm[(lane >> 2) * 2] = m_run[0]; wm[(lane >> 2) * 2 + 1] = l_run[0];
-            wm[((lane >> 2) + 8) * 2] = m_run[1]; wm[((lane >> 2) + 8) * 2 + 1] = l_run[1];
+            float* wm = loc_ml + ((size_t)g * Tpad) * 2;
+            wm[row_a * 2] = m_run[0]; wm[row_a * 2 + 1] = l_run[0];
+            wm[row_b * 2] = m_run[1]; wm[row_b * 2 + 1] = l_run[1];
         }
     }
     __syncthreads();
-    if (active && g == 0) {
-        float M[2] = {m_run[0], m_run[1]};
-        for (int gg = 1; gg < p.kvg; ++gg) {
-            const float* wm = mrg_ml + (size_t)(gg * p.n_mt + mt) * 32;
-            M[0] = fmaxf(M[0], wm[(lane >> 2) * 2]);
-            M[1] = fmaxf(M[1], wm[((lane >> 2) + 8) * 2]);
+    const int csize = p.csize;
+    const int rank = split % csize, outer = split / csize;
+    if (csize > 1) cluster_sync_all();
+    const int n_parts = csize * p.kvg;                         // <= 32
+    const uint32_t ml_base = smem_u32(loc_ml), o_base = smem_u32(loc_o);
+    for (int row = rank + csize * warp; row < p.T; row += csize * 8) {
+        float mp = -INFINITY, lp = 0.f;
+        uint32_t my_o = 0;
+        if (lane < n_parts) {
+            const int c = lane / p.kvg, gg = lane - c * p.kvg;
+            const uint32_t off = (uint32_t)((gg * Tpad + row) * 2 * 4);
+            float2 ml = ld_cluster_f2(cluster_map(ml_base + off, c));
+            mp = ml.x; lp = ml.y;
+            my_o = cluster_map(o_base + (uint32_t)((gg * Tpad + row) * HD * 4), c);
         }
-        float ref[2] = {M[0] == -INFINITY ? 0.f : M[0], M[1] == -INFINITY ? 0.f : M[1]};
-        float w0[2] = {exp2f(m_run[0] - ref[0]), exp2f(m_run[1] - ref[1])};
-        float L[2] = {l_run[0] * w0[0], l_run[1] * w0[1]};
+        float M = mp;
 #pragma unroll
-        for (int j = 0; j < NT; ++j) { o[j][0] *= w0[0]; o[j][1] *= w0[0]; o[j][2] *= w0[1]; o[j][3] *= w0[1]; }
-        for (int gg = 1; gg < p.kvg; ++gg) {
-            int ow = gg * p.n_mt + mt;
-            const float* wm = mrg_ml + (size_t)ow * 32;
-            const float* wo = mrg_o + (size_t)ow * 16 * HD;
-            float wa = exp2f(wm[(lane >> 2) * 2] - ref[0]), wb = exp2f(wm[((lane >> 2) + 8) * 2] - ref[1]);
-            L[0] += wm[(lane >> 2) * 2 + 1] * wa;
-            L[1] += wm[((lane >> 2) + 8) * 2 + 1] * wb;
+        for (int ofs = 16; ofs > 0; ofs >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, ofs));
+        const float ref = (M == -INFINITY) ? 0.f : M;
+        const float wp = exp2f(mp - ref);
+        float L = lp * wp;
 #pragma unroll
-            for (int j = 0; j < NT; ++j) {
-                int col = j * 8 + (lane & 3) * 2;
-                float2 va = *reinterpret_cast<const float2*>(wo + (lane >> 2) * HD + col);
-                float2 vb = *reinterpret_cast<const float2*>(wo + ((lane >> 2) + 8) * HD + col);
-                o[j][0] += va.x * wa; o[j][1] += va.y * wa; o[j][2] += vb.x * wb; o[j][3] += vb.y * wb;
+        for (int ofs = 16; ofs > 0; ofs >>= 1) L += __shfl_xor_sync(0xffffffffu, L, ofs);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const bool col_ok = lane < HD / 4;
+        for (int p0 = 0; p0 < n_parts; p0 += 8) {      // eight remote loads in flight at a time
+            float4 v[8];
+            float w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int pp = (p0 + i) & 31;
+                w[i] = (p0 + i < n_parts) ? __shfl_sync(0xffffffffu, wp, pp) : 0.f;
+                const uint32_t oa = __shfl_sync(0xffffffffu, my_o, pp);
+                v[i] = (col_ok && w[i] != 0.f) ? ld_cluster_f4(oa + (uint32_t)lane * 16) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-        }
-        if (p.n_splits == 1) {
-            float ia = 1.f / L[0], ib = 1.f / L[1];
 #pragma unroll
-            for (int j = 0; j < NT; ++j) {
-                int col = j * 8 + (lane & 3) * 2;
+            for (int i = 0; i < 8; ++i) { acc.x += v[i].x * w[i]; acc.y += v[i].y * w[i]; acc.z += v[i].z * w[i]; acc.w += v[i].w * w[i]; }
+        }
+        if (p.n_outer == 1) {
+            if (col_ok) {
+                const float inv = 1.f / L;
+                uint2 pk = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
                 uint8_t* ob = reinterpret_cast<uint8_t*>(p.out);
-                size_t off_a, off_b;
-                if (p.out_npad > 0) {
-                    off_a = packed_act_offset(row_a, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2;
-                    off_b = packed_act_offset(row_b, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2;
-                } else {
-                    off_a = (((size_t)row_a * p.nh + h) * HD + col) * 2;
-                    off_b = (((size_t)row_b * p.nh + h) * HD + col) * 2;
-                }
-                if (row_a < p.T) *reinterpret_cast<uint32_t*>(ob + off_a) = pack_bf16x2(o[j][0] * ia, o[j][1] * ia);
-                if (row_b < p.T) *reinterpret_cast<uint32_t*>(ob + off_b) = pack_bf16x2(o[j][2] * ib, o[j][3] * ib);
+                const int col = lane * 4;
+                size_t off = p.out_npad > 0 ? packed_act_offset(row, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2
+                                            : (((size_t)row * p.nh + h) * HD + col) * 2;
+                *reinterpret_cast<uint2*>(ob + off) = pk;
             }
         } else {
-            float* po = p.part_o + ((size_t)h * p.n_splits + split) * Tpad * HD;
-            float* pml = p.part_ml + ((size_t)h * p.n_splits + split) * Tpad * 2;
-#pragma unroll
-            for (int j = 0; j < NT; ++j) {
-                int col = j * 8 + (lane & 3) * 2;
-                *reinterpret_cast<float2*>(po + (size_t)row_a * HD + col) = make_float2(o[j][0], o[j][1]);
-                *reinterpret_cast<float2*>(po + (size_t)row_b * HD + col) = make_float2(o[j][2], o[j][3]);
-            }
-            if ((lane & 3) == 0) {
-                pml[row_a * 2] = M[0]; pml[row_a * 2 + 1] = L[0];
-                pml[row_b * 2] = M[1]; pml[row_b * 2 + 1] = L[1];
-            }
+            const size_t base = ((size_t)h * p.n_outer + outer) * Tpad + row;
+            if (col_ok) *reinterpret_cast<float4*>(p.part_o + base * HD + lane * 4) = acc;
+            if (lane == 0) { p.part_ml[base * 2] = M; p.part_ml[base * 2 + 1] = L; }
         }
     }
+    if (csize > 1) cluster_sync_all();   // nobody leaves while a peer may still read its shared memory
 }
 
-// out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s.  One CTA per (node, head), hd threads.
+// out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
 __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                       int n_splits, int Tpad, int nh, int hd, uint16_t* __restrict__ out,
                                                       int out_npad) {
@@ -323,22 +348,55 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
     }
 }
 
+// Chooses the cluster size (CTAs per head that share one merge through distributed shared memory) and, for long
+// prefixes with few heads, the number of clusters per head.  Returns the bytes of workspace the outer merge needs.
 size_t attn_plan(AttnProblem& p) {
-    int S = p.prefix_len + p.T;
-    int blocks = (S + kKvBlock - 1) / kKvBlock;
-    int tpad = ((p.T + 15) / 16) * 16;
-    int by_ctas = 296 / p.nh;
-    if (by_ctas < 1) by_ctas = 1;
-    int min_bps = tpad / kKvBlock;
-    if (min_bps < 1) min_bps = 1;
-    int by_traffic = (blocks + min_bps - 1) / min_bps;
-    int ns = by_ctas < by_traffic ? by_ctas : by_traffic;
-    if (ns < 1) ns = 1;
-    int bps = (blocks + ns - 1) / ns;
-    ns = (blocks + bps - 1) / bps;
-    p.n_splits = ns;
-    p.blocks_per_split = bps;
-    return ns > 1 ? (size_t)p.nh * ns * tpad * (p.hd + 2) * sizeof(float) : 0;
+    const int S = p.prefix_len + p.T;
+    const int units16 = (S + 15) / 16;
+    const int tpad = ((p.T + 15) / 16) * 16;
+    // as many CTAs per head as fit one wave of the 148 SMs (each CTA fills an SM), at most 8, at least 32 rows each
+    int csize = 148 / p.nh;
+    if (csize > 8) csize = 8;
+    if (csize > units16 / 2) csize = units16 / 2;
+    if (csize < 1) csize = 1;
+    int n_outer = 1;
+    int rows = (units16 + csize - 1) / csize * 16;
+    if (p.nh * csize < 120 && rows > 128) {
+        n_outer = (148 + p.nh * csize - 1) / (p.nh * csize);
+        if (n_outer > rows / 128) n_outer = rows / 128;
+        if (n_outer < 1) n_outer = 1;
+    }
+    const int splits = csize * n_outer;
+    p.n_splits = n_outer;
+    p.cluster = csize;
+    p.rows_per_split = (units16 + splits - 1) / splits * 16;
+    return n_outer > 1 ? (size_t)p.nh * n_outer * tpad * (p.hd + 2) * sizeof(float) : 0;
+}
+
+template <typename Kern>
+static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t smem, int csize, cudaStream_t st, const AttnDev& d) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)csize;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+    if (!g_call_boundary) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    g_call_boundary = false;
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    ++g_launch_count;
+    return cudaLaunchKernelEx(&cfg, kernel, d);
 }
 
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
@@ -357,21 +415,23 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.kvg = 8 / d.n_mt;
     if (d.kvg > 4) d.kvg = 4;
     if (d.kvg == 3) d.kvg = 2;
-    d.n_splits = p.n_splits; d.bps = p.blocks_per_split;
+    d.csize = p.cluster; d.n_outer = p.n_splits; d.rows_per_split = p.rows_per_split;
     d.kv_stride = p.kv_stride;
     d.scale_log2 = p.scale * 1.4426950408889634f;
     d.out = (uint16_t*)p.out;
     d.out_npad = p.out_packed_npad;
     d.part_o = p.part_o; d.part_ml = p.part_ml;
+    d.pf_ptr = (const uint8_t*)p.pf.ptr; d.pf_bytes = p.pf.bytes;
     int tpad = d.n_mt * 16;
-    size_t merge = (size_t)8 * 16 * p.hd * 4;                       // aliases the KV buffers
+    size_t merge = (size_t)d.kvg * tpad * p.hd * 4;                 // aliases the KV buffers
     size_t kv = (size_t)2 * 2 * kKvBlock * p.hd * 2;
-    size_t qbytes = (size_t)tpad * p.hd * 2;
-    if (qbytes < 8 * 32 * 4) qbytes = 8 * 32 * 4;                   // the (m, l) merge area aliases Q
+    size_t qbytes = (size_t)tpad * p.hd * 2;                        // the (m, l) deposit area aliases Q
+    if (qbytes < (size_t)d.kvg * tpad * 8) qbytes = (size_t)d.kvg * tpad * 8;
     size_t smem = qbytes + (kv > merge ? kv : merge) + (size_t)tpad * 16;
     cudaError_t e;
-    if (p.hd == 128) e = launch_pdl(k_tree_attn<128>, dim3(p.n_splits, p.nh), dim3(kAttnThreads), smem, st, d);
-    else e = launch_pdl(k_tree_attn<64>, dim3(p.n_splits, p.nh), dim3(kAttnThreads), smem, st, d);
+    dim3 grid(p.cluster * p.n_splits, p.nh);
+    if (p.hd == 128) e = launch_cluster(k_tree_attn<128>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
+    else e = launch_cluster(k_tree_attn<64>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);

@@ -31,14 +31,15 @@
 
 namespace cats {
 
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 224;
 constexpr int kCtrlBytes = 1024;
 constexpr int kMaxStages = 14;
 constexpr int kWChunk = 16384;        // 128 rows x 64 bf16
+constexpr int kUnitKb = 2;            // K blocks per pipeline stage (one bulk copy of W, one of X)
 constexpr int kStagingCols = 32;      // epilogue staging tile: 32 nodes x 128 features fp32
 
 struct GemmDev {
-    int epi, T, n_pad, n_out, n_kb, n_tiles, tiles_per_mat, units_per_cta, n_stages, max_pieces;
+    int epi, T, n_pad, n_out, n_kb, n_ku, n_tiles, tiles_per_mat, units_per_cta, n_stages, max_pieces;
     long long total_units;
     uint32_t x_chunk_bytes, stage_bytes, tmem_cols;
     const uint8_t* Wp;
@@ -55,6 +56,8 @@ struct GemmDev {
     float* pmax;
     int32_t* pidx;
     int32_t* d_status;
+    const uint8_t* pf_ptr;
+    size_t pf_bytes;
     int dbg;
     unsigned long long* trace;   // debug: [cta][32] timestamps
 };
@@ -109,7 +112,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     if (threadIdx.x == 0) {
         TRACE(0);
         for (int s = 0; s < S; ++s) {
-            mbar_init(&ctrl->full[s], 1);
+            mbar_init(&ctrl->full[s], 2);      // one arrive.expect_tx from each copy producer
             mbar_init(&ctrl->empty[s], 1);
         }
         mbar_init(&ctrl->acc_full[0], 1);
@@ -129,38 +132,44 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     pdl_launch_dependents();
     const uint32_t tmem_acc = ctrl->tmem_base;
 
-    if (warp == 0) {
-        // ---------------- copy producer ----------------
+    if (warp == 0 || warp == 6) {
+        // ---------------- copy producers: warp 0 streams W, warp 6 streams X ----------------
+        // One bulk copy costs its issuing thread a fixed ~0.45 us whatever its size (measured), so a stage holds
+        // kUnitKb K blocks fetched by ONE copy of W (contiguous in the packed matrix) and ONE copy of X, and the two
+        // kinds of copies come from different threads.
         if (lane == 0) {
-            const uint64_t pol_w = l2_policy_evict_first();
-            const uint64_t pol_x = l2_policy_evict_last();
-            const uint32_t tx = kWChunk + ((p.dbg & 2) ? 0u : p.x_chunk_bytes);
-            auto issue_w = [&](int i) {
-                int s = i % S;
-                mbar_expect_tx(&ctrl->full[s], tx);
-                bulk_load(stages + (size_t)s * p.stage_bytes, p.Wp + (size_t)(u0 + i) * kWChunk, kWChunk, &ctrl->full[s], pol_w);
+            const bool is_w = (warp == 0);
+            const uint64_t pol = is_w ? l2_policy_evict_first() : l2_policy_evict_last();
+            auto issue = [&](int i) {
+                const int s = i % S;
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.n_ku);
+                const int kb = (int)(u - (long long)tile * p.n_ku) * kUnitKb;
+                const int nk = min(kUnitKb, p.n_kb - kb);
+                uint8_t* stage = stages + (size_t)s * p.stage_bytes;
+                if (is_w) {
+                    const uint32_t bytes = (uint32_t)nk * kWChunk;
+                    mbar_expect_tx(&ctrl->full[s], bytes);
+                    bulk_load(stage, p.Wp + ((size_t)tile * p.n_kb + kb) * kWChunk, bytes, &ctrl->full[s], pol);
+                } else {
+                    const uint32_t bytes = (uint32_t)nk * p.x_chunk_bytes;
+                    mbar_expect_tx(&ctrl->full[s], bytes);
+                    bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &ctrl->full[s], pol);
+                }
             };
-            auto issue_x = [&](int i) {
-                if (p.dbg & 2) return;
-                int s = i % S;
-                int kb = (int)((u0 + i) % p.n_kb);
-                bulk_load(stages + (size_t)s * p.stage_bytes + kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, p.x_chunk_bytes,
-                          &ctrl->full[s], pol_x);
-            };
-            int pre = min(S, n_units);
-            TRACE(1);
-            for (int i = 0; i < pre; ++i) issue_w(i);   // weights do not depend on the previous kernel
-            pdl_wait();
-            TRACE(2);
-            for (int i = 0; i < pre; ++i) issue_x(i);
-            int issued = pre;
-            for (int i = pre; i < n_units; ++i) {
-                if (!mbar_wait(&ctrl->empty[i % S], ((i / S) - 1) & 1, abort_flag)) break;
-                issue_w(i);
-                issue_x(i);
+            if (is_w) TRACE(1);
+            if (!is_w) pdl_wait();     // activations come from the previous kernel; weights never do
+            int issued = 0;
+            for (int i = 0; i < n_units; ++i) {
+                if (i >= S && !mbar_wait(&ctrl->empty[i % S], ((i / S) - 1) & 1, abort_flag)) break;
+                issue(i);
                 issued = i + 1;
             }
-            TRACE(3);
+            if (is_w) {
+                TRACE(3);
+                // all of this launch's weights are requested: start pulling the next projection's into L2
+                l2_prefetch_slice(p.pf_ptr, p.pf_bytes, cta, gridDim.x);
+            }
             if (*abort_flag) {   // let the copies in flight land (bounded) before the CTA goes away
                 volatile int ignore = 0;
                 for (int i = max(0, issued - S); i < issued; ++i) mbar_wait(&ctrl->full[i % S], (i / S) & 1, &ignore);
@@ -173,7 +182,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
             int i = 0, seg = 0;
             bool ok = true;
             for (long long u = u0; u < u1 && ok; ++seg) {
-                const long long tile_end = (u / p.n_kb + 1) * p.n_kb;
+                const long long tile_end = (u / p.n_ku + 1) * p.n_ku;
                 const long long seg_end = min(u1, tile_end);
                 const int b = seg & 1;
                 if (seg >= 2) ok = mbar_wait(&ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, abort_flag);
@@ -185,21 +194,24 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                     ok = mbar_wait(&ctrl->full[s], (i / S) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    uint32_t a_addr = smem_u32(stages + (size_t)s * p.stage_bytes);
-                    uint64_t da = umma_desc_sw128(a_addr);
-                    uint64_t db = umma_desc_sw128(a_addr + kWChunk);
-                    if (!(p.dbg & 1)) {
+                    const int kb = (int)(u % p.n_ku) * kUnitKb;
+                    const int nk = min(kUnitKb, p.n_kb - kb);
+                    const uint32_t a_addr = smem_u32(stages + (size_t)s * p.stage_bytes);
+                    const uint32_t b_addr = a_addr + kUnitKb * kWChunk;
+                    for (int j = 0; j < nk; ++j) {
+                        const uint64_t da = umma_desc_sw128(a_addr + j * kWChunk);
+                        const uint64_t db = umma_desc_sw128(b_addr + j * p.x_chunk_bytes);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) umma_bf16(d_addr, da + 2 * k, db + 2 * k, idesc, !(first && k == 0));
+                        for (int k = 0; k < 4; ++k) umma_bf16(d_addr, da + 2 * k, db + 2 * k, idesc, !(first && k == 0));
+                        first = false;
                     }
-                    first = false;
                     umma_commit(&ctrl->empty[s]);
                 }
                 umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
                 if (seg < 4) TRACE(4 + seg);
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ---------------- epilogue warps ----------------
         const int q4 = warp & 3;               // TMEM lane quadrant this warp may read
         const int f = q4 * 32 + lane;          // accumulator row = weight row inside the tile
@@ -208,21 +220,50 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
         int seg = 0;
         bool ok = true;
         for (long long u = u0; u < u1; ++seg) {
-            const int tile = (int)(u / p.n_kb);
-            const long long tile_begin = (long long)tile * p.n_kb;
-            const long long tile_end = tile_begin + p.n_kb;
+            const int tile = (int)(u / p.n_ku);
+            const long long tile_begin = (long long)tile * p.n_ku;
+            const long long tile_end = tile_begin + p.n_ku;
             const long long seg_end = min(u1, tile_end);
             const bool head = (u == tile_begin) || (p.dbg & 32), tail = (seg_end == tile_end) || (p.dbg & 8);
             u = seg_end;
             const int b = seg & 1;
+            const int head_cta = (int)(tile_begin / p.units_per_cta);
+            const int last_cta = (int)((tile_end - 1) / p.units_per_cta);
             if (et == 0 && seg < 4) TRACE(8 + 4 * seg);
+            // A tile this CTA owns but shares with later CTAs: their partial tiles are usually published long before
+            // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
+            const bool gather = head && !tail && p.epi != EPI_PARTIAL;
+            float pre[64];
+            if (ok && gather) {
+                if (et == 0) {
+                    unsigned long long t0 = globaltimer_ns();
+                    for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                        while (ld_acquire(p.fix_flags + c2) == 0) {
+                            if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+                        }
+                    }
+                }
+                epi_barrier();
+                ok = !*abort_flag;
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pre[cc * 16 + i] = 0.f;
+                    if (ok && cc * 16 < p.n_pad) {
+                        for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                            const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(cc * 16) * 128 + f;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) pre[cc * 16 + i] += __ldcg(src + (size_t)i * 128);
+                        }
+                    }
+                }
+                if (et == 0 && seg < 4) TRACE(10 + 4 * seg);
+            }
             if (ok) ok = mbar_wait(&ctrl->acc_full[b], (seg >> 1) & 1, abort_flag);
             ok = ok && !*abort_flag;
             if (et == 0 && seg < 4) TRACE(9 + 4 * seg);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * p.n_pad);
-            const int head_cta = (int)(tile_begin / p.units_per_cta);
-            const int last_cta = (int)((tile_end - 1) / p.units_per_cta);
             int mat = 0, row0;
             if (p.epi == EPI_SWIGLU) row0 = tile * 64;
             else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
@@ -261,30 +302,27 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                 epi_barrier();
                 if (et == 0) st_release(p.fix_flags + cta, 1);
             } else {
-                // this CTA owns the tile: gather the other pieces (if any), then the fused epilogue
-                if (!tail) {
-                    if (et == 0) {
-                        unsigned long long t0 = globaltimer_ns();
-                        for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
-                            while (ld_acquire(p.fix_flags + c2) == 0) {
-                                if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
-                            }
-                        }
-                    }
-                    epi_barrier();
-                    ok = !*abort_flag;
-                    if (et == 0 && seg < 4) TRACE(10 + 4 * seg);
-                }
-                for (int c0 = 0; c0 < p.T && ok; c0 += kStagingCols) {
-                    const int ncols = min(kStagingCols, p.n_pad - c0);
-                    for (int c = 0; c < ncols; c += 16) {
+                // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
+#pragma unroll
+                for (int qc = 0; qc < CATS_MAX_TREE / kStagingCols; ++qc) {
+                    const int c0 = qc * kStagingCols;
+                    if (c0 >= p.T || !ok) break;
+#pragma unroll
+                    for (int hc = 0; hc < kStagingCols / 16; ++hc) {
+                        const int c = hc * 16;
+                        if (c0 + c >= p.n_pad) break;
                         float v[16];
                         tmem_ld16(taddr + c0 + c, v);
-                        if (!tail) {
-                            for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
-                                const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
+                        if (gather) {
+                            if (qc * (kStagingCols / 16) + hc < 4) {
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] += __ldcg(src + (size_t)i * 128);
+                                for (int i = 0; i < 16; ++i) v[i] += pre[((qc * (kStagingCols / 16) + hc) & 3) * 16 + i];
+                            } else {
+                                for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                                    const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
+#pragma unroll
+                                    for (int i = 0; i < 16; ++i) v[i] += __ldcg(src + (size_t)i * 128);
+                                }
                             }
                         }
                         if (p.epi == EPI_LMHEAD && p.logits != nullptr && row0 + f < p.n_out) {
@@ -296,8 +334,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                         }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) acc_s[(c + i) * 128 + f] = v[i];
+                        if (et == 0 && c0 == 0 && c == 0 && seg_end == u1) TRACE(25);
                     }
+                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(26);
                     epi_barrier();
+                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(27);
                     const int n_hi = (p.dbg & 16) ? 0 : min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
                     if (p.epi == EPI_QKV) {
                         // thread -> feature pair (2j, 2j+1), every other node.  All loads of the thread are issued
@@ -356,14 +397,15 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                             const int nl = (et >> 5) + 4 * it;
                             float2 g = *reinterpret_cast<const float2*>(acc_s + nl * 128 + j2);
                             float2 u = *reinterpret_cast<const float2*>(acc_s + nl * 128 + 64 + j2);
-                            packed[it] = pack_bf16x2(g.x / (1.f + __expf(-g.x)) * u.x, g.y / (1.f + __expf(-g.y)) * u.y);
+                            packed[it] = pack_bf16x2(__fdividef(g.x, 1.f + __expf(-g.x)) * u.x, __fdividef(g.y, 1.f + __expf(-g.y)) * u.y);
                         }
 #pragma unroll
                         for (int it = 0; it < NI; ++it) {
                             const int nl = (et >> 5) + 4 * it;
-                            if (nl < n_hi)
+                            if (nl < n_hi && !(p.dbg & 64))
                                 *reinterpret_cast<uint32_t*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad) +
                                                              (size_t)(feat & 7) * 2) = packed[it];
+                            if ((p.dbg & 64) && packed[it] == 0x12345678u) p.act_out[0] = 1;
                         }
                     } else if (p.epi == EPI_LMHEAD) {
                         for (int nl = warp - 2; nl < n_hi; nl += 4) {
@@ -387,7 +429,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                             }
                         }
                     }
+                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(28);
                     epi_barrier();
+                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(29);
                 }
                 if (!tail && et == 0)
                     for (int c2 = cta + 1; c2 <= last_cta; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
@@ -479,7 +523,7 @@ int gemm_num_tiles(const GemmProblem& p) {
 
 GemmPlan gemm_plan(const GemmProblem& p) {
     GemmPlan pl;
-    int n_kb = (p.K + 63) / 64;
+    int n_kb = ((p.K + 63) / 64 + kUnitKb - 1) / kUnitKb;   // units (groups of kUnitKb K blocks) per tile
     long long total = (long long)gemm_num_tiles(p) * n_kb;
     long long upc = (total + kGemmCtas - 1) / kGemmCtas;
     if (p.epi == EPI_PARTIAL) {   // a tile may not be cut into more pieces than there are partial-sum slots
@@ -510,13 +554,14 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.n_pad = ((p.T + 15) / 16) * 16;
     d.n_out = p.n_out;
     d.n_kb = (p.K + 63) / 64;
+    d.n_ku = (d.n_kb + kUnitKb - 1) / kUnitKb;
     d.n_tiles = gemm_num_tiles(p);
     d.tiles_per_mat = (p.n_out + 127) / 128;
-    d.total_units = (long long)d.n_tiles * d.n_kb;
+    d.total_units = (long long)d.n_tiles * d.n_ku;
     d.units_per_cta = pl.units_per_cta;
     d.max_pieces = pl.max_pieces;
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
-    d.stage_bytes = kWChunk + ((d.x_chunk_bytes + 1023) / 1024) * 1024;
+    d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
     size_t staging = (size_t)kStagingCols * 128 * 4;
     int stages = (int)((kMaxSmem - 1024 - kCtrlBytes - staging) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
@@ -544,6 +589,8 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.pmax = p.pmax;
     d.pidx = p.pidx;
     d.d_status = p.d_status;
+    d.pf_ptr = (const uint8_t*)p.pf.ptr;
+    d.pf_bytes = p.pf.bytes;
     {
         d.trace = g_trace_buf;
         const char* e = getenv("CATS_DBG");

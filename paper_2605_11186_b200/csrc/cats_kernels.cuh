@@ -33,6 +33,12 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// A span of upcoming weights a kernel should pull into L2 while it runs (see l2_prefetch_slice).
+struct PrefetchSpan {
+    const void* ptr;
+    size_t bytes;
+};
+
 // ---- small kernels ---------------------------------------------------------------------------
 cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64_t* mask, int32_t* pos, int32_t* depth,
                             int32_t* d_status, cudaStream_t st);
@@ -40,7 +46,7 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
                          cudaStream_t st);
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st);
+                           float rope_base, int* zero_flags, int n_flags, PrefetchSpan pf, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
@@ -87,6 +93,7 @@ struct GemmProblem {
     float* pmax;           //   [n_tiles][128]
     int32_t* pidx;
     int32_t* d_status;
+    PrefetchSpan pf;       // issued once this launch has requested all of its own weights
 };
 
 struct GemmPlan {
@@ -113,11 +120,13 @@ struct AttnProblem {
     float scale;
     void* out;          // [T][nh][hd] bf16, or the packed activation layout if out_packed_npad > 0
     int out_packed_npad;
-    float* part_o;      // [nh][n_splits][T_pad][hd] fp32
+    float* part_o;      // [nh][n_splits][T_pad][hd] fp32 (n_splits > 1 only)
     float* part_ml;     // [nh][n_splits][T_pad][2]
-    int n_splits;       // filled by attn_plan
-    int blocks_per_split;
+    int n_splits;       // filled by attn_plan: clusters per head (> 1 only for long prefixes with few heads)
+    int cluster;        //   CTAs per cluster
+    int rows_per_split; //   cache rows per CTA (multiple of 16)
     int32_t* d_status;
+    PrefetchSpan pf;
 };
 // Chooses the KV split; returns bytes of partial storage needed.
 size_t attn_plan(AttnProblem& p);

@@ -69,8 +69,8 @@ def _static(cats, c):
 
 
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(cats):
-    first = _case(cats, "a", gen.tree_heap(64), 1024, 32, 128)          # several KV splits: the scratch is used
-    second = _case(cats, "b", gen.tree_random(37, 11), 2000, 8, 64)     # other shape, other split layout, same array
+    first = _case(cats, "a", gen.tree_heap(64), 4096, 8, 128)           # few heads, long prefix: several clusters per head,
+    second = _case(cats, "b", gen.tree_random(37, 11), 3000, 4, 64)     # their partial results go through the scratch array
     want1 = _with_workspace(cats, first)
     want2 = _with_workspace(cats, second)
     got1 = _static(cats, first)
@@ -90,7 +90,7 @@ def test_static_scratch_single_split_needs_no_scratch(cats):
 
 
 def test_static_scratch_refuses_oversized_problems(cats):
-    c = _case(cats, "d", gen.tree_random(128, 5), 4096, 40, 128)        # 40 heads x 128 at T = 128: > 16 MiB of partials
+    c = _case(cats, "d", gen.tree_random(128, 5), 20000, 14, 128)       # 14 heads x 128, T = 128, prefix 20000: 1.9 MB of partials
     out = torch.zeros((c["T"], c["nh"], c["hd"]), dtype=torch.bfloat16, device="cuda")
     st = cats.new_status()
     with pytest.raises(cats.CatsError) as e:
