@@ -127,7 +127,7 @@ PrefetchSpan span_of(const void* base, size_t total, int offset_mb, int len_mb) 
 
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               const void* next_w, size_t next_w_bytes, int32_t* d_status, cudaStream_t st) {
+               const void* next_w, size_t next_w_bytes, bool next_is_head, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
     const int tpad = (T + 15) / 16 * 16;
     const PrefetchPolicy& pf = pf_policy();
@@ -143,6 +143,9 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
     g.d_status = d_status;
     g.pf = span_of(w->wo, b_o, 0, pf.qkv_o);
+    GemmProblem nxt = {};
+    nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = D; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->wo;
+    g.warm_next = &nxt;
     if (stage_on(1)) CATS_CUDA(launch_gemm(g, st));
 
     AttnProblem a = {};
@@ -158,6 +161,9 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_o = gemm_plan(g).max_pieces;
     g.pf = span_of(w->w_gate_up, b_gu, pf.attn_gu, pf.o_gu);
+    nxt = GemmProblem{};
+    nxt.epi = EPI_SWIGLU; nxt.T = T; nxt.K = H; nxt.n_out = F; nxt.n_mats = 2; nxt.W[0] = w->w_gate_up;
+    g.warm_next = &nxt;
     if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
@@ -167,6 +173,9 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.act_out = ws.act; g.d_status = d_status;
     g.pf = span_of(w->w_down, b_d, 0, pf.gu_down);
+    nxt = GemmProblem{};
+    nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = F; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->w_down;
+    g.warm_next = &nxt;
     if (stage_on(5)) CATS_CUDA(launch_gemm(g, st));
 
     g = GemmProblem{};
@@ -174,6 +183,10 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_d = gemm_plan(g).max_pieces;
     g.pf = span_of(next_w, next_w_bytes, 0, pf.down_next);
+    nxt = GemmProblem{};
+    if (next_is_head) { nxt.epi = EPI_LMHEAD; nxt.T = T; nxt.K = H; nxt.n_out = c->vocab; nxt.n_mats = 1; nxt.W[0] = next_w; }
+    else { nxt.epi = EPI_QKV; nxt.T = T; nxt.K = H; nxt.n_out = D; nxt.n_mats = 3; nxt.W[0] = next_w; }
+    g.warm_next = next_w ? &nxt : nullptr;
     if (stage_on(6)) CATS_CUDA(launch_gemm(g, st));
     return pieces_d;
 }
@@ -312,7 +325,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, nullptr, 0,
-                             d_status, st);
+                             false, d_status, st);
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
@@ -419,7 +432,7 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
                                    : packed_weight_bytes(3, 0, c->n_heads * c->head_dim, c->hidden);
         pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
                              (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, next_w, next_b,
-                             a->d_status, st);
+                             last, a->d_status, st);
         if (pending < 0) return pending;
     }
     rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T, pending, a->d_logits,

@@ -39,7 +39,7 @@ constexpr int kUnitKb = 2;            // K blocks per pipeline stage (one bulk c
 constexpr int kStagingCols = 32;      // epilogue staging tile: 32 nodes x 128 features fp32
 
 struct GemmDev {
-    int epi, T, n_pad, n_out, n_kb, n_ku, n_tiles, tiles_per_mat, units_per_cta, n_stages, max_pieces;
+    int epi, T, n_pad, n_out, n_kb, n_ku, n_tiles, tiles_per_mat, units_per_cta, n_stages, max_pieces, split_s;
     long long total_units;
     uint32_t x_chunk_bytes, stage_bytes, tmem_cols;
     const uint8_t* Wp;
@@ -58,6 +58,10 @@ struct GemmDev {
     int32_t* d_status;
     const uint8_t* pf_ptr;
     size_t pf_bytes;
+    const uint8_t* warm_ptr;     // next projection's packed weights: this CTA's first chunks of it
+    int warm_chunks;             // 16 KB chunks to pull through a landing buffer (warms L2)
+    int warm_upc, warm_n_ku, warm_n_kb;
+    long long warm_total_chunks;
     int dbg;
     unsigned long long* trace;   // debug: [cta][32] timestamps
 };
@@ -67,6 +71,7 @@ struct GemmCtrl {
     uint64_t empty[kMaxStages];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
+    uint64_t warm;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -99,14 +104,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(smem);
     uint8_t* stages = smem + kCtrlBytes;
     float* acc_s = reinterpret_cast<float*>(stages + (size_t)p.n_stages * p.stage_bytes);   // [32][128] fp32
+    uint8_t* landing = reinterpret_cast<uint8_t*>(acc_s) + (size_t)kStagingCols * 128 * 4;  // 16 KB, contents never read
     volatile int* abort_flag = &ctrl->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
     const int S = p.n_stages;
-    const long long u0 = (long long)cta * p.units_per_cta;
-    const long long u1 = min(p.total_units, u0 + (long long)p.units_per_cta);
+    // split_s == 0: even contiguous shares of all (tile, K) units; split_s > 0: every tile cut into split_s aligned pieces
+    long long u0, u1;
+    if (p.split_s > 0) {
+        const long long t0 = (long long)(cta / p.split_s) * p.n_ku;
+        u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
+        u1 = min(t0 + p.n_ku, u0 + (long long)p.units_per_cta);
+    } else {
+        u0 = (long long)cta * p.units_per_cta;
+        u1 = min(p.total_units, u0 + (long long)p.units_per_cta);
+    }
     const int n_units = (int)max(0ll, u1 - u0);
 
     if (threadIdx.x == 0) {
@@ -119,6 +133,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
         mbar_init(&ctrl->acc_full[1], 1);
         mbar_init(&ctrl->acc_empty[0], 128);
         mbar_init(&ctrl->acc_empty[1], 128);
+        mbar_init(&ctrl->warm, 1);
         ctrl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -169,6 +184,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                 TRACE(3);
                 // all of this launch's weights are requested: start pulling the next projection's into L2
                 l2_prefetch_slice(p.pf_ptr, p.pf_bytes, cta, gridDim.x);
+                // Real copies of the first chunks the same CTA of the next projection will read, into a landing buffer
+                // nobody reads: they leave those lines in L2 while this kernel drains and runs its last epilogue.
+                if (p.warm_ptr != nullptr && p.warm_chunks > 0) {
+                    // first chunk of this CTA's range in the next matrix: unit cta * upc -> (tile, K block)
+                    const long long wu = (long long)cta * p.warm_upc;
+                    const long long wt = wu / p.warm_n_ku;
+                    long long first = wt * p.warm_n_kb + (wu - wt * p.warm_n_ku) * kUnitKb;
+                    long long n = min((long long)p.warm_chunks, p.warm_total_chunks - first);
+                    if (n < 0) n = 0;
+                    mbar_expect_tx(&ctrl->warm, (uint32_t)n * kWChunk);
+                    for (long long j = 0; j < n; ++j)
+                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                     ::"r"(smem_u32(landing)), "l"(p.warm_ptr + (size_t)(first + j) * kWChunk), "r"(kWChunk), "r"(smem_u32(&ctrl->warm))
+                                     : "memory");
+                    volatile int ignore = 0;
+                    mbar_wait(&ctrl->warm, 0, &ignore);   // the landing buffer must stay alive until the copies have landed
+                }
             }
             if (*abort_flag) {   // let the copies in flight land (bounded) before the CTA goes away
                 volatile int ignore = 0;
@@ -272,7 +304,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                 // nothing: fall through to the arrive below so that nobody waits on this accumulator
             } else if (p.epi == EPI_PARTIAL) {
                 const int feat = row0 + f;
-                const int piece = cta - head_cta;
+                const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
                 float* dst = p.part + (size_t)piece * p.part_stride + feat;
                 for (int c = 0; c < p.T; c += 16) {
                     float v[16];
@@ -283,7 +315,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                             if (c + i < p.T) dst[(size_t)(c + i) * p.n_out] = v[i];
                     }
                 }
-                if (head && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
+                if (head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
                     for (int sl = last_cta - head_cta + 1; sl < p.max_pieces; ++sl) {
                         float* z = p.part + (size_t)sl * p.part_stride + feat;
                         for (int n = 0; n < p.T; ++n) z[(size_t)n * p.n_out] = 0.f;
@@ -523,18 +555,33 @@ int gemm_num_tiles(const GemmProblem& p) {
 
 GemmPlan gemm_plan(const GemmProblem& p) {
     GemmPlan pl;
-    int n_kb = ((p.K + 63) / 64 + kUnitKb - 1) / kUnitKb;   // units (groups of kUnitKb K blocks) per tile
-    long long total = (long long)gemm_num_tiles(p) * n_kb;
-    long long upc = (total + kGemmCtas - 1) / kGemmCtas;
-    if (p.epi == EPI_PARTIAL) {   // a tile may not be cut into more pieces than there are partial-sum slots
-        long long lim = (n_kb + kMaxPartSlots - 3) / (kMaxPartSlots - 2);
+    const int n_ku = ((p.K + 63) / 64 + kUnitKb - 1) / kUnitKb;   // units (groups of kUnitKb K blocks) per tile
+    const int tiles = gemm_num_tiles(p);
+    const long long total = (long long)tiles * n_ku;
+    long long upc = (total + kGemmCtas - 1) / kGemmCtas;          // stream-K: even, contiguous shares
+    if (p.epi == EPI_PARTIAL) {
+        // partial sums: cut every tile into the same number of aligned pieces when that keeps most SMs busy (fewer
+        // partial-sum slots for the following reduction, no zero filling), else even shares with a bounded number of
+        // pieces.  (One whole tile per CTA for the fused epilogues was measured too: 96 SMs cannot pull what 148 can.)
+        int s = kGemmCtas / tiles;
+        if (s > kMaxPartSlots) s = kMaxPartSlots;
+        if (s >= 2 && (long long)tiles * s * 10 >= kGemmCtas * 8 && n_ku >= s) {
+            pl.split_s = s;
+            pl.units_per_cta = (n_ku + s - 1) / s;
+            pl.n_ctas = tiles * s;
+            pl.max_pieces = s;
+            return pl;
+        }
+        long long lim = (n_ku + kMaxPartSlots - 3) / (kMaxPartSlots - 2);
         if (upc < lim) upc = lim;
     }
     if (upc < 1) upc = 1;
+    pl.split_s = 0;
     pl.units_per_cta = (int)upc;
     pl.n_ctas = (int)((total + upc - 1) / upc);
-    // pieces of one tile: a range of n_kb units cut by boundaries every upc units
-    pl.max_pieces = (int)((n_kb + upc - 2) / upc) + 1;
+    // pieces of one tile: a range of n_ku units cut by boundaries every upc units
+    pl.max_pieces = (n_ku % upc == 0) ? (int)(n_ku / upc) : (int)((n_ku + upc - 2) / upc) + 1;
+    if (upc >= n_ku && upc % n_ku == 0) pl.max_pieces = 1;
     if (pl.max_pieces > kMaxPartSlots) pl.max_pieces = kMaxPartSlots;
     return pl;
 }
@@ -560,9 +607,10 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.total_units = (long long)d.n_tiles * d.n_ku;
     d.units_per_cta = pl.units_per_cta;
     d.max_pieces = pl.max_pieces;
+    d.split_s = pl.split_s;
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
-    size_t staging = (size_t)kStagingCols * 128 * 4;
+    size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
     int stages = (int)((kMaxSmem - 1024 - kCtrlBytes - staging) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl.units_per_cta) stages = pl.units_per_cta;
@@ -591,6 +639,20 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.d_status = p.d_status;
     d.pf_ptr = (const uint8_t*)p.pf.ptr;
     d.pf_bytes = p.pf.bytes;
+    d.warm_ptr = nullptr;
+    d.warm_chunks = 0;
+    if (p.warm_next != nullptr && p.warm_next->W[0] != nullptr) {
+        static int n_warm = -1;
+        if (n_warm < 0) { const char* e = getenv("CATS_WARM_CHUNKS"); n_warm = e ? atoi(e) : 4; }
+        GemmPlan np = gemm_plan(*p.warm_next);
+        // the per-CTA base differs by CTA: pass the matrix base and let the CTA add its own offset
+        d.warm_ptr = (const uint8_t*)p.warm_next->W[0];
+        d.warm_chunks = d.n_pad > 64 ? 0 : n_warm;   // measured: a small gain for T <= 64, a small loss above
+        d.warm_upc = np.units_per_cta;
+        d.warm_n_ku = ((p.warm_next->K + 63) / 64 + kUnitKb - 1) / kUnitKb;
+        d.warm_n_kb = (p.warm_next->K + 63) / 64;
+        d.warm_total_chunks = (long long)gemm_num_tiles(*p.warm_next) * d.warm_n_kb;
+    }
     {
         d.trace = g_trace_buf;
         const char* e = getenv("CATS_DBG");

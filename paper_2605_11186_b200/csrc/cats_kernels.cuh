@@ -94,12 +94,14 @@ struct GemmProblem {
     int32_t* pidx;
     int32_t* d_status;
     PrefetchSpan pf;       // issued once this launch has requested all of its own weights
+    const GemmProblem* warm_next;   // the projection that follows (only W[0], K, n_out, n_mats, epi are read), or null
 };
 
 struct GemmPlan {
     int units_per_cta;   // (tile, K block) pairs per CTA, contiguous
     int n_ctas;
     int max_pieces;      // EPI_PARTIAL: number of partial-sum slots the following reduction must fold
+    int split_s;         // > 0: every tile is cut into this many aligned pieces (CTA = tile * split_s + piece)
 };
 
 // Number of 128-row tiles the problem has (SwiGLU: tiles of 64 gate + 64 up rows).
