@@ -255,7 +255,7 @@ def run_ours(args, rank, world, local_rank):
         "e2e": {"value": world * T / sec_e2e, "unit": UNIT, "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 16 + 2 * T * 4},
         "gpu_launches": main["launches"] * args.steps,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "k_gemm_tc (all %d projection launches of a forward)" % n_gemm,
+        "roofline": {"bound": "hbm", "kernel": "k_gemm_sk (all %d projection launches of a forward)" % n_gemm,
                      "achieved": wb / n_gemm / (gemm_sec / n_gemm) / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": wb / gemm_sec / 1e9 / peak, "peak_kind": peak_kind, "traffic": None,
                      "bytes_per_launch": wb / n_gemm, "us_per_launch": gemm_sec / n_gemm * 1e6,
