@@ -116,10 +116,15 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
     float ss = 0.f;
     for (int c = threadIdx.x; c < H / 4; c += blockDim.x) {
         float4 v = r4[c];
-        for (int s = 0; s < n_part; ++s) {
-            float4 pv = reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H)[c];
-            v.x += pv.x; v.y += pv.y; v.z += pv.z; v.w += pv.w;
-        }
+        // all partial-sum loads of this column group are issued before the first add (their latencies overlap);
+        // the adds keep slot order, so the result does not depend on how the loads return
+        float4 pv[kMaxPartSlots];
+#pragma unroll
+        for (int s = 0; s < kMaxPartSlots; ++s)
+            if (s < n_part) pv[s] = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + c);
+#pragma unroll
+        for (int s = 0; s < kMaxPartSlots; ++s)
+            if (s < n_part) { v.x += pv[s].x; v.y += pv[s].y; v.z += pv[s].z; v.w += pv[s].w; }
         reinterpret_cast<float4*>(srow)[c] = v;
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }

@@ -201,6 +201,9 @@ def test_compaction_bit_exact(cats):
 # a5: tree attention alone (config 5 shapes at sizes the oracle finishes quickly, plus ragged cases)
 # ---------------------------------------------------------------------------------------------------
 
+CONFIG5_FULL = [(P, name, parent) for P in (256, 1024, 4096, 16384)
+                for name, parent in (("chain16", gen.tree_chain(16)), ("heap64", gen.tree_heap(64)), ("rand128", gen.tree_random(128, 5)))]
+
 ATTN_CASES = [
     ("chain16_P256", gen.tree_chain(16), 256, 32, 128), ("heap64_P256", gen.tree_heap(64), 256, 32, 128),
     ("rand128_P256", gen.tree_random(128, 5), 256, 32, 128), ("rand128_P1024", gen.tree_random(128, 5), 1024, 32, 128),
@@ -230,6 +233,36 @@ def test_tree_attention_matches_oracle(cats, name, parent, P, nh, hd):
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     err = np.abs(out.float().cpu().numpy() - want).max()
+    assert err <= TOL, err
+
+
+@pytest.mark.parametrize("P,name,parent", CONFIG5_FULL, ids=["P%d_%s" % (c[0], c[1]) for c in CONFIG5_FULL])
+def test_config5_attention_sweep_full_size(cats, P, name, parent):
+    """Config 5 at its full sizes: 32 heads x 128, prefixes up to 16384, the three tree shapes, K/V ~ N(0,1).  The oracle is
+    evaluated on a sample of heads (every head is computed independently); all heads of the GPU result are checked for
+    finiteness and the sampled ones element by element."""
+    T, nh, hd = len(parent), 32, 128
+    S, D = P + T, nh * hd
+    q = gen.normal_bf16((T, nh, hd), 1.0, "cuda", "cfg5", P, name, "q")
+    k = gen.normal_bf16((S, D), 1.0, "cuda", "cfg5", P, name, "k")
+    v = gen.normal_bf16((S, D), 1.0, "cuda", "cfg5", P, name, "v")
+    _, mask, _, _ = oracle.build_tree_mask(parent, P)
+    scale = 1.0 / np.sqrt(hd)
+    out = torch.zeros((T, nh, hd), dtype=torch.bfloat16, device="cuda")
+    cfg = cats.model_cfg(gen.ModelShape(hidden=D, n_heads=nh, head_dim=hd, ffn=64, vocab=128, n_layers=1), S)
+    ws = cats.new_workspace(cfg, T, P)
+    st = cats.new_status()
+    cats.cats_tree_attention(q, k, v, dev(mask.view(np.int64)), T, P, nh, hd, D, float(scale), out, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    g = out.float().cpu().numpy()
+    assert np.isfinite(g).all()
+    heads = [0, 13, 31]
+    qs = q[:, heads].float().cpu().numpy().astype(np.float64)
+    ks = k.view(S, nh, hd)[:, heads].reshape(S, -1).float().cpu().numpy()
+    vs = v.view(S, nh, hd)[:, heads].reshape(S, -1).float().cpu().numpy()
+    want = oracle.tree_attention(qs, ks, vs, mask, P, len(heads), hd, scale)
+    err = np.abs(g[:, heads] - want).max()
     assert err <= TOL, err
 
 
@@ -431,10 +464,18 @@ def test_7b_shape_stack_with_head(cats, T, n_layers):
     _stack_case(cats, gen.LLAMA_7B, "cfg3_small", n_layers, parent, 512, T)
 
 
-def test_config3_full_depth(cats):
-    """Config 3 at full size: 32 layers of the 7B shape + LM head, prefix 512, T = 16 (the oracle needs a few seconds)."""
-    parent, _ = gen.tree_topk_shape(16, gen.topk_k_for(16))
-    _stack_case(cats, gen.LLAMA_7B, "cfg3_full", 32, parent, 512, 16)
+@pytest.mark.parametrize("T", [16, 64])
+def test_config3_full_depth(cats, T):
+    """Config 3 at full size, in the launch configuration bench.py times: 32 layers of the 7B shape + LM head, prefix 512,
+    top-k tree of T nodes (T = 64 is the benchmark's headline point; the oracle needs about a minute for it)."""
+    parent, _ = gen.tree_topk_shape(T, gen.topk_k_for(T))
+    _stack_case(cats, gen.LLAMA_7B, "cfg3_full", 32, parent, 512, T)
+
+
+def test_config4_full_depth(cats):
+    """Config 4 at full size: 40 layers of the 13B shape + LM head, prefix 2048, 64-node tree [6,3,2,2,1,1]."""
+    parent = gen.tree_branching([6, 3, 2, 2, 1, 1], 64)
+    _stack_case(cats, gen.LLAMA_13B, "cfg4_full", 40, parent, 2048, "t")
 
 
 def test_13b_shape_layer_stack(cats):
