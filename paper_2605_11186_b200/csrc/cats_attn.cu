@@ -49,7 +49,7 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 struct AttnDev {
     const uint16_t *q, *k, *v;
     const uint64_t* mask;
-    int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split;
+    int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split, blk, kv_area;   // blk: cache rows per pipeline block (multiple of 16*kvg); kv_area: bytes of the K/V buffers
     long long kv_stride;
     float scale_log2;
     int out_npad;        // > 0: out is in the packed activation layout with this many rows per K block
@@ -88,24 +88,24 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     constexpr int NT = HD / 8;                   // n-tiles of the output
     uint8_t* q_s = sm;                                           // [n_mt*16][HD]
     uint8_t* kv_s = q_s + (size_t)p.n_mt * 16 * ROWB;            // 2 buffers x (K [64][HD], V [64][HD])
-    uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + 2 * 2 * kKvBlock * ROWB);   // [n_mt*16][2]
+    uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + p.kv_area);   // [n_mt*16][2]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y;
     const int S = p.P + p.T;
     const int c_begin = min(S, split * p.rows_per_split);
     const int c_end = min(S, c_begin + p.rows_per_split);
-    const int nb = (c_end - c_begin + kKvBlock - 1) / kKvBlock;
+    const int nb = (c_end - c_begin + p.blk - 1) / p.blk;
     const int mt = warp % p.n_mt, g = warp / p.n_mt;
     const bool active = g < p.kvg;
-    const int R = kKvBlock / p.kvg;              // rows of each block this warp's group handles
+    const int R = p.blk / p.kvg;                 // rows of each block this warp's group handles
     const int Tpad = p.n_mt * 16;
 
     auto load_kv = [&](int b, int buf) {
-        uint8_t* ks = kv_s + (size_t)buf * 2 * kKvBlock * ROWB;
-        uint8_t* vs = ks + kKvBlock * ROWB;
-        int r0 = c_begin + b * kKvBlock;
-        for (int e = threadIdx.x; e < kKvBlock * NCH; e += kAttnThreads) {
+        uint8_t* ks = kv_s + (size_t)buf * 2 * p.blk * ROWB;
+        uint8_t* vs = ks + p.blk * ROWB;
+        int r0 = c_begin + b * p.blk;
+        for (int e = threadIdx.x; e < p.blk * NCH; e += kAttnThreads) {
             int r = e / NCH, ch = e % NCH;
             int row = r0 + r;
             uint32_t off = tile_off<HD>(r, ch);
@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 
     pdl_launch_dependents();
     // the first block can be requested before the previous kernel has finished if it lies in the prefix
-    const bool early = (c_begin + kKvBlock <= p.P);
+    const bool early = (c_begin + p.blk <= p.P);
     if (early) load_kv(0, 0);
     pdl_wait();
     for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
@@ -161,10 +161,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
             }
         }
         if (active) {
-            const uint8_t* ks_s = kv_s + (size_t)(b & 1) * 2 * kKvBlock * ROWB;
-            const uint8_t* vs_s = ks_s + kKvBlock * ROWB;
+            const uint8_t* ks_s = kv_s + (size_t)(b & 1) * 2 * p.blk * ROWB;
+            const uint8_t* vs_s = ks_s + p.blk * ROWB;
             const int rbase = g * R;                              // first row of this warp's slice in the block
-            const int cbase = c_begin + b * kKvBlock + rbase;     // its global cache row
+            const int cbase = c_begin + b * p.blk + rbase;     // its global cache row
             // 16 rows of the slice at a time: S = Q K^T (16 x 16), mask, online softmax, O += P V
             for (int sub = 0; sub < R; sub += 16) {
                 if (cbase + sub >= c_end) break;
@@ -402,8 +402,8 @@ static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t sme
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 120 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 120 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -424,10 +424,22 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.pf_ptr = (const uint8_t*)p.pf.ptr; d.pf_bytes = p.pf.bytes;
     int tpad = d.n_mt * 16;
     size_t merge = (size_t)d.kvg * tpad * p.hd * 4;                 // aliases the KV buffers
-    size_t kv = (size_t)2 * 2 * kKvBlock * p.hd * 2;
+    // Block size of the KV pipeline: a CTA whose whole share fits two or three 64-row blocks takes it in one block
+    // instead (one wait and one barrier round instead of three); long shares stream 64-row blocks.
+    int blk = kKvBlock;
+    {
+        const int gran = 16 * d.kvg;
+        const int whole = (p.rows_per_split + gran - 1) / gran * gran;
+        if (whole <= 192) blk = whole;
+    }
+    d.blk = blk;
+    const int n_buf = (p.rows_per_split <= blk) ? 1 : 2;            // a single block needs no second buffer
+    size_t kv = (size_t)n_buf * 2 * blk * p.hd * 2;
     size_t qbytes = (size_t)tpad * p.hd * 2;                        // the (m, l) deposit area aliases Q
     if (qbytes < (size_t)d.kvg * tpad * 8) qbytes = (size_t)d.kvg * tpad * 8;
-    size_t smem = qbytes + (kv > merge ? kv : merge) + (size_t)tpad * 16;
+    if (kv < merge) kv = merge;
+    d.kv_area = (int)kv;
+    size_t smem = qbytes + kv + (size_t)tpad * 16;
     cudaError_t e;
     dim3 grid(p.cluster * p.n_splits, p.nh);
     if (p.hd == 128) e = launch_cluster(k_tree_attn<128>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);

@@ -611,7 +611,9 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
     size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
-    int stages = (int)((kMaxSmem - 1024 - kCtrlBytes - staging) / d.stage_bytes);
+    static int budget_kb = -1;
+    if (budget_kb < 0) { const char* e = getenv("CATS_SMEM_KB"); budget_kb = e ? atoi(e) : 227; }
+    int stages = (int)(((size_t)budget_kb * 1024 - 1024 - kCtrlBytes - staging) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl.units_per_cta) stages = pl.units_per_cta;
     if (stages < 1) stages = 1;
