@@ -1,7 +1,5 @@
 // C-ABI layer of libcats: argument checks, workspace layout, and the launch sequence of the
 // tree-verification forward.  See include/cats.h for the contract of every entry point.
-#include <cstdio>
-#include <cstdlib>
 #include <cstring>
 
 #include "cats_kernels.cuh"
@@ -86,63 +84,19 @@ inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintp
 // One decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still
 // to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
 // sums this layer's down projection left pending (>0) or a negative status.
-// L2 prefetch schedule (MB): how much of which upcoming weight matrix each kernel of a layer asks the memory system
-// to pull into L2 while it runs (HBM idles during the latency-bound kernels and during the tail of every projection).
-// Off by default: measured on B200, the bulk L2 prefetch instruction brings in only part of what it is asked for and
-// the forward got slower with every schedule tried.  The hook stays for measurements: CATS_PREFETCH_MB=a,b,c,d,e,f.
-struct PrefetchPolicy {
-    int norm1_qkv = 0;      // first RMSNorm: Wqkv, after what the previous down projection already requested
-    int qkv_o = 0;          // QKV projection, once its own weights are requested: Wo
-    int attn_gu = 0;        // attention: start of Wgate/up
-    int o_gu = 0;           // O projection: Wgate/up, continuing
-    int gu_down = 0;        // gate/up projection: Wdown
-    int down_next = 0;      // down projection: next layer's Wqkv (or the LM head)
-    bool loaded = false;
-};
-PrefetchPolicy g_pf;
-
-const PrefetchPolicy& pf_policy() {
-    if (!g_pf.loaded) {
-        g_pf.loaded = true;
-        if (const char* e = getenv("CATS_PREFETCH_MB")) {
-            int v[6];
-            if (sscanf(e, "%d,%d,%d,%d,%d,%d", &v[0], &v[1], &v[2], &v[3], &v[4], &v[5]) == 6) {
-                g_pf.norm1_qkv = v[0]; g_pf.qkv_o = v[1]; g_pf.attn_gu = v[2]; g_pf.o_gu = v[3]; g_pf.gu_down = v[4]; g_pf.down_next = v[5];
-            }
-        }
-    }
-    return g_pf;
-}
-
-// [offset_mb, offset_mb + len_mb) of a buffer of `total` bytes, clipped
-PrefetchSpan span_of(const void* base, size_t total, int offset_mb, int len_mb) {
-    PrefetchSpan s = {nullptr, 0};
-    size_t off = (size_t)offset_mb << 20, len = (size_t)len_mb << 20;
-    if (!base || len == 0 || off >= total) return s;
-    if (off + len > total) len = total - off;
-    s.ptr = (const uint8_t*)base + off;
-    s.bytes = len;
-    return s;
-}
-
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
                const void* next_w, size_t next_w_bytes, bool next_is_head, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
     const int tpad = (T + 15) / 16 * 16;
-    const PrefetchPolicy& pf = pf_policy();
-    const size_t b_qkv = packed_weight_bytes(3, 0, D, H), b_o = packed_weight_bytes(1, 0, H, D);
-    const size_t b_gu = packed_weight_bytes(2, 1, F, H), b_d = packed_weight_bytes(1, 0, H, F);
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas,
-                                 span_of(w->wqkv, b_qkv, pf.down_next, pf.norm1_qkv), st));
+                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
     g.d_status = d_status;
-    g.pf = span_of(w->wo, b_o, 0, pf.qkv_o);
     GemmProblem nxt = {};
     nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = D; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->wo;
     g.warm_next = &nxt;
@@ -152,7 +106,6 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
     a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.out_packed_npad = tpad;
     a.part_o = ws.attn_o; a.part_ml = ws.attn_ml; a.d_status = d_status;
-    a.pf = span_of(w->w_gate_up, b_gu, 0, pf.attn_gu);
     attn_plan(a);
     if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
@@ -160,19 +113,17 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_o = gemm_plan(g).max_pieces;
-    g.pf = span_of(w->w_gate_up, b_gu, pf.attn_gu, pf.o_gu);
     nxt = GemmProblem{};
     nxt.epi = EPI_SWIGLU; nxt.T = T; nxt.K = H; nxt.n_out = F; nxt.n_mats = 2; nxt.W[0] = w->w_gate_up;
     g.warm_next = &nxt;
     if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, PrefetchSpan{nullptr, 0}, st));
+                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
 
     g = GemmProblem{};
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.act_out = ws.act; g.d_status = d_status;
-    g.pf = span_of(w->w_down, b_d, 0, pf.gu_down);
     nxt = GemmProblem{};
     nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = F; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->w_down;
     g.warm_next = &nxt;
@@ -182,7 +133,6 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
     int pieces_d = gemm_plan(g).max_pieces;
-    g.pf = span_of(next_w, next_w_bytes, 0, pf.down_next);
     nxt = GemmProblem{};
     if (next_is_head) { nxt.epi = EPI_LMHEAD; nxt.T = T; nxt.K = H; nxt.n_out = c->vocab; nxt.n_mats = 1; nxt.W[0] = next_w; }
     else { nxt.epi = EPI_QKV; nxt.T = T; nxt.K = H; nxt.n_out = D; nxt.n_mats = 3; nxt.W[0] = next_w; }
@@ -195,8 +145,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas,
-                             span_of(w_lm, packed_weight_bytes(1, 0, V, H), pf_policy().down_next, pf_policy().norm1_qkv), st));
+                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -329,7 +278,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, PrefetchSpan{nullptr, 0}, st));
+                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
     return CATS_OK;
 }
 

@@ -56,8 +56,6 @@ struct AttnDev {
     uint16_t* out;
     float* part_o;       // n_outer > 1: [nh][n_outer][T_pad][hd] fp32
     float* part_ml;      //              [nh][n_outer][T_pad][2]
-    const uint8_t* pf_ptr;
-    size_t pf_bytes;
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -134,8 +132,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) mask_s[e] = (e < p.T * 2) ? p.mask[e] : 0ull;
     if (!early && nb > 0) load_kv(0, 0);
     cp_async_commit();
-    if (threadIdx.x == kAttnThreads - 1)    // upcoming weights into L2 while this kernel is busy with the KV cache
-        l2_prefetch_slice(p.pf_ptr, p.pf_bytes, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
 
     uint32_t qf[KS][4];
     float o[NT][4];
@@ -421,7 +417,6 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.out = (uint16_t*)p.out;
     d.out_npad = p.out_packed_npad;
     d.part_o = p.part_o; d.part_ml = p.part_ml;
-    d.pf_ptr = (const uint8_t*)p.pf.ptr; d.pf_bytes = p.pf.bytes;
     int tpad = d.n_mt * 16;
     size_t merge = (size_t)d.kvg * tpad * p.hd * 4;                 // aliases the KV buffers
     // Block size of the KV pipeline: a CTA whose whole share fits two or three 64-row blocks takes it in one block

@@ -116,23 +116,6 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, in
         : "memory");
 }
 
-// Asks the memory system to bring [ptr, ptr + bytes) into L2 (no destination, no completion to wait for).
-// The span is cut into n_parts contiguous slices of 16 KB pieces; the caller (one thread) issues slice `part`.
-// Used to keep HBM busy with the next projection's weights while a latency-bound kernel runs.
-__device__ __forceinline__ void l2_prefetch_slice(const uint8_t* ptr, size_t bytes, int part, int n_parts) {
-    if (ptr == nullptr || bytes == 0) return;
-    const size_t pieces = (bytes + 16383) >> 14;
-    const size_t per = (pieces + n_parts - 1) / n_parts;
-    size_t c0 = (size_t)part * per, c1 = c0 + per;
-    if (c1 > pieces) c1 = pieces;
-    for (size_t c = c0; c < c1; ++c) {
-        size_t n = bytes - (c << 14);
-        if (n > 16384) n = 16384;
-        n &= ~(size_t)15;
-        if (n) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr + (c << 14)), "r"((uint32_t)n) : "memory");
-    }
-}
-
 // ---- tcgen05 (5th-generation tensor cores, accumulators in tensor memory) -------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_slot, uint32_t ncols) {  // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_slot)), "r"(ncols)

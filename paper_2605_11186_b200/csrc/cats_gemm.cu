@@ -56,14 +56,10 @@ struct GemmDev {
     float* pmax;
     int32_t* pidx;
     int32_t* d_status;
-    const uint8_t* pf_ptr;
-    size_t pf_bytes;
     const uint8_t* warm_ptr;     // next projection's packed weights: this CTA's first chunks of it
     int warm_chunks;             // 16 KB chunks to pull through a landing buffer (warms L2)
     int warm_upc, warm_n_ku, warm_n_kb;
     long long warm_total_chunks;
-    int dbg;
-    unsigned long long* trace;   // debug: [cta][32] timestamps
 };
 
 struct GemmCtrl {
@@ -95,9 +91,6 @@ __device__ __forceinline__ void st_release(int* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-unsigned long long* g_trace_buf = nullptr;
-#define TRACE(slot) do { if (p.trace) p.trace[(size_t)blockIdx.x * 32 + (slot)] = globaltimer_ns(); } while (0)
-
 __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -124,7 +117,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     const int n_units = (int)max(0ll, u1 - u0);
 
     if (threadIdx.x == 0) {
-        TRACE(0);
         for (int s = 0; s < S; ++s) {
             mbar_init(&ctrl->full[s], 2);      // one arrive.expect_tx from each copy producer
             mbar_init(&ctrl->empty[s], 1);
@@ -172,7 +164,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                     bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &ctrl->full[s], pol);
                 }
             };
-            if (is_w) TRACE(1);
             if (!is_w) pdl_wait();     // activations come from the previous kernel; weights never do
             int issued = 0;
             for (int i = 0; i < n_units; ++i) {
@@ -181,9 +172,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                 issued = i + 1;
             }
             if (is_w) {
-                TRACE(3);
-                // all of this launch's weights are requested: start pulling the next projection's into L2
-                l2_prefetch_slice(p.pf_ptr, p.pf_bytes, cta, gridDim.x);
                 // Real copies of the first chunks the same CTA of the next projection will read, into a landing buffer
                 // nobody reads: they leave those lines in L2 while this kernel drains and runs its last epilogue.
                 if (p.warm_ptr != nullptr && p.warm_chunks > 0) {
@@ -240,7 +228,6 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                     umma_commit(&ctrl->empty[s]);
                 }
                 umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
-                if (seg < 4) TRACE(4 + seg);
             }
         }
     } else if (warp < 6) {
@@ -256,12 +243,11 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
             const long long tile_begin = (long long)tile * p.n_ku;
             const long long tile_end = tile_begin + p.n_ku;
             const long long seg_end = min(u1, tile_end);
-            const bool head = (u == tile_begin) || (p.dbg & 32), tail = (seg_end == tile_end) || (p.dbg & 8);
+            const bool head = (u == tile_begin), tail = (seg_end == tile_end);
             u = seg_end;
             const int b = seg & 1;
             const int head_cta = (int)(tile_begin / p.units_per_cta);
             const int last_cta = (int)((tile_end - 1) / p.units_per_cta);
-            if (et == 0 && seg < 4) TRACE(8 + 4 * seg);
             // A tile this CTA owns but shares with later CTAs: their partial tiles are usually published long before
             // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
             const bool gather = head && !tail && p.epi != EPI_PARTIAL;
@@ -289,18 +275,16 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                         }
                     }
                 }
-                if (et == 0 && seg < 4) TRACE(10 + 4 * seg);
             }
             if (ok) ok = mbar_wait(&ctrl->acc_full[b], (seg >> 1) & 1, abort_flag);
             ok = ok && !*abort_flag;
-            if (et == 0 && seg < 4) TRACE(9 + 4 * seg);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * p.n_pad);
             int mat = 0, row0;
             if (p.epi == EPI_SWIGLU) row0 = tile * 64;
             else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
 
-            if (!ok || (p.dbg & 4)) {
+            if (!ok) {
                 // nothing: fall through to the arrive below so that nobody waits on this accumulator
             } else if (p.epi == EPI_PARTIAL) {
                 const int feat = row0 + f;
@@ -366,12 +350,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                         }
 #pragma unroll
                         for (int i = 0; i < 16; ++i) acc_s[(c + i) * 128 + f] = v[i];
-                        if (et == 0 && c0 == 0 && c == 0 && seg_end == u1) TRACE(25);
                     }
-                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(26);
                     epi_barrier();
-                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(27);
-                    const int n_hi = (p.dbg & 16) ? 0 : min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
+                    const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
                     if (p.epi == EPI_QKV) {
                         // thread -> feature pair (2j, 2j+1), every other node.  All loads of the thread are issued
                         // before the first store, so their latencies overlap.
@@ -434,10 +415,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
 #pragma unroll
                         for (int it = 0; it < NI; ++it) {
                             const int nl = (et >> 5) + 4 * it;
-                            if (nl < n_hi && !(p.dbg & 64))
+                            if (nl < n_hi)
                                 *reinterpret_cast<uint32_t*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad) +
                                                              (size_t)(feat & 7) * 2) = packed[it];
-                            if ((p.dbg & 64) && packed[it] == 0x12345678u) p.act_out[0] = 1;
                         }
                     } else if (p.epi == EPI_LMHEAD) {
                         for (int nl = warp - 2; nl < n_hi; nl += 4) {
@@ -461,16 +441,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                             }
                         }
                     }
-                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(28);
                     epi_barrier();
-                    if (et == 0 && c0 == 0 && seg_end == u1) TRACE(29);
                 }
                 if (!tail && et == 0)
                     for (int c2 = cta + 1; c2 <= last_cta; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
             }
             tc_fence_before_sync();
             mbar_arrive(&ctrl->acc_empty[b]);
-            if (et == 0 && seg < 4) TRACE(11 + 4 * seg);
         }
     }
     tc_fence_before_sync();
@@ -480,11 +457,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_acc, p.tmem_cols);
     }
-    if (threadIdx.x == 0) TRACE(24);
     if (threadIdx.x == 0 && ctrl->abort_flag) report(p.d_status, CATS_ERR_TIMEOUT);
 }
-
-extern "C" void cats_debug_set_trace(unsigned long long* buf) { g_trace_buf = buf; }
 
 // ---------------------------------------------------------------------------------------------------
 // Weight packing: nn.Linear [rows][cols] bf16 -> 16 KB chunks (tile, K block) in the tcgen05 K-major
@@ -611,9 +585,7 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
     size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
-    static int budget_kb = -1;
-    if (budget_kb < 0) { const char* e = getenv("CATS_SMEM_KB"); budget_kb = e ? atoi(e) : 227; }
-    int stages = (int)(((size_t)budget_kb * 1024 - 1024 - kCtrlBytes - staging) / d.stage_bytes);
+    int stages = (int)((kMaxSmem - 1024 - kCtrlBytes - staging) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl.units_per_cta) stages = pl.units_per_cta;
     if (stages < 1) stages = 1;
@@ -639,13 +611,10 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.pmax = p.pmax;
     d.pidx = p.pidx;
     d.d_status = p.d_status;
-    d.pf_ptr = (const uint8_t*)p.pf.ptr;
-    d.pf_bytes = p.pf.bytes;
     d.warm_ptr = nullptr;
     d.warm_chunks = 0;
     if (p.warm_next != nullptr && p.warm_next->W[0] != nullptr) {
-        static int n_warm = -1;
-        if (n_warm < 0) { const char* e = getenv("CATS_WARM_CHUNKS"); n_warm = e ? atoi(e) : 4; }
+        const int n_warm = 4;   // 64 KB per CTA, 9.5 MB in all: what lands while the last epilogue runs
         GemmPlan np = gemm_plan(*p.warm_next);
         // the per-CTA base differs by CTA: pass the matrix base and let the CTA add its own offset
         d.warm_ptr = (const uint8_t*)p.warm_next->W[0];
@@ -654,13 +623,6 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         d.warm_n_ku = ((p.warm_next->K + 63) / 64 + kUnitKb - 1) / kUnitKb;
         d.warm_n_kb = (p.warm_next->K + 63) / 64;
         d.warm_total_chunks = (long long)gemm_num_tiles(*p.warm_next) * d.warm_n_kb;
-    }
-    {
-        d.trace = g_trace_buf;
-        const char* e = getenv("CATS_DBG");
-        d.dbg = e ? atoi(e) : 0;
-        const char* st_ = getenv("CATS_DBG_STAGES");
-        if (st_ && atoi(st_) > 0 && atoi(st_) < d.n_stages) d.n_stages = atoi(st_);
     }
     return launch_pdl(k_gemm_sk, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
 }

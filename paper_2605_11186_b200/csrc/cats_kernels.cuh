@@ -33,12 +33,6 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// A span of upcoming weights a kernel should pull into L2 while it runs (see l2_prefetch_slice).
-struct PrefetchSpan {
-    const void* ptr;
-    size_t bytes;
-};
-
 // ---- small kernels ---------------------------------------------------------------------------
 cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64_t* mask, int32_t* pos, int32_t* depth,
                             int32_t* d_status, cudaStream_t st);
@@ -46,7 +40,7 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
                          cudaStream_t st);
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, int* zero_flags, int n_flags, PrefetchSpan pf, cudaStream_t st);
+                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
@@ -93,7 +87,6 @@ struct GemmProblem {
     float* pmax;           //   [n_tiles][128]
     int32_t* pidx;
     int32_t* d_status;
-    PrefetchSpan pf;       // issued once this launch has requested all of its own weights
     const GemmProblem* warm_next;   // the projection that follows (only W[0], K, n_out, n_mats, epi are read), or null
 };
 
@@ -128,7 +121,6 @@ struct AttnProblem {
     int cluster;        //   CTAs per cluster
     int rows_per_split; //   cache rows per CTA (multiple of 16)
     int32_t* d_status;
-    PrefetchSpan pf;
 };
 // Chooses the KV split; returns bytes of partial storage needed.
 size_t attn_plan(AttnProblem& p);

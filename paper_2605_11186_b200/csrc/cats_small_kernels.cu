@@ -93,12 +93,11 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
                                                  const uint16_t* __restrict__ gain, int H, float eps,
                                                  uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
                                                  float2* __restrict__ rope, int hd, float rope_base, int* zero_flags,
-                                                 int n_flags, const uint8_t* pf_ptr, size_t pf_bytes) {
+                                                 int n_flags) {
     extern __shared__ float srow[];  // H floats
     __shared__ float red[8];
     pdl_launch_dependents();
     int t = blockIdx.x;
-    if (threadIdx.x == 0) l2_prefetch_slice(pf_ptr, pf_bytes, t, gridDim.x);   // weights: no dependency on earlier kernels
     pdl_wait();
     if (zero_flags != nullptr && t == 0)
         for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
@@ -291,10 +290,10 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, int* zero_flags, int n_flags, PrefetchSpan pf, cudaStream_t st) {
+                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st) {
     return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
                       part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, (T + 15) / 16 * 16, pos, rope, hd,
-                      rope_base, zero_flags, n_flags, (const uint8_t*)pf.ptr, pf.bytes);
+                      rope_base, zero_flags, n_flags);
 }
 
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
