@@ -123,6 +123,19 @@ def plant_tokens(cats, fwd, parent, rank, vocab, seed_key, p_keep=0.7):
     return tokens
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of floats over all ranks (identity when not launched under torchrun)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if torch.distributed.is_available() and torch.distributed.is_initialized() and torch.distributed.get_world_size() > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(tree_nodes, world, sec_per_step):
+    """Replicas: every rank scores its own tree per step; the job's throughput is the sum over ranks, per the slowest rank."""
+    return world * tree_nodes / sec_per_step
+
+
 def time_steps(fn, steps, warmup, stream):
     for _ in range(warmup):
         fn()
@@ -234,10 +247,7 @@ def run_ours(args, rank, world, local_rank):
             sweep[str(T_)] = {"tok_s": T_ / r["sec_per_step"], "ms": r["sec_per_step"] * 1e3,
                               "gbs": b / r["sec_per_step"] / 1e9, "accepted": r["accepted"]}
 
-    sec = torch.tensor([main["sec_per_step"], e2e_sec / args.steps], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(sec, op=torch.distributed.ReduceOp.MAX)
-    sec_step, sec_e2e = float(sec[0]), float(sec[1])
+    sec_step, sec_e2e = max_over_ranks([main["sec_per_step"], e2e_sec / args.steps], dev)
     if rank != 0:
         return None
     peak, peak_kind = measured_peaks()
@@ -246,14 +256,14 @@ def run_ours(args, rank, world, local_rank):
     gemm_sec = main["breakdown"]["gemm_only"]
     n_gemm = roofline.gemm_launches(shape)
     out = {
-        "metric": METRIC, "value": world * T / sec_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_value(T, world, sec_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec_step * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "cfg3: 32-layer 7B-shaped verification forward + LM head (vocab 32000), prefix 512, "
                                "top-k draft tree of T=%d nodes, greedy walk + KV compaction" % T,
                    "tree_nodes": T, "prefix_len": PREFIX, "replicas": world, "cuda_graph": not args.no_graph,
                    "l2": "inputs_larger_than_l2 (13.5 GB of weights per step)", "accepted_tokens_per_step": main["accepted"]},
-        "e2e": {"value": world * T / sec_e2e, "unit": UNIT, "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 16 + 2 * T * 4},
+        "e2e": {"value": whole_job_value(T, world, sec_e2e), "unit": UNIT, "h2d_bytes_per_step": 2 * T * 4, "d2h_bytes_per_step": 16 + 2 * T * 4},
         "gpu_launches": main["launches"] * args.steps,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "k_gemm_sk (all %d projection launches of a forward)" % n_gemm,
