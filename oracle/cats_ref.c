@@ -181,6 +181,10 @@ void cats_ref_rope_head(double *x, int32_t hd, int32_t pos, double base) {
     }
 }
 
+int cats_ref_tree_attention_rows(const double *q, const float *kc, const float *vc, const uint64_t *mask,
+                                 int32_t nq, int32_t T, int32_t P, int32_t nh, int32_t hd,
+                                 int64_t kv_row_stride, double scale, double *out, double *probs);
+
 /* ---- O3 attention (tree-masked): node i of head h attends to every prefix
  * row [0,P) and to tree row P+j iff bit j of mask[i] is set; softmax of
  * scale * q.k over the visible columns; out = sum p * v.
@@ -191,11 +195,22 @@ void cats_ref_rope_head(double *x, int32_t hd, int32_t pos, double base) {
 int cats_ref_tree_attention(const double *q, const float *kc, const float *vc, const uint64_t *mask,
                             int32_t T, int32_t P, int32_t nh, int32_t hd, int64_t kv_row_stride,
                             double scale, double *out, double *probs) {
-    if (T < 1 || T > CATS_REF_MAX_T || P < 0) return -1;
+    return cats_ref_tree_attention_rows(q, kc, vc, mask, T, T, P, nh, hd, kv_row_stride, scale, out, probs);
+}
+
+/* The same attention for nq query rows that need not be all T tree nodes: query
+ * i carries its own 128-bit visibility row mask[i] over the T tree rows P..P+T-1
+ * (Stage 2 of Algorithm 1 re-forwards only the correction nodes "under
+ * tree-masked attention"; the other tree rows are already in the cache).
+ * q, out [nq][nh][hd]; probs (optional) [nh][nq][P+T]. */
+int cats_ref_tree_attention_rows(const double *q, const float *kc, const float *vc, const uint64_t *mask,
+                                 int32_t nq, int32_t T, int32_t P, int32_t nh, int32_t hd,
+                                 int64_t kv_row_stride, double scale, double *out, double *probs) {
+    if (T < 1 || T > CATS_REF_MAX_T || nq < 1 || nq > T || P < 0) return -1;
     int S = P + T;
 #pragma omp parallel for schedule(static) collapse(2)
     for (int h = 0; h < nh; ++h) {
-        for (int i = 0; i < T; ++i) {
+        for (int i = 0; i < nq; ++i) {
             double *s = (double *)malloc((size_t)S * sizeof(double));
             unsigned char *vis = (unsigned char *)malloc((size_t)S);
             const double *qi = q + ((size_t)i * nh + h) * hd;
@@ -222,7 +237,7 @@ int cats_ref_tree_attention(const double *q, const float *kc, const float *vc, c
             for (int e = 0; e < hd; ++e) oi[e] = 0.0;
             for (int c = 0; c < S; ++c) {
                 double p = vis[c] ? s[c] / l : 0.0;
-                if (probs) probs[((size_t)h * T + i) * S + c] = p;
+                if (probs) probs[((size_t)h * nq + i) * S + c] = p;
                 if (!vis[c]) continue;
                 const float *vr = vc + (size_t)c * kv_row_stride + (size_t)h * hd;
                 for (int e = 0; e < hd; ++e) oi[e] += p * (double)vr[e];
@@ -288,6 +303,65 @@ int cats_ref_verify_layer(const cats_ref_cfg *cfg, const cats_ref_layer_weights 
     for (size_t i = 0; i < (size_t)T * H; ++i) resid[i] = (float)((double)resid[i] + y[i]);
 
     free(xn); free(q); free(k); free(v); free(o); free(y); free(g); free(u);
+    return 0;
+}
+
+/* ---- O3 over a subset of the tree (Algorithm 1, Stage 2: the correction
+ * tokens are "re-forwarded from layer 1 through L_SV under tree-masked
+ * attention"; the main-chain nodes already have their K/V in these layers).
+ * nodes[0..m) are tree node indices, strictly ascending; resid [m][H] holds the
+ * hidden states of those nodes only.  The K/V of node nodes[j] is written to
+ * cache row P + nodes[j]; every other cache row is read-only.  Node nodes[j]
+ * attends to the prefix and to the tree rows its mask row names, which must
+ * be rows of active nodes or rows cached earlier. */
+int cats_ref_verify_layer_nodes(const cats_ref_cfg *cfg, const cats_ref_layer_weights *w, float *resid,
+                                float *kc, float *vc, const uint64_t *mask /*[T][2]*/, const int32_t *pos /*[T]*/,
+                                const int32_t *nodes, int32_t m, int32_t T, int32_t P) {
+    int H = cfg->hidden, nh = cfg->n_heads, hd = cfg->head_dim, F = cfg->ffn;
+    int D = nh * hd;
+    if (T < 1 || T > CATS_REF_MAX_T || m < 1 || m > T || P < 0 || P + T > cfg->max_seq || (hd & 1)) return -1;
+    for (int j = 0; j < m; ++j)
+        if (nodes[j] < 0 || nodes[j] >= T || (j > 0 && nodes[j] <= nodes[j - 1])) return -2;
+    double *xn = (double *)malloc((size_t)m * H * sizeof(double));
+    double *q = (double *)malloc((size_t)m * D * sizeof(double));
+    double *k = (double *)malloc((size_t)m * D * sizeof(double));
+    double *v = (double *)malloc((size_t)m * D * sizeof(double));
+    double *o = (double *)malloc((size_t)m * D * sizeof(double));
+    double *y = (double *)malloc((size_t)m * H * sizeof(double));
+    double *g = (double *)malloc((size_t)m * F * sizeof(double));
+    double *u = (double *)malloc((size_t)m * F * sizeof(double));
+    uint64_t *mrows = (uint64_t *)malloc((size_t)m * 2 * sizeof(uint64_t));
+
+    cats_ref_rmsnorm(resid, w->attn_norm, m, H, cfg->rms_eps, xn);
+    cats_ref_linear(w->wq, D, H, xn, m, q);
+    cats_ref_linear(w->wk, D, H, xn, m, k);
+    cats_ref_linear(w->wv, D, H, xn, m, v);
+    for (int j = 0; j < m; ++j) {
+        int n = nodes[j];
+        for (int h = 0; h < nh; ++h) {
+            cats_ref_rope_head(q + (size_t)j * D + (size_t)h * hd, hd, pos[n], (double)cfg->rope_base);
+            cats_ref_rope_head(k + (size_t)j * D + (size_t)h * hd, hd, pos[n], (double)cfg->rope_base);
+        }
+        for (int e = 0; e < D; ++e) {
+            q[(size_t)j * D + e] = rnd16(q[(size_t)j * D + e]);
+            kc[(size_t)(P + n) * D + e] = (float)rnd16(k[(size_t)j * D + e]);
+            vc[(size_t)(P + n) * D + e] = (float)rnd16(v[(size_t)j * D + e]);
+        }
+        mrows[2 * j] = mask[2 * n];
+        mrows[2 * j + 1] = mask[2 * n + 1];
+    }
+    cats_ref_tree_attention_rows(q, kc, vc, mrows, m, T, P, nh, hd, D, 1.0 / sqrt((double)hd), o, NULL);
+    cats_ref_linear(w->wo, H, D, o, m, y);
+    for (size_t i = 0; i < (size_t)m * H; ++i) resid[i] = (float)((double)resid[i] + y[i]);
+
+    cats_ref_rmsnorm(resid, w->mlp_norm, m, H, cfg->rms_eps, xn);
+    cats_ref_linear(w->w_gate, F, H, xn, m, g);
+    cats_ref_linear(w->w_up, F, H, xn, m, u);
+    for (size_t i = 0; i < (size_t)m * F; ++i) g[i] = rnd16(silu(g[i]) * u[i]);
+    cats_ref_linear(w->w_down, H, F, g, m, y);
+    for (size_t i = 0; i < (size_t)m * H; ++i) resid[i] = (float)((double)resid[i] + y[i]);
+
+    free(xn); free(q); free(k); free(v); free(o); free(y); free(g); free(u); free(mrows);
     return 0;
 }
 

@@ -13,7 +13,7 @@ from .build import build as _build
 
 __all__ = [
     "RefCfg", "set_contract", "set_accum32", "to_bf16", "from_bf16", "build_tree_mask", "rmsnorm", "linear",
-    "rope_head", "tree_attention", "verify_layer", "embed", "lm_head_argmax", "accept_path",
+    "rope_head", "tree_attention", "tree_attention_rows", "verify_layer", "verify_layer_nodes", "embed", "lm_head_argmax", "accept_path",
     "compact_kv", "verify_forward", "n_threads",
 ]
 
@@ -133,6 +133,22 @@ def tree_attention(q, kc, vc, mask, P, nh, hd, scale, kv_row_stride=None, want_p
     return (out, probs) if want_probs else out
 
 
+def tree_attention_rows(q, kc, vc, mask_rows, T, P, nh, hd, scale):
+    """nq query rows, each with its own visibility row over the T tree rows (see cats_ref.c)."""
+    q = _chk(q, np.float64, "q")
+    kc = _chk(kc, np.float32, "kc")
+    vc = _chk(vc, np.float32, "vc")
+    mask_rows = _chk(mask_rows, np.uint64, "mask_rows")
+    nq = q.shape[0]
+    assert mask_rows.shape == (nq, 2) and kc.size >= (P + T) * nh * hd
+    out = np.empty((nq, nh, hd), np.float64)
+    rc = _lib.cats_ref_tree_attention_rows(_p(q), _p(kc), _p(vc), _p(mask_rows), C.c_int32(nq), C.c_int32(T),
+                                           C.c_int32(P), C.c_int32(nh), C.c_int32(hd), C.c_int64(nh * hd),
+                                           C.c_double(scale), _p(out), None)
+    assert rc == 0, rc
+    return out
+
+
 def _layer_struct(w, keep):
     s = _LayerW()
     for n in LAYER_FIELDS:
@@ -156,6 +172,22 @@ def verify_layer(cfg: RefCfg, w: dict, resid, kc, vc, mask, pos, P, want_q=False
                                     C.c_int32(T), C.c_int32(P), _p(q))
     assert rc == 0, rc
     return q
+
+
+def verify_layer_nodes(cfg: RefCfg, w: dict, resid, kc, vc, mask, pos, nodes, P):
+    """The layer over the tree nodes `nodes` only (ascending).  In place on resid (float32 [m,H]) and on the cache rows
+    P + nodes[j]; mask [T,2] and pos [T] describe the whole tree."""
+    assert resid.dtype == np.float32 and resid.flags.c_contiguous
+    assert kc.dtype == np.float32 and kc.flags.c_contiguous and vc.dtype == np.float32 and vc.flags.c_contiguous
+    mask = _chk(mask, np.uint64, "mask")
+    pos = _chk(pos, np.int32, "pos")
+    nodes = _chk(nodes, np.int32, "nodes")
+    assert resid.shape[0] == nodes.shape[0]
+    keep = []
+    s = _layer_struct(w, keep)
+    rc = _lib.cats_ref_verify_layer_nodes(C.byref(cfg), C.byref(s), _p(resid), _p(kc), _p(vc), _p(mask), _p(pos),
+                                          _p(nodes), C.c_int32(nodes.shape[0]), C.c_int32(pos.shape[0]), C.c_int32(P))
+    return rc
 
 
 def embed(E, tokens):
