@@ -127,6 +127,27 @@ int cats_verify_layer(const cats_model_cfg *cfg, const cats_layer_weights *w, fl
                       void *d_vcache, const uint64_t *d_mask, const int32_t *d_pos, int32_t T,
                       int32_t prefix_len, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
 
+/* The same layer over a SUBSET of the tree (Algorithm 1, Stage 2: the
+ * correction tokens are re-forwarded through layers 1..L_SV "under tree-masked
+ * attention" while the main-chain nodes already have their K/V in those
+ * layers).
+ *   d_nodes [m] int32, device: tree node indices, strictly ascending, in [0,T).
+ *   d_resid [m][hidden] fp32 in/out: hidden states of those nodes only.
+ *   d_mask [T][2], d_pos [T]: of the WHOLE tree (cats_build_tree_mask).
+ *   Row j is rotated to d_pos[d_nodes[j]], its K/V are written to cache row
+ *   prefix_len + d_nodes[j], and it attends to the prefix and to the tree rows
+ *   mask row d_nodes[j] names.  Every cache row prefix_len..prefix_len+T-1
+ *   that this call does not write is only read and must hold finite values
+ *   (rows the mask hides are multiplied by a probability of exactly zero).
+ *   The workspace is the one cats_workspace_bytes(cfg, T, ...) sizes.
+ * A malformed node list sets *d_status = CATS_ERR_INVALID_ARG; the layer then
+ * runs on the list clamped into [0,T) (no access leaves the buffers) and its
+ * results are unspecified. */
+int cats_verify_layer_nodes(const cats_model_cfg *cfg, const cats_layer_weights *w, float *d_resid, void *d_kcache,
+                            void *d_vcache, const uint64_t *d_mask, const int32_t *d_pos, const int32_t *d_nodes,
+                            int32_t m, int32_t T, int32_t prefix_len, void *d_ws, size_t ws_bytes,
+                            int32_t *d_status, void *stream);
+
 /* Tree-masked attention alone: node i of every head attends to cache rows
  * [0,prefix_len) and to row prefix_len+j iff bit j of d_mask[i] is set
  * (Fig. 4, tree attention mask; softmax(q.k * scale) v).

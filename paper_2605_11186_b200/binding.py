@@ -60,6 +60,8 @@ lib.cats_build_tree_mask.argtypes = [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp]
 lib.cats_embed_tokens.argtypes = [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
 lib.cats_verify_layer.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp,
                                   C.c_size_t, _vp, _vp]
+lib.cats_verify_layer_nodes.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32,
+                                        _i32, _vp, C.c_size_t, _vp, _vp]
 lib.cats_tree_attention.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, C.c_float, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.cats_lm_head_argmax.argtypes = [C.POINTER(ModelCfg), _vp, _vp, _vp, _i32, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.cats_accept_path.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -209,6 +211,13 @@ def cats_embed_tokens(embed, tokens, resid, status):
 def cats_verify_layer(cfg, w: LayerWeights, resid, kcache, vcache, mask, pos, T, prefix_len, ws, status):
     _check(lib.cats_verify_layer(C.byref(cfg), C.byref(w), _ptr(resid), _ptr(kcache), _ptr(vcache), _ptr(mask), _ptr(pos), T,
                                  prefix_len, _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_verify_layer")
+
+
+def cats_verify_layer_nodes(cfg, w: LayerWeights, resid, kcache, vcache, mask, pos, nodes, T, prefix_len, ws, status):
+    """The layer over the tree nodes `nodes` (int32 device tensor, ascending) of a tree of T nodes; resid [len(nodes), H]."""
+    _check(lib.cats_verify_layer_nodes(C.byref(cfg), C.byref(w), _ptr(resid), _ptr(kcache), _ptr(vcache), _ptr(mask), _ptr(pos),
+                                       _ptr(nodes), nodes.numel(), T, prefix_len, _ptr(ws), ws.numel(), _ptr(status), _stream()),
+           "cats_verify_layer_nodes")
 
 
 def cats_tree_attention(q, k, v, mask, T, prefix_len, n_heads, head_dim, kv_row_stride, scale, out, ws, status):

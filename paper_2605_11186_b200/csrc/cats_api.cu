@@ -31,6 +31,7 @@ struct Workspace {
     float* fix_part;
     int* fix_flags;
     float* scratch;             // [T][hidden] fp32
+    int32_t* nodes;             // [CATS_MAX_TREE] clamped node list of a partial-tree forward
     size_t bytes;
 };
 
@@ -60,6 +61,7 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     w.fix_part = (float*)take((size_t)kGemmCtas * tpad * 128 * 4);
     w.fix_flags = (int*)take((size_t)kGemmCtas * sizeof(int));
     w.scratch = (float*)take((size_t)T * c->hidden * 4);
+    w.nodes = (int32_t*)take((size_t)CATS_MAX_TREE * sizeof(int32_t));
     w.bytes = off;
     return w;
 }
@@ -81,21 +83,24 @@ inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintp
         if (e__ != cudaSuccess) return CATS_ERR_CUDA; \
     } while (0)
 
-// One decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still
+// One decoder layer over T rows.  nodes == nullptr: the rows are the T tree nodes.  Else row t is tree node nodes[t] of
+// a tree of T_tree nodes (mask and pos describe that whole tree): its K/V go to cache row P + nodes[t], it is rotated
+// to pos[nodes[t]] and attends under mask row nodes[t]; the other tree rows are read from the cache.  n_pending: split-K partial sums of the previous layer's down projection still
 // to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
 // sums this layer's down projection left pending (>0) or a negative status.
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               const void* next_w, size_t next_w_bytes, bool next_is_head, int32_t* d_status, cudaStream_t st) {
+               const void* next_w, size_t next_w_bytes, bool next_is_head, int32_t* d_status, cudaStream_t st,
+               const int32_t* nodes = nullptr, int T_tree = 0) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
-    g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P;
+    g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P; g.kv_rows = nodes;
     g.d_status = d_status;
     GemmProblem nxt = {};
     nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = D; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->wo;
@@ -106,6 +111,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     a.q = ws.q; a.k = kc; a.v = vc; a.mask = mask; a.T = T; a.prefix_len = P; a.nh = c->n_heads; a.hd = c->head_dim;
     a.kv_stride = D; a.scale = 1.0f / sqrtf((float)c->head_dim); a.out = ws.o; a.out_packed_npad = tpad;
     a.part_o = ws.attn_o; a.part_ml = ws.attn_ml; a.d_status = d_status;
+    a.nodes = nodes; a.T_tree = nodes ? T_tree : 0;
     attn_plan(a);
     if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
@@ -119,7 +125,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                                 nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
+                                 nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
 
     g = GemmProblem{};
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
@@ -145,7 +151,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -278,7 +284,35 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
+                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
+    return CATS_OK;
+}
+
+int cats_verify_layer_nodes(const cats_model_cfg* cfg, const cats_layer_weights* w, float* d_resid, void* d_kcache,
+                            void* d_vcache, const uint64_t* d_mask, const int32_t* d_pos, const int32_t* d_nodes, int32_t m,
+                            int32_t T, int32_t prefix_len, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    int rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!w || !d_resid || !d_kcache || !d_vcache || !d_mask || !d_pos || !d_nodes || !d_ws || !d_status) return CATS_ERR_INVALID_ARG;
+    if (!w->attn_norm || !w->wqkv || !w->wo || !w->mlp_norm || !w->w_gate_up || !w->w_down) return CATS_ERR_INVALID_ARG;
+    rc = check_tree_args(T, prefix_len);
+    if (rc) return rc;
+    if (m < 1 || m > T || prefix_len + T > cfg->max_seq) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(d_resid, 16) || misaligned(d_kcache, 16) || misaligned(d_vcache, 16)) return CATS_ERR_INVALID_ARG;
+    const void* ws_ptrs[] = {w->wqkv, w->wo, w->w_gate_up, w->w_down, w->attn_norm, w->mlp_norm};
+    for (const void* p : ws_ptrs) if (misaligned(p, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, m, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    CATS_CUDA(launch_check_nodes(d_nodes, m, T, ws.nodes, d_status, st));
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, m, prefix_len, ws, 0, nullptr, 0,
+                             false, d_status, st, ws.nodes, T);
+    if (pending < 0) return pending;
+    CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, m, cfg->hidden, cfg->rms_eps, nullptr,
+                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
     return CATS_OK;
 }
 

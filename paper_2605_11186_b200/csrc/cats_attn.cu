@@ -49,6 +49,8 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 struct AttnDev {
     const uint16_t *q, *k, *v;
     const uint64_t* mask;
+    const int32_t* nodes;   // null, or the tree node of each query row (selects its mask row)
+    int Tk;                 // tree rows in the cache after the prefix
     int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split, blk, kv_area;   // blk: cache rows per pipeline block (multiple of 16*kvg); kv_area: bytes of the K/V buffers
     long long kv_stride;
     float scale_log2;
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y;
-    const int S = p.P + p.T;
+    const int S = p.P + p.Tk;
     const int c_begin = min(S, split * p.rows_per_split);
     const int c_end = min(S, c_begin + p.rows_per_split);
     const int nb = (c_end - c_begin + p.blk - 1) / p.blk;
@@ -129,7 +131,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         if (r < p.T) cp_async16(q_s + off, p.q + ((size_t)r * p.nh + h) * HD + ch * 8);
         else *reinterpret_cast<uint4*>(q_s + off) = make_uint4(0, 0, 0, 0);
     }
-    for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) mask_s[e] = (e < p.T * 2) ? p.mask[e] : 0ull;
+    for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) {
+        uint64_t w = 0ull;
+        if (e < p.T * 2) w = p.nodes != nullptr ? p.mask[(size_t)p.nodes[e >> 1] * 2 + (e & 1)] : p.mask[e];
+        mask_s[e] = w;
+    }
     if (!early && nb > 0) load_kv(0, 0);
     cp_async_commit();
 
@@ -347,7 +353,7 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
 // Chooses the cluster size (CTAs per head that share one merge through distributed shared memory) and, for long
 // prefixes with few heads, the number of clusters per head.  Returns the bytes of workspace the outer merge needs.
 size_t attn_plan(AttnProblem& p) {
-    const int S = p.prefix_len + p.T;
+    const int S = p.prefix_len + (p.T_tree > 0 ? p.T_tree : p.T);
     const int units16 = (S + 15) / 16;
     const int tpad = ((p.T + 15) / 16) * 16;
     // as many CTAs per head as fit one wave of the 148 SMs (each CTA fills an SM), at most 8, at least 32 rows each
@@ -406,6 +412,8 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     AttnDev d;
     d.q = (const uint16_t*)p.q; d.k = (const uint16_t*)p.k; d.v = (const uint16_t*)p.v;
     d.mask = p.mask;
+    d.nodes = p.nodes;
+    d.Tk = p.T_tree > 0 ? p.T_tree : p.T;
     d.T = p.T; d.P = p.prefix_len; d.nh = p.nh;
     d.n_mt = (p.T + 15) / 16;
     d.kvg = 8 / d.n_mt;

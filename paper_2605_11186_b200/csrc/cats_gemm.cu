@@ -51,6 +51,7 @@ struct GemmDev {
     uint16_t *q_out, *kcache, *vcache;
     const float2* rope;
     int head_dim, prefix_len;
+    const int32_t* kv_rows;
     uint8_t* act_out;     // packed activation layout
     float* logits;
     float* pmax;
@@ -390,12 +391,23 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                                     packed[it] = pack_bf16x2(x.x, x.y);
                                 }
                             }
-                            uint16_t* base = mat == 0 ? p.q_out + (size_t)c0 * p.n_out
-                                                      : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
+                            if (mat == 0 || p.kv_rows == nullptr) {
+                                uint16_t* base = mat == 0 ? p.q_out + (size_t)c0 * p.n_out
+                                                          : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
 #pragma unroll
-                            for (int it = 0; it < NI; ++it) {
-                                const int nl = (et >> 6) + 2 * it;
-                                if (nl < n_hi) *reinterpret_cast<uint32_t*>(base + (size_t)nl * p.n_out + feat) = packed[it];
+                                for (int it = 0; it < NI; ++it) {
+                                    const int nl = (et >> 6) + 2 * it;
+                                    if (nl < n_hi) *reinterpret_cast<uint32_t*>(base + (size_t)nl * p.n_out + feat) = packed[it];
+                                }
+                            } else {
+                                // a subset of the tree: row t of the batch is tree node kv_rows[t]
+                                uint16_t* base = (mat == 1 ? p.kcache : p.vcache) + (size_t)p.prefix_len * p.n_out;
+#pragma unroll
+                                for (int it = 0; it < NI; ++it) {
+                                    const int nl = (et >> 6) + 2 * it;
+                                    if (nl < n_hi)
+                                        *reinterpret_cast<uint32_t*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
+                                }
                             }
                         }
                     } else if (p.epi == EPI_SWIGLU) {
@@ -606,6 +618,7 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.rope = p.rope;
     d.head_dim = p.head_dim;
     d.prefix_len = p.prefix_len;
+    d.kv_rows = p.kv_rows;
     d.act_out = (uint8_t*)p.act_out;
     d.logits = p.logits;
     d.pmax = p.pmax;

@@ -39,8 +39,10 @@ cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64
 cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int vocab, float* resid, int32_t* d_status,
                          cudaStream_t st);
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
-                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st);
+                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
+                           float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st);
+// Checks a partial-tree node list (strictly ascending, inside [0, T)) and writes a copy clamped into range.
+cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
@@ -82,6 +84,7 @@ struct GemmProblem {
     const float2* rope;    //   [T][head_dim/2] (cos, sin)
     int head_dim;
     int prefix_len;
+    const int32_t* kv_rows; //   null: node t goes to cache row prefix_len + t; else to prefix_len + kv_rows[t]
     void* act_out;         // EPI_SWIGLU: packed activations, ceil(n_out/64) K blocks
     float* logits;         // EPI_LMHEAD: [T][n_out] fp32 or null
     float* pmax;           //   [n_tiles][128]
@@ -110,7 +113,9 @@ struct AttnProblem {
     const void* k;      // rows of kv_stride elements, head h at h*hd
     const void* v;
     const uint64_t* mask;
-    int T, prefix_len, nh, hd;
+    int T, prefix_len, nh, hd;   // T: query rows
+    int T_tree;                  // tree rows in the cache after the prefix (0: the same as T)
+    const int32_t* nodes;        // null: query t is tree node t; else query t is tree node nodes[t] (its mask row)
     long long kv_stride;
     float scale;
     void* out;          // [T][nh][hd] bf16, or the packed activation layout if out_packed_npad > 0

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
                                                  const float* __restrict__ part, int n_part, size_t part_stride,
                                                  const uint16_t* __restrict__ gain, int H, float eps,
                                                  uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
-                                                 float2* __restrict__ rope, int hd, float rope_base, int* zero_flags,
+                                                 const int32_t* __restrict__ nodes, float2* __restrict__ rope, int hd, float rope_base, int* zero_flags,
                                                  int n_flags) {
     extern __shared__ float srow[];  // H floats
     __shared__ float red[8];
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
         for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
     if (rope != nullptr) {
         int half = hd / 2;
-        int p = pos[t];
+        int p = pos[nodes != nullptr ? nodes[t] : t];   // row t holds tree node nodes[t]
         for (int i = threadIdx.x; i < half; i += blockDim.x) {
             double inv_freq = pow((double)rope_base, -2.0 * (double)i / (double)hd);
             double s, c;
@@ -151,6 +151,24 @@ __global__ void __launch_bounds__(256) k_rmsnorm(float* __restrict__ resid, cons
             *reinterpret_cast<uint4*>(xn + packed_act_offset(t, c, n_pad)) = o;
         }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Node list of a partial-tree forward: must be strictly ascending indices into a tree of T nodes.
+// The layer's kernels index cache rows, mask rows and positions with it, so they are given a copy
+// clamped into [0, T) (a malformed list then cannot reach outside the caller's buffers); the
+// malformed list itself is reported through the status word.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_check_nodes(const int32_t* __restrict__ nodes, int m, int T, int32_t* __restrict__ clamped,
+                                                     int32_t* __restrict__ d_status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int j = threadIdx.x;
+    if (j >= m) return;
+    int n = nodes[j];
+    bool bad = n < 0 || n >= T || (j > 0 && nodes[j - 1] >= n);
+    clamped[j] = min(max(n, 0), T - 1);
+    if (bad) report(d_status, CATS_ERR_INVALID_ARG);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -289,11 +307,15 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 }
 
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
-                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, float2* rope, int hd,
-                           float rope_base, int* zero_flags, int n_flags, cudaStream_t st) {
+                           const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
+                           float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st) {
     return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
-                      part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, (T + 15) / 16 * 16, pos, rope, hd,
-                      rope_base, zero_flags, n_flags);
+                      part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, (T + 15) / 16 * 16, pos, nodes, rope,
+                      hd, rope_base, zero_flags, n_flags);
+}
+
+cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st) {
+    return launch_pdl(k_check_nodes, dim3(1), dim3(128), 0, st, nodes, m, T, clamped, d_status);
 }
 
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
