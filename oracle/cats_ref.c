@@ -425,6 +425,134 @@ int cats_ref_accept_path(const int32_t *parent, const int32_t *tokens, const int
     return 0;
 }
 
+/* ---- O5b: typical (relaxed) acceptance, the second criterion Acc of
+ * Algorithm 1 ("greedy or typical"; the tables' "relaxed (temperature = 0.7)"
+ * setting), as the cited Medusa work defines it: with p = softmax(logits / t)
+ * at the parent, a child token x is acceptable iff
+ *     p(x) > min(eps, delta * exp(-H(p))),      H(p) = -sum_v p_v log p_v.
+ * Per-node statistics by their definitions, in fp64:
+ *   lse[n]     = log sum_v exp(logits[n][v] / t)
+ *   entropy[n] = H(softmax(logits[n] / t))
+ *   cand_logit[i] = logits[parent[i]][tokens[i]]   (0 for the root)
+ *   prob[i]    = p_parent(i)(tokens[i])            (optional, fp64; 0 for the root)
+ * lse, entropy and cand_logit are delivered as fp32 (what the walk consumes). */
+int cats_ref_typical_stats(const float *logits, int32_t T, int32_t V, double temperature,
+                           const int32_t *parent, const int32_t *tokens, float *lse, float *entropy,
+                           float *cand_logit, double *prob) {
+    if (T < 1 || T > CATS_REF_MAX_T || V < 1 || !(temperature > 0.0)) return -1;
+    double *lse64 = (double *)malloc((size_t)T * sizeof(double));
+    for (int n = 0; n < T; ++n) {
+        const float *l = logits + (size_t)n * V;
+        double m = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+            double z = (double)l[v] / temperature;
+            if (z > m) m = z;
+        }
+        double Z = 0.0;
+        for (int v = 0; v < V; ++v) Z += exp((double)l[v] / temperature - m);
+        lse64[n] = m + log(Z);
+        double H = 0.0;
+        for (int v = 0; v < V; ++v) {
+            double lp = (double)l[v] / temperature - lse64[n];
+            double pv = exp(lp);
+            if (pv > 0.0) H -= pv * lp;
+        }
+        lse[n] = (float)lse64[n];
+        entropy[n] = (float)H;
+    }
+    for (int i = 0; i < T; ++i) {
+        int pa = parent[i];
+        if (i == 0 || pa < 0 || pa >= i || tokens[i] < 0 || tokens[i] >= V) {
+            cand_logit[i] = 0.f;
+            if (prob) prob[i] = 0.0;
+            continue;
+        }
+        float c = logits[(size_t)pa * V + tokens[i]];
+        cand_logit[i] = c;
+        if (prob) prob[i] = exp((double)c / temperature - lse64[pa]);
+    }
+    free(lse64);
+    return 0;
+}
+
+/* The walk of Algorithm 1 with a per-node verdict: starting at the root, take
+ * the first acceptable child in node order (on a CATS tree: the main draft
+ * token d_a, else the correction at that position), stop when none is; the
+ * bonus token is the argmax at the last accepted node. */
+static int walk_with_verdicts(const int32_t *parent, const int32_t *tokens, const int32_t *argmax,
+                              const unsigned char *ok, int32_t T, int32_t *path, int32_t *path_len,
+                              int32_t *out_tokens, int32_t *n_out) {
+    int cur = 0, len = 0, no = 0;
+    path[len++] = 0;
+    for (;;) {
+        int next = -1;
+        for (int j = cur + 1; j < T; ++j)
+            if (parent[j] == cur && ok[j]) { next = j; break; }
+        if (next < 0) break;
+        out_tokens[no++] = tokens[next];
+        path[len++] = next;
+        cur = next;
+    }
+    out_tokens[no++] = argmax[cur];
+    *path_len = len;
+    *n_out = no;
+    return 0;
+}
+
+/* Typical acceptance straight from the definition, in fp64, on the logits. */
+int cats_ref_accept_path_typical_def(const int32_t *parent, const int32_t *tokens, const int32_t *argmax,
+                                     const float *logits, int32_t T, int32_t V, double temperature,
+                                     double eps, double delta, int32_t *path, int32_t *path_len,
+                                     int32_t *out_tokens, int32_t *n_out) {
+    if (T < 1 || T > CATS_REF_MAX_T) return -1;
+    float lse[CATS_REF_MAX_T], H[CATS_REF_MAX_T], cand[CATS_REF_MAX_T];
+    double prob[CATS_REF_MAX_T];
+    unsigned char ok[CATS_REF_MAX_T];
+    /* entropy again in fp64 here, so that the verdict does not pass through fp32 */
+    int rc = cats_ref_typical_stats(logits, T, V, temperature, parent, tokens, lse, H, cand, prob);
+    if (rc) return rc;
+    ok[0] = 0;
+    for (int i = 1; i < T; ++i) {
+        int pa = parent[i];
+        const float *l = logits + (size_t)pa * V;
+        double m = -INFINITY, Z = 0.0, Hd = 0.0;
+        for (int v = 0; v < V; ++v) if ((double)l[v] / temperature > m) m = (double)l[v] / temperature;
+        for (int v = 0; v < V; ++v) Z += exp((double)l[v] / temperature - m);
+        for (int v = 0; v < V; ++v) {
+            double lp = (double)l[v] / temperature - m - log(Z);
+            if (exp(lp) > 0.0) Hd -= exp(lp) * lp;
+        }
+        double thr = delta * exp(-Hd);
+        if (eps < thr) thr = eps;
+        ok[i] = (unsigned char)(prob[i] > thr);
+    }
+    return walk_with_verdicts(parent, tokens, argmax, ok, T, path, path_len, out_tokens, n_out);
+}
+
+/* The same walk from the fp32 statistics, with the verdict taken in the log
+ * domain in fp32 and a fixed operation order, so that any implementation given
+ * the same inputs reaches the same verdict bit for bit:
+ *     logp = fma(cand_logit[i], inv_temperature, -lse[parent])        (one rounding)
+ *     thr  = min(log_eps, log_delta - entropy[parent])
+ *     acceptable iff logp > thr          (log is monotone: the same criterion). */
+int cats_ref_accept_path_typical(const int32_t *parent, const int32_t *tokens, const int32_t *argmax,
+                                 const float *cand_logit, const float *lse, const float *entropy, int32_t T,
+                                 float inv_temperature, float log_eps, float log_delta, int32_t *path,
+                                 int32_t *path_len, int32_t *out_tokens, int32_t *n_out) {
+    if (T < 1 || T > CATS_REF_MAX_T) return -1;
+    unsigned char ok[CATS_REF_MAX_T];
+    ok[0] = 0;
+    for (int i = 1; i < T; ++i) {
+        int pa = parent[i];
+        if (pa < 0 || pa >= i) return -2;
+        float logp = fmaf(cand_logit[i], inv_temperature, -lse[pa]);
+        volatile float d = log_delta - entropy[pa];
+        float thr = fminf(log_eps, d);
+        ok[i] = (unsigned char)(logp > thr);
+    }
+    return walk_with_verdicts(parent, tokens, argmax, ok, T, path, path_len, out_tokens, n_out);
+}
+
 /* ---- O6: KV rollback along the accepted path (Algorithm 1, "Roll back KV_M
  * ... to length s along the accepted path").  For every layer, K and V: row
  * P+path[k] moves to row P+k, k ascending, in place.  src/dst (optional)

@@ -14,7 +14,8 @@ from .build import build as _build
 __all__ = [
     "RefCfg", "set_contract", "set_accum32", "to_bf16", "from_bf16", "build_tree_mask", "rmsnorm", "linear",
     "rope_head", "tree_attention", "tree_attention_rows", "verify_layer", "verify_layer_nodes", "embed", "lm_head_argmax", "accept_path",
-    "compact_kv", "verify_forward", "n_threads",
+    "compact_kv", "verify_forward", "n_threads", "typical_stats", "accept_path_typical_def",
+    "accept_path_typical",
 ]
 
 _lib = C.CDLL(_build())
@@ -224,6 +225,59 @@ def accept_path(parent, tokens, argmax):
     rc = _lib.cats_ref_accept_path(_p(parent), _p(tokens), _p(argmax), C.c_int32(T), _p(path), C.byref(pl),
                                    _p(out), C.byref(no))
     assert rc == 0
+    return path[:pl.value].copy(), out[:no.value].copy()
+
+
+def typical_stats(logits, temperature, parent, tokens):
+    """Per-node softmax statistics at the given temperature: (lse f32 [T], entropy f32 [T], cand_logit f32 [T],
+    prob f64 [T] = p_parent(token))."""
+    logits = _chk(logits, np.float32, "logits")
+    parent = _chk(parent, np.int32, "parent")
+    tokens = _chk(tokens, np.int32, "tokens")
+    T, V = logits.shape
+    lse = np.empty(T, np.float32)
+    ent = np.empty(T, np.float32)
+    cand = np.empty(T, np.float32)
+    prob = np.empty(T, np.float64)
+    rc = _lib.cats_ref_typical_stats(_p(logits), C.c_int32(T), C.c_int32(V), C.c_double(temperature), _p(parent),
+                                     _p(tokens), _p(lse), _p(ent), _p(cand), _p(prob))
+    assert rc == 0, rc
+    return lse, ent, cand, prob
+
+
+def _walk_out(T):
+    return np.full(T, -1, np.int32), np.full(T, -1, np.int32), C.c_int32(0), C.c_int32(0)
+
+
+def accept_path_typical_def(parent, tokens, argmax, logits, temperature, eps, delta):
+    """Typical acceptance from its definition (fp64, on the logits).  Returns (path, out_tokens)."""
+    parent = _chk(parent, np.int32, "parent")
+    tokens = _chk(tokens, np.int32, "tokens")
+    argmax = _chk(argmax, np.int32, "argmax")
+    logits = _chk(logits, np.float32, "logits")
+    T, V = logits.shape
+    path, out, pl, no = _walk_out(T)
+    rc = _lib.cats_ref_accept_path_typical_def(_p(parent), _p(tokens), _p(argmax), _p(logits), C.c_int32(T), C.c_int32(V),
+                                               C.c_double(temperature), C.c_double(eps), C.c_double(delta), _p(path),
+                                               C.byref(pl), _p(out), C.byref(no))
+    assert rc == 0, rc
+    return path[:pl.value].copy(), out[:no.value].copy()
+
+
+def accept_path_typical(parent, tokens, argmax, cand_logit, lse, entropy, inv_temperature, log_eps, log_delta):
+    """The same walk from fp32 statistics, verdict in the log domain in fp32 (see cats_ref.c)."""
+    parent = _chk(parent, np.int32, "parent")
+    tokens = _chk(tokens, np.int32, "tokens")
+    argmax = _chk(argmax, np.int32, "argmax")
+    cand_logit = _chk(cand_logit, np.float32, "cand")
+    lse = _chk(lse, np.float32, "lse")
+    entropy = _chk(entropy, np.float32, "entropy")
+    T = parent.shape[0]
+    path, out, pl, no = _walk_out(T)
+    rc = _lib.cats_ref_accept_path_typical(_p(parent), _p(tokens), _p(argmax), _p(cand_logit), _p(lse), _p(entropy),
+                                           C.c_int32(T), C.c_float(inv_temperature), C.c_float(log_eps),
+                                           C.c_float(log_delta), _p(path), C.byref(pl), _p(out), C.byref(no))
+    assert rc == 0, rc
     return path[:pl.value].copy(), out[:no.value].copy()
 
 
