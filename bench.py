@@ -166,11 +166,11 @@ def run_ours(args, rank, world, local_rank):
     kc, vc = gen.make_kv_prefix(shape, shape.n_layers, max_seq, PREFIX, ("bench", rank), device=dev)
     stream = torch.cuda.current_stream()
 
-    def setup(T_):
+    def setup(T_, typical=None):
         parent, srank = gen.tree_topk_shape(T_, gen.topk_k_for(T_))
         fwd = cats.VerifyForward(shape, model, kc, vc, T_, PREFIX, want_logits=True, compact=True)
         tokens = plant_tokens(cats, fwd, parent, srank, shape.vocab, (rank,))
-        fwd_t = cats.VerifyForward(shape, model, kc, vc, T_, PREFIX, want_logits=False, compact=True)
+        fwd_t = cats.VerifyForward(shape, model, kc, vc, T_, PREFIX, want_logits=False, compact=True, typical=typical)
         return parent, tokens, fwd_t
 
     def graph_of(fwd, d_parent, d_tokens):
@@ -181,8 +181,8 @@ def run_ours(args, rank, world, local_rank):
             fwd.run(d_parent, d_tokens)
         return g
 
-    def measure(T_, steps, warmup, with_breakdown):
-        parent, tokens, fwd = setup(T_)
+    def measure(T_, steps, warmup, with_breakdown, typical=None):
+        parent, tokens, fwd = setup(T_, typical)
         d_parent, d_tokens = torch.from_numpy(parent).cuda(), torch.from_numpy(tokens).cuda()
         launches = None
         if args.no_graph:
@@ -247,6 +247,19 @@ def run_ours(args, rank, world, local_rank):
             sweep[str(T_)] = {"tok_s": T_ / r["sec_per_step"], "ms": r["sec_per_step"] * 1e3,
                               "gbs": b / r["sec_per_step"] / 1e9, "accepted": r["accepted"]}
 
+    # the rows built after the greedy path: the same forward under typical acceptance (softmax statistics in the LM-head
+    # epilogue, relaxed walk), and the draft-stage shape (a one-token pass, the other weight-streaming loop of a cycle)
+    widening = {}
+    if rank == 0 and not args.no_sweep:
+        import math
+        typ = (np.float32(1.0) / np.float32(0.7), np.float32(math.log(0.09)), np.float32(math.log(0.3)))
+        r, _, _, _ = measure(T, max(5, args.steps // 2), 3, with_breakdown=False, typical=typ)
+        widening["typical_acceptance"] = {"tree_nodes": T, "ms": r["sec_per_step"] * 1e3, "tok_s": T / r["sec_per_step"],
+                                          "accepted": r["accepted"], "temperature": 0.7, "eps": 0.09, "delta": 0.3}
+        r, _, _, _ = measure(1, max(5, args.steps // 2), 3, with_breakdown=False)
+        b1 = roofline.forward_bytes(shape, PREFIX, 1)
+        widening["one_token_pass"] = {"tree_nodes": 1, "ms": r["sec_per_step"] * 1e3, "gbs": b1 / r["sec_per_step"] / 1e9}
+
     sec_step, sec_e2e = max_over_ranks([main["sec_per_step"], e2e_sec / args.steps], dev)
     if rank != 0:
         return None
@@ -277,6 +290,7 @@ def run_ours(args, rank, world, local_rank):
                      "forward_frac_of_8TBs": fb / sec_step / 8e12},
         "breakdown_ms": {k: v * 1e3 for k, v in main["breakdown"].items()},
         "sweep": sweep,
+        "widening": widening,
     }
     return out
 

@@ -204,6 +204,40 @@ int cats_accept_path(const int32_t *d_parent, const int32_t *d_tokens, const int
                      int32_t *d_path, int32_t *d_path_len, int32_t *d_out_tokens, int32_t *d_n_out,
                      int32_t *d_status, void *stream);
 
+/* Typical (relaxed) acceptance, the second criterion Acc of Algorithm 1
+ * ("greedy or typical"; the tables' relaxed setting at temperature 0.7), as the
+ * cited Medusa work defines it: with p = softmax(logits / t) at the parent, a
+ * child token x is acceptable iff  p(x) > min(eps, delta * exp(-H(p))).
+ *
+ * cats_lm_head_typical is cats_lm_head_argmax that also leaves, per node,
+ *   d_lse [T] fp32        log sum_v exp(logits[n][v] / t)
+ *   d_entropy [T] fp32    H(softmax(logits[n] / t))
+ *   d_cand_logit [T] fp32 logits[parent[i]][tokens[i]] (0 for the root and for
+ *                         tokens outside the vocabulary)
+ * computed inside the LM-head kernel from its fp32 accumulators (the logits
+ * need not be written).  d_parent, d_tokens: [T] int32, the tree.
+ * inv_temperature = 1/t as fp32, 0 < 1/t < 1e6.
+ *
+ * cats_accept_path_typical walks the tree as Algorithm 1's loop does: from the
+ * root, take the FIRST acceptable child in node order (the main draft token
+ * before the correction at the same position), stop when there is none; the
+ * bonus token is d_argmax at the last accepted node.  The verdict is taken in
+ * the log domain in fp32, round to nearest, in this order:
+ *     fma(d_cand_logit[i], inv_temperature, -d_lse[parent]) >
+ *         min(log_eps, log_delta - d_entropy[parent])
+ * so the caller passes log(eps) and log(delta) (the cited defaults: eps = 0.09,
+ * delta = 0.3).  Outputs as cats_accept_path. */
+int cats_lm_head_typical(const cats_model_cfg *cfg, const void *d_final_norm, const void *d_w_lm,
+                         const float *d_resid, const int32_t *d_parent, const int32_t *d_tokens, int32_t T,
+                         float inv_temperature, float *d_logits, int32_t *d_argmax, float *d_lse,
+                         float *d_entropy, float *d_cand_logit, void *d_ws, size_t ws_bytes,
+                         int32_t *d_status, void *stream);
+int cats_accept_path_typical(const int32_t *d_parent, const int32_t *d_tokens, const int32_t *d_argmax,
+                             const float *d_cand_logit, const float *d_lse, const float *d_entropy, int32_t T,
+                             float inv_temperature, float log_eps, float log_delta, int32_t *d_path,
+                             int32_t *d_path_len, int32_t *d_out_tokens, int32_t *d_n_out,
+                             int32_t *d_status, void *stream);
+
 /* KV roll-back along the accepted path (Algorithm 1, "Roll back KV_M ... to
  * length s along the accepted path"): for every layer, K and V, row
  * prefix_len + d_path[k] moves to row prefix_len + k, in place;
@@ -214,6 +248,8 @@ int cats_compact_kv(void *d_kcache, void *d_vcache, int32_t n_layers, int64_t la
                     int64_t row_elems, int32_t prefix_len, const int32_t *d_path, const int32_t *d_path_len,
                     int32_t *d_new_len, int32_t *d_src_rows, int32_t *d_dst_rows, int32_t *d_status,
                     void *stream);
+
+enum { CATS_ACCEPT_GREEDY = 0, CATS_ACCEPT_TYPICAL = 1 };
 
 /* Arguments of a whole verification forward (Stage 3 plus walk and roll-back). */
 typedef struct {
@@ -236,6 +272,11 @@ typedef struct {
     void *d_ws;
     size_t ws_bytes;
     int32_t *d_status;
+    /* acceptance criterion of the walk */
+    int32_t accept_mode;              /* CATS_ACCEPT_GREEDY or CATS_ACCEPT_TYPICAL */
+    float inv_temperature;            /* typical: 1/t, log(eps), log(delta) as for cats_accept_path_typical */
+    float log_eps, log_delta;
+    float *d_typical;                 /* typical: [3][T] fp32 out: lse, entropy, candidate logits */
 } cats_forward_args;
 
 /* The whole path on device buffers: mask/pos, embedding (or caller's hidden

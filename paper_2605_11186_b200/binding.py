@@ -46,7 +46,12 @@ class ForwardArgs(C.Structure):
                 ("d_hidden_in", C.c_void_p), ("T", C.c_int32), ("prefix_len", C.c_int32), ("compact", C.c_int32),
                 ("d_mask", C.c_void_p), ("d_pos", C.c_void_p), ("d_depth", C.c_void_p), ("d_resid", C.c_void_p),
                 ("d_logits", C.c_void_p), ("d_argmax", C.c_void_p), ("d_path", C.c_void_p), ("d_out_tokens", C.c_void_p),
-                ("d_scalars", C.c_void_p), ("d_ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("d_status", C.c_void_p)]
+                ("d_scalars", C.c_void_p), ("d_ws", C.c_void_p), ("ws_bytes", C.c_size_t), ("d_status", C.c_void_p),
+                ("accept_mode", C.c_int32), ("inv_temperature", C.c_float), ("log_eps", C.c_float), ("log_delta", C.c_float),
+                ("d_typical", C.c_void_p)]
+
+
+ACCEPT_GREEDY, ACCEPT_TYPICAL = 0, 1
 
 
 lib.cats_status_string.restype = C.c_char_p
@@ -65,6 +70,10 @@ lib.cats_verify_layer_nodes.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeig
 lib.cats_tree_attention.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i64, C.c_float, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.cats_lm_head_argmax.argtypes = [C.POINTER(ModelCfg), _vp, _vp, _vp, _i32, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.cats_accept_path.argtypes = [_vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.cats_lm_head_typical.argtypes = [C.POINTER(ModelCfg), _vp, _vp, _vp, _vp, _vp, _i32, C.c_float, _vp, _vp, _vp, _vp, _vp, _vp,
+                                     C.c_size_t, _vp, _vp]
+lib.cats_accept_path_typical.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, C.c_float, C.c_float, C.c_float, _vp, _vp, _vp,
+                                         _vp, _vp, _vp]
 lib.cats_compact_kv.argtypes = [_vp, _vp, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.cats_verify_forward.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp]
 lib.cats_verify_forward_host.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -243,6 +252,21 @@ def cats_lm_head_argmax(cfg, final_norm, w_lm, resid, T, logits, argmax, ws, sta
                                    _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_lm_head_argmax")
 
 
+def cats_lm_head_typical(cfg, final_norm, w_lm, resid, parent, tokens, T, inv_temperature, logits, argmax, lse, entropy,
+                         cand_logit, ws, status):
+    _check(lib.cats_lm_head_typical(C.byref(cfg), _ptr(final_norm), _ptr(w_lm), _ptr(resid), _ptr(parent), _ptr(tokens), T,
+                                    float(inv_temperature), _ptr(logits), _ptr(argmax), _ptr(lse), _ptr(entropy),
+                                    _ptr(cand_logit), _ptr(ws), ws.numel(), _ptr(status), _stream()), "cats_lm_head_typical")
+
+
+def cats_accept_path_typical(parent, tokens, argmax, cand_logit, lse, entropy, T, inv_temperature, log_eps, log_delta, path,
+                             path_len, out_tokens, n_out, status):
+    _check(lib.cats_accept_path_typical(_ptr(parent), _ptr(tokens), _ptr(argmax), _ptr(cand_logit), _ptr(lse), _ptr(entropy),
+                                        T, float(inv_temperature), float(log_eps), float(log_delta), _ptr(path),
+                                        _ptr(path_len), _ptr(out_tokens), _ptr(n_out), _ptr(status), _stream()),
+           "cats_accept_path_typical")
+
+
 def cats_accept_path(parent, tokens, argmax, T, path, path_len, out_tokens, n_out, status):
     _check(lib.cats_accept_path(_ptr(parent), _ptr(tokens), _ptr(argmax), T, _ptr(path), _ptr(path_len), _ptr(out_tokens),
                                 _ptr(n_out), _ptr(status), _stream()), "cats_accept_path")
@@ -260,7 +284,8 @@ class VerifyForward:
     every output plus the workspace, all allocated once here (the library itself allocates nothing)."""
 
     def __init__(self, shape, model: dict, kcache, vcache, T: int, prefix_len: int, want_logits=True, compact=True,
-                 hidden_in=None):
+                 hidden_in=None, typical=None):
+        """typical: None for greedy acceptance, else (inv_temperature, log_eps, log_delta) as float32 values."""
         dev = kcache.device
         self.shape = shape
         self.T, self.prefix_len = T, prefix_len
@@ -298,6 +323,12 @@ class VerifyForward:
         a.d_logits, a.d_argmax, a.d_path = _ptr(self.logits), _ptr(self.argmax), _ptr(self.path)
         a.d_out_tokens, a.d_scalars = _ptr(self.out_tokens), _ptr(self.scalars)
         a.d_ws, a.ws_bytes, a.d_status = _ptr(self.ws), self.ws.numel(), _ptr(self.status)
+        self.typical = None
+        if typical is not None:
+            self.typical = torch.zeros((3, T), dtype=torch.float32, device=dev)     # lse, entropy, candidate logits
+            a.accept_mode = ACCEPT_TYPICAL
+            a.inv_temperature, a.log_eps, a.log_delta = float(typical[0]), float(typical[1]), float(typical[2])
+            a.d_typical = _ptr(self.typical)
         self.args = a
 
     def set_prefix_len(self, prefix_len: int):

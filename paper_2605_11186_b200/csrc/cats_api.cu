@@ -28,6 +28,7 @@ struct Workspace {
     float *attn_o, *attn_ml;
     float* pmax;
     int32_t* pidx;
+    float *psum, *ps1;          // per-tile softmax statistics of the LM head (typical acceptance)
     float* fix_part;
     int* fix_flags;
     float* scratch;             // [T][hidden] fp32
@@ -58,6 +59,8 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     int vt = (c->vocab + 127) / 128;
     w.pmax = (float*)take((size_t)vt * 128 * 4);
     w.pidx = (int32_t*)take((size_t)vt * 128 * 4);
+    w.psum = (float*)take((size_t)vt * 128 * 4);
+    w.ps1 = (float*)take((size_t)vt * 128 * 4);
     w.fix_part = (float*)take((size_t)kGemmCtas * tpad * 128 * 4);
     w.fix_flags = (int*)take((size_t)kGemmCtas * sizeof(int));
     w.scratch = (float*)take((size_t)T * c->hidden * 4);
@@ -147,8 +150,16 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     return pieces_d;
 }
 
+// Typical acceptance: what the LM head must leave behind besides the argmax.
+struct TypicalOut {
+    const int32_t *parent, *tokens;   // [T] the tree
+    float inv_temperature;
+    float *lse, *entropy, *cand;      // [T] each
+};
+
 int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm, float* resid, const float* copy_from,
-              int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st) {
+              int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st,
+              const TypicalOut* ty = nullptr) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
                              nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
@@ -156,8 +167,16 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.logits = logits; g.pmax = ws.pmax; g.pidx = ws.pidx; g.d_status = d_status;
+    if (ty) {
+        g.psum = ws.psum; g.ps1 = ws.ps1; g.inv_temperature = ty->inv_temperature;
+        g.tree_parent = ty->parent; g.tree_tokens = ty->tokens; g.cand = ty->cand;
+    }
     CATS_CUDA(launch_gemm(g, st));
-    CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, st));
+    if (ty)
+        CATS_CUDA(launch_head_reduce(ws.pmax, ws.pidx, ws.psum, ws.ps1, (V + 127) / 128, 128, T, ty->inv_temperature, amax,
+                                     ty->lse, ty->entropy, st));
+    else
+        CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, st));
     return CATS_OK;
 }
 
@@ -358,6 +377,44 @@ int cats_lm_head_argmax(const cats_model_cfg* cfg, const void* d_final_norm, con
     return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, 0, d_logits, d_argmax, ws, d_status, (cudaStream_t)stream);
 }
 
+int cats_lm_head_typical(const cats_model_cfg* cfg, const void* d_final_norm, const void* d_w_lm, const float* d_resid,
+                         const int32_t* d_parent, const int32_t* d_tokens, int32_t T, float inv_temperature, float* d_logits,
+                         int32_t* d_argmax, float* d_lse, float* d_entropy, float* d_cand_logit, void* d_ws, size_t ws_bytes,
+                         int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    int rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!d_final_norm || !d_w_lm || !d_resid || !d_parent || !d_tokens || !d_argmax || !d_lse || !d_entropy || !d_cand_logit ||
+        !d_ws || !d_status)
+        return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE || cfg->vocab < 1 || !(inv_temperature > 0.f) || !(inv_temperature < 1e6f)) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(d_resid, 16) || misaligned(d_w_lm, 16) || misaligned(d_final_norm, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    CATS_CUDA(cudaMemsetAsync(d_cand_logit, 0, (size_t)T * sizeof(float), st));
+    g_call_boundary = true;   // the memset is not a kernel: the first kernel still takes full stream ordering
+    TypicalOut ty = {d_parent, d_tokens, inv_temperature, d_lse, d_entropy, d_cand_logit};
+    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, 0, d_logits, d_argmax, ws, d_status, st, &ty);
+}
+
+int cats_accept_path_typical(const int32_t* d_parent, const int32_t* d_tokens, const int32_t* d_argmax, const float* d_cand_logit,
+                             const float* d_lse, const float* d_entropy, int32_t T, float inv_temperature, float log_eps,
+                             float log_delta, int32_t* d_path, int32_t* d_path_len, int32_t* d_out_tokens, int32_t* d_n_out,
+                             int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    g_call_boundary = true;
+    if (!d_parent || !d_tokens || !d_argmax || !d_cand_logit || !d_lse || !d_entropy || !d_path || !d_path_len || !d_out_tokens ||
+        !d_n_out || !d_status)
+        return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE || !(inv_temperature > 0.f)) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_walk_typical(d_parent, d_tokens, d_argmax, d_cand_logit, d_lse, d_entropy, T, inv_temperature, log_eps,
+                                  log_delta, d_path, d_path_len, d_out_tokens, d_n_out, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
 int cats_accept_path(const int32_t* d_parent, const int32_t* d_tokens, const int32_t* d_argmax, int32_t T, int32_t* d_path,
                      int32_t* d_path_len, int32_t* d_out_tokens, int32_t* d_n_out, int32_t* d_status, void* stream) {
     g_launch_count = 0;
@@ -396,6 +453,9 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     rc = check_tree_args(a->T, a->prefix_len);
     if (rc) return rc;
     if (a->prefix_len + a->T > c->max_seq || c->n_layers < 0 || c->vocab < 1) return CATS_ERR_INVALID_ARG;
+    if (a->accept_mode != CATS_ACCEPT_GREEDY && a->accept_mode != CATS_ACCEPT_TYPICAL) return CATS_ERR_INVALID_ARG;
+    const bool typical = a->accept_mode == CATS_ACCEPT_TYPICAL;
+    if (typical && (!a->d_typical || !(a->inv_temperature > 0.f) || !(a->inv_temperature < 1e6f))) return CATS_ERR_INVALID_ARG;
     if (misaligned(a->d_ws, 1024)) return CATS_ERR_WORKSPACE;
     if (misaligned(a->d_resid, 16) || misaligned(a->d_kcache, 16) || misaligned(a->d_vcache, 16)) return CATS_ERR_INVALID_ARG;
     Workspace ws = carve(c, a->T, a->d_ws);
@@ -404,6 +464,7 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     const int T = a->T, P = a->prefix_len;
     const size_t lstride = (size_t)c->max_seq * c->n_heads * c->head_dim;
 
+    if (typical) CATS_CUDA(cudaMemsetAsync(a->d_typical + 2 * T, 0, (size_t)T * sizeof(float), st));   // candidate logits
     CATS_CUDA(launch_mask_pos(d_parent, T, P, a->d_mask, a->d_pos, a->d_depth, a->d_status, st));
     const float* copy_from = a->d_hidden_in;
     if (!copy_from) CATS_CUDA(launch_embed(a->d_embed, d_tokens, T, c->hidden, c->vocab, a->d_resid, a->d_status, st));
@@ -418,10 +479,16 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
                              last, a->d_status, st);
         if (pending < 0) return pending;
     }
+    TypicalOut ty = {d_parent, d_tokens, a->inv_temperature, a->d_typical, a->d_typical ? a->d_typical + T : nullptr,
+                     a->d_typical ? a->d_typical + 2 * T : nullptr};
     rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T, pending, a->d_logits,
-                   a->d_argmax, ws, a->d_status, st);
+                   a->d_argmax, ws, a->d_status, st, typical ? &ty : nullptr);
     if (rc) return rc;
-    CATS_CUDA(launch_walk(d_parent, d_tokens, a->d_argmax, T, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
+    if (typical)
+        CATS_CUDA(launch_walk_typical(d_parent, d_tokens, a->d_argmax, ty.cand, ty.lse, ty.entropy, T, a->inv_temperature,
+                                      a->log_eps, a->log_delta, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
+    else
+        CATS_CUDA(launch_walk(d_parent, d_tokens, a->d_argmax, T, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
     if (a->compact)
         CATS_CUDA(launch_compact(a->d_kcache, a->d_vcache, c->n_layers, (long long)lstride, (long long)c->n_heads * c->head_dim, P,
                                  a->d_path, a->d_scalars + 0, a->d_scalars + 2, nullptr, nullptr, a->d_status, st));

@@ -56,6 +56,10 @@ struct GemmDev {
     float* logits;
     float* pmax;
     int32_t* pidx;
+    float *psum, *ps1;            // EPI_LMHEAD, optional: per-tile softmax statistics [n_tiles][128]
+    float inv_temp_log2e;         //   log2(e) / temperature
+    const int32_t *tree_parent, *tree_tokens;   //   [T]
+    float* cand;                  //   [T]: logit of every node's own token at its parent
     int32_t* d_status;
     const uint8_t* warm_ptr;     // next projection's packed weights: this CTA's first chunks of it
     int warm_chunks;             // 16 KB chunks to pull through a landing buffer (warms L2)
@@ -451,6 +455,36 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                                 p.pmax[(size_t)tile * 128 + c0 + nl] = best;
                                 p.pidx[(size_t)tile * 128 + c0 + nl] = bi;
                             }
+                            if (p.psum != nullptr) {
+                                // softmax statistics of this vocabulary tile at the given temperature, relative to the
+                                // tile's own maximum: Z = sum e, S1 = sum e * (logit - max), e = exp((logit - max) / t)
+                                float z = 0.f, s1 = 0.f;
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    int ff = lane + 32 * i;
+                                    if (row0 + ff < p.n_out) {
+                                        float d = acc_s[nl * 128 + ff] - best;
+                                        float e = exp2f(d * p.inv_temp_log2e);
+                                        z += e;
+                                        s1 = fmaf(e, d, s1);
+                                    }
+                                }
+#pragma unroll
+                                for (int o = 16; o > 0; o >>= 1) {
+                                    z += __shfl_xor_sync(0xffffffffu, z, o);
+                                    s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+                                }
+                                if (lane == 0) {
+                                    p.psum[(size_t)tile * 128 + c0 + nl] = z;
+                                    p.ps1[(size_t)tile * 128 + c0 + nl] = s1;
+                                }
+                            }
+                        }
+                        if (p.cand != nullptr && et > 0 && et < p.T) {
+                            // logit of tree node et's own token under its parent's distribution, if this tile holds it
+                            const int pa = __ldg(p.tree_parent + et), tk = __ldg(p.tree_tokens + et);
+                            if (pa >= c0 && pa < c0 + n_hi && tk >= row0 && tk < row0 + 128 && tk < p.n_out)
+                                p.cand[et] = acc_s[(pa - c0) * 128 + (tk - row0)];
                         }
                     }
                     epi_barrier();
@@ -623,6 +657,12 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.logits = p.logits;
     d.pmax = p.pmax;
     d.pidx = p.pidx;
+    d.psum = p.psum;
+    d.ps1 = p.ps1;
+    d.inv_temp_log2e = p.inv_temperature * 1.4426950408889634f;
+    d.tree_parent = p.tree_parent;
+    d.tree_tokens = p.tree_tokens;
+    d.cand = p.cand;
     d.d_status = p.d_status;
     d.warm_ptr = nullptr;
     d.warm_chunks = 0;

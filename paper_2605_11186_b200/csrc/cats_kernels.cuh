@@ -45,6 +45,15 @@ cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* pa
 cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st);
+// The same reduction plus the merge of the per-tile softmax statistics: lse[n] = log sum_v exp(logit/t),
+// entropy[n] = H(softmax(logit/t)).
+cudaError_t launch_head_reduce(const float* pmax, const int32_t* pidx, const float* psum, const float* ps1, int n_tiles,
+                               int t_stride, int T, float inv_temperature, int32_t* amax, float* lse, float* entropy,
+                               cudaStream_t st);
+cudaError_t launch_walk_typical(const int32_t* parent, const int32_t* tokens, const int32_t* amax, const float* cand,
+                                const float* lse, const float* entropy, int T, float inv_temperature, float log_eps,
+                                float log_delta, int32_t* path, int32_t* path_len, int32_t* out_tokens, int32_t* n_out,
+                                cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
                         int32_t* path_len, int32_t* out_tokens, int32_t* n_out, cudaStream_t st);
 cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_stride, long long row_elems, int prefix_len,
@@ -89,6 +98,12 @@ struct GemmProblem {
     float* logits;         // EPI_LMHEAD: [T][n_out] fp32 or null
     float* pmax;           //   [n_tiles][128]
     int32_t* pidx;
+    float* psum;           //   optional (typical acceptance): per-tile sum of exp((logit - tile max) / t) ...
+    float* ps1;            //   ... and sum of exp(..) * (logit - tile max), [n_tiles][128] each
+    float inv_temperature;
+    const int32_t* tree_parent;   //   [T] parent of every tree node
+    const int32_t* tree_tokens;   //   [T] token of every tree node
+    float* cand;           //   [T] out: logits[parent[i]][tokens[i]]
     int32_t* d_status;
     const GemmProblem* warm_next;   // the projection that follows (only W[0], K, n_out, n_mats, epi are read), or null
 };

@@ -200,6 +200,60 @@ __global__ void __launch_bounds__(128) k_argmax_reduce(const float* __restrict__
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same reduction with the softmax statistics typical acceptance needs.  Tile k of node t carries
+// its maximum m_k, Z_k = sum exp((l - m_k)/t) and S_k = sum exp((l - m_k)/t) (l - m_k).  With
+// M = max_k m_k and w_k = exp((m_k - M)/t):
+//   Z = sum_k w_k Z_k,   S = sum_k w_k (S_k + (m_k - M) Z_k)          (= sum_v e_v (l_v - M))
+//   lse = M/t + log Z,   entropy = log Z - S / (t Z).
+// Lanes take tiles in strides of 32 and the partial sums meet in a fixed shuffle order, so the
+// result does not depend on timing.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_head_reduce(const float* __restrict__ pmax, const int32_t* __restrict__ pidx,
+                                                     const float* __restrict__ psum, const float* __restrict__ ps1,
+                                                     int n_tiles, int t_stride, int T, float inv_t,
+                                                     int32_t* __restrict__ amax, float* __restrict__ lse,
+                                                     float* __restrict__ entropy) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int t = blockIdx.x * 4 + (threadIdx.x >> 5);
+    int lane = threadIdx.x & 31;
+    if (t >= T) return;
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int k = lane; k < n_tiles; k += 32) {
+        float v = pmax[(size_t)k * t_stride + t];
+        int ix = pidx[(size_t)k * t_stride + t];
+        if (v > best || (v == best && ix < bi)) { best = v; bi = ix; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    const float M = best;
+    float Z = 0.f, S = 0.f;
+    for (int k = lane; k < n_tiles; k += 32) {
+        float d = pmax[(size_t)k * t_stride + t] - M;
+        float w = exp2f(d * inv_t * 1.4426950408889634f);
+        float zk = psum[(size_t)k * t_stride + t];
+        Z = fmaf(w, zk, Z);
+        S = fmaf(w, fmaf(d, zk, ps1[(size_t)k * t_stride + t]), S);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Z += __shfl_xor_sync(0xffffffffu, Z, o);
+        S += __shfl_xor_sync(0xffffffffu, S, o);
+    }
+    if (lane == 0) {
+        amax[t] = bi;
+        float lz = logf(Z);
+        lse[t] = fmaf(M, inv_t, lz);
+        entropy[t] = lz - S * inv_t / Z;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Greedy longest-accepted-path walk, one warp.  At node cur the target wants token argmax[cur];
 // each lane tests four nodes, a ballot plus find-first-set gives the lowest matching child.
 // ---------------------------------------------------------------------------------------------
@@ -229,6 +283,64 @@ __global__ void __launch_bounds__(32) k_walk(const int32_t* __restrict__ parent,
         }
         if (next < 0) break;
         if (lane == 0) { out_tokens[no] = want; path[len] = next; }
+        ++no; ++len;
+        cur = next;
+    }
+    if (lane == 0) {
+        out_tokens[no] = amax[cur];
+        *path_len = len;
+        *n_out = no + 1;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The walk under typical acceptance (Algorithm 1's loop with Acc = the relaxed criterion): child
+// i of the current node is acceptable iff p_parent(token_i) > min(eps, delta * exp(-H_parent)),
+// taken in the log domain with one fused multiply-add and one subtraction, both fp32 round to
+// nearest:  fma(cand[i], 1/t, -lse[parent]) > min(log eps, log delta - entropy[parent]).
+// The first acceptable child in node order is taken; the bonus token is the argmax at the last
+// accepted node.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) k_walk_typical(const int32_t* __restrict__ parent, const int32_t* __restrict__ tokens,
+                                                     const int32_t* __restrict__ amax, const float* __restrict__ cand,
+                                                     const float* __restrict__ lse, const float* __restrict__ entropy, int T,
+                                                     float inv_t, float log_eps, float log_delta, int32_t* __restrict__ path,
+                                                     int32_t* __restrict__ path_len, int32_t* __restrict__ out_tokens,
+                                                     int32_t* __restrict__ n_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int lane = threadIdx.x;
+    int par[4], tok[4];
+    bool ok[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        int j = q * 32 + lane;
+        par[q] = j < T ? parent[j] : -2;
+        tok[q] = j < T ? tokens[j] : -1;
+        ok[q] = false;
+        if (j > 0 && j < T && par[q] >= 0 && par[q] < j) {
+            float logp = __fmaf_rn(cand[j], inv_t, -lse[par[q]]);
+            float thr = fminf(log_eps, __fsub_rn(log_delta, entropy[par[q]]));
+            ok[q] = logp > thr;
+        }
+    }
+    int cur = 0, len = 1, no = 0;
+    if (lane == 0) path[0] = 0;
+    for (int step = 0; step < T; ++step) {
+        int next = -1;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            unsigned b = __ballot_sync(0xffffffffu, par[q] == cur && ok[q]);
+            if (next < 0 && b) next = q * 32 + __ffs(b) - 1;
+        }
+        if (next < 0) break;
+        int t = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int v = __shfl_sync(0xffffffffu, tok[q], next & 31);
+            if (q == (next >> 5)) t = v;
+        }
+        if (lane == 0) { out_tokens[no] = t; path[len] = next; }
         ++no; ++len;
         cur = next;
     }
@@ -321,6 +433,21 @@ cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clam
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
                                  cudaStream_t st) {
     return launch_pdl(k_argmax_reduce, dim3((T + 3) / 4), dim3(128), 0, st, pmax, pidx, n_tiles, t_stride, T, amax);
+}
+
+cudaError_t launch_head_reduce(const float* pmax, const int32_t* pidx, const float* psum, const float* ps1, int n_tiles,
+                               int t_stride, int T, float inv_temperature, int32_t* amax, float* lse, float* entropy,
+                               cudaStream_t st) {
+    return launch_pdl(k_head_reduce, dim3((T + 3) / 4), dim3(128), 0, st, pmax, pidx, psum, ps1, n_tiles, t_stride, T,
+                      inv_temperature, amax, lse, entropy);
+}
+
+cudaError_t launch_walk_typical(const int32_t* parent, const int32_t* tokens, const int32_t* amax, const float* cand,
+                                const float* lse, const float* entropy, int T, float inv_temperature, float log_eps,
+                                float log_delta, int32_t* path, int32_t* path_len, int32_t* out_tokens, int32_t* n_out,
+                                cudaStream_t st) {
+    return launch_pdl(k_walk_typical, dim3(1), dim3(32), 0, st, parent, tokens, amax, cand, lse, entropy, T, inv_temperature,
+                      log_eps, log_delta, path, path_len, out_tokens, n_out);
 }
 
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
