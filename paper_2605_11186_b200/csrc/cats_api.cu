@@ -99,7 +99,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -128,7 +128,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                                 nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st));
+                                 nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st, d_status));
 
     g = GemmProblem{};
     g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
@@ -162,7 +162,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               const TypicalOut* ty = nullptr) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st));
+                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -303,7 +303,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
+                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st, d_status));
     return CATS_OK;
 }
 
@@ -331,7 +331,7 @@ int cats_verify_layer_nodes(const cats_model_cfg* cfg, const cats_layer_weights*
                              false, d_status, st, ws.nodes, T);
     if (pending < 0) return pending;
     CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, m, cfg->hidden, cfg->rms_eps, nullptr,
-                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st));
+                             nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st, d_status));
     return CATS_OK;
 }
 

@@ -17,6 +17,7 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
+CATS_TRACE_DEFINE(attn)
 
 constexpr int kAttnThreads = 256;
 constexpr int kKvBlock = 64;
@@ -123,8 +124,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     pdl_launch_dependents();
     // the first block can be requested before the previous kernel has finished if it lies in the prefix
     const bool early = (c_begin + p.blk <= p.P);
+    if (threadIdx.x == 0) TR(2, 0);
     if (early) load_kv(0, 0);
     pdl_wait();
+    if (threadIdx.x == 0) TR(2, 1);
     for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
         int r = e / NCH, ch = e % NCH;
         uint32_t off = tile_off<HD>(r, ch);
@@ -322,6 +325,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         }
     }
     if (csize > 1) cluster_sync_all();   // nobody leaves while a peer may still read its shared memory
+    if (threadIdx.x == 0) TR(2, 4);
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).

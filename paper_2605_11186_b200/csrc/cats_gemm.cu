@@ -30,9 +30,10 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
+CATS_TRACE_DEFINE(gemm)
 
 constexpr int kGemmThreads = 224;
-constexpr int kCtrlBytes = 1024;
+constexpr int kCtrlBytes = 512;
 constexpr int kMaxStages = 14;
 constexpr int kWChunk = 16384;        // 128 rows x 64 bf16
 constexpr int kUnitKb = 2;            // K blocks per pipeline stage (one bulk copy of W, one of X)
@@ -96,14 +97,25 @@ __device__ __forceinline__ void st_release(int* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(smem);
-    uint8_t* stages = smem + kCtrlBytes;
+// Register and shared-memory footprint are chosen so that one CTA of the RMSNorm kernel (256 threads, <= 80 registers,
+// no dynamic shared memory) fits on the SM beside a resident CTA of this kernel: 224 x 192 + 256 x 80 registers <= 64 K,
+// and 224.5 KB + 2 x 1 KB reserved + the norm's static 32 B <= 228 KB.  With programmatic dependent launch the CTAs of
+// the projection that FOLLOWS a norm then take the SMs as soon as the previous projection leaves them and fill their
+// weight ring while the norm is still running.
+#ifndef CATS_GEMM_MAXREG
+#define CATS_GEMM_MAXREG 192
+#endif
+__global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* stages = smem_raw;                                                             // 1024-byte aligned (checked)
     float* acc_s = reinterpret_cast<float*>(stages + (size_t)p.n_stages * p.stage_bytes);   // [32][128] fp32
     uint8_t* landing = reinterpret_cast<uint8_t*>(acc_s) + (size_t)kStagingCols * 128 * 4;  // 16 KB, contents never read
+    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(landing + kWChunk);
     volatile int* abort_flag = &ctrl->abort_flag;
+    if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled operand tiles need this alignment; never seen violated
+        if (threadIdx.x == 0) report(p.d_status, CATS_ERR_UNSUPPORTED);
+        return;
+    }
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -142,6 +154,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     __syncthreads();
     tc_fence_after_sync();
     pdl_launch_dependents();
+    if (threadIdx.x == 0) TR(10 + p.epi, 0);
     const uint32_t tmem_acc = ctrl->tmem_base;
 
     if (warp == 0 || warp == 6) {
@@ -169,7 +182,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                     bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &ctrl->full[s], pol);
                 }
             };
-            if (!is_w) pdl_wait();     // activations come from the previous kernel; weights never do
+            if (!is_w) { pdl_wait(); TR(10 + p.epi, 1); }    // activations come from the previous kernel; weights never do
             int issued = 0;
             for (int i = 0; i < n_units; ++i) {
                 if (i >= S && !mbar_wait(&ctrl->empty[i % S], ((i / S) - 1) & 1, abort_flag)) break;
@@ -218,6 +231,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                     int s = i % S;
                     ok = mbar_wait(&ctrl->full[s], (i / S) & 1, abort_flag);
                     if (!ok) break;
+                    if (i == 0) TR(10 + p.epi, 2);
+                    if (i == S) TR(10 + p.epi, 5);
                     tc_fence_after_sync();
                     const int kb = (int)(u % p.n_ku) * kUnitKb;
                     const int nk = min(kUnitKb, p.n_kb - kb);
@@ -234,6 +249,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
                 }
                 umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
             }
+            TR(10 + p.epi, 3);
         }
     } else if (warp < 6) {
         // ---------------- epilogue warps ----------------
@@ -498,6 +514,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) k_gemm_sk(const GemmDev p) {
     }
     tc_fence_before_sync();
     __syncthreads();
+    if (threadIdx.x == 0) TR(10 + p.epi, 4);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -608,7 +625,7 @@ GemmPlan gemm_plan(const GemmProblem& p) {
 
 cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     static bool attr_set = false;
-    const int kMaxSmem = 227 * 1024;
+    const int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gemm_sk, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
@@ -631,12 +648,12 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
     size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
-    int stages = (int)((kMaxSmem - 1024 - kCtrlBytes - staging) / d.stage_bytes);
+    int stages = (int)((kMaxSmem - kCtrlBytes - staging) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages > pl.units_per_cta) stages = pl.units_per_cta;
     if (stages < 1) stages = 1;
     d.n_stages = stages;
-    size_t smem = 1024 + kCtrlBytes + (size_t)stages * d.stage_bytes + staging;
+    size_t smem = (size_t)stages * d.stage_bytes + staging + kCtrlBytes;
     uint32_t cols = 32;
     while ((int)cols < 2 * d.n_pad) cols <<= 1;
     d.tmem_cols = cols;

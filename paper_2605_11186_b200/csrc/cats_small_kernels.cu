@@ -4,6 +4,7 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
+CATS_TRACE_DEFINE(small)
 
 // ---------------------------------------------------------------------------------------------
 // Ancestor mask, depth, position ids.  One CTA of 128 threads; thread i walks from node i to the
@@ -408,6 +409,169 @@ __global__ void __launch_bounds__(256) k_compact(uint16_t* __restrict__ kc, uint
 // ---------------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------------
+// The same operation with the row held in registers and no dynamic shared memory, one row per CLUSTER of cs CTAs
+// (cs = 1, 2 or 4): CTA `rank` owns columns [rank, rank + 1) * H / cs, NC float4 per thread, so that all loads of a
+// thread are in flight at once; the sums of squares meet through distributed shared memory, added in rank order.
+// Footprint: a CTA of this kernel fits on an SM beside a resident CTA of the projection kernel, so the projection that
+// follows can already be resident and stream its first weight stages while the norm runs.  Thread pairs (even, odd
+// lane) hold the two halves of one 16-byte group of the packed output.
+template <int NC>
+__global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, const float* __restrict__ copy_from,
+                                                     const float* __restrict__ part, int n_part, size_t part_stride,
+                                                     const uint16_t* __restrict__ gain, int H, float eps,
+                                                     uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
+                                                     const int32_t* __restrict__ nodes, float2* __restrict__ rope, int hd,
+                                                     float rope_base, int* zero_flags, int n_flags, int cs,
+                                                     int32_t* d_status) {
+    __shared__ float red[8];
+    __shared__ __align__(8) uint64_t xbar;     // completes when the partial sums of squares of all cs CTAs have landed
+    __shared__ float slots[4];                 // slots[r]: the partial sum of the cluster's CTA r
+    __shared__ int wait_expired;
+    pdl_launch_dependents();
+    const int t = blockIdx.x / cs, rank = blockIdx.x - t * cs;
+    const int cols_cta = H / 4 / cs;          // float4 columns of this CTA
+    const int col0 = rank * cols_cta;
+    if (threadIdx.x == 0) TR(1, 0);
+    // everything that does not depend on the previous kernel: the exchange barrier and the gains
+    if (cs > 1) {
+        if (threadIdx.x == 0) {
+            wait_expired = 0;
+            mbar_init(&xbar, 1);
+            mbar_fence_init();
+            mbar_expect_tx(&xbar, 4u * (uint32_t)cs);
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
+    uint2 g[NC];
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        const int cl = threadIdx.x + 256 * j;
+        g[j] = make_uint2(0u, 0u);
+        if (xn != nullptr && cl < cols_cta) g[j] = __ldg(reinterpret_cast<const uint2*>(gain) + col0 + cl);
+    }
+    pdl_wait();
+    if (threadIdx.x == 0) TR(1, 1);
+    if (zero_flags != nullptr && blockIdx.x == 0)
+        for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
+    if (rope != nullptr && rank == cs - 1) {
+        int half = hd / 2;
+        int p = pos[nodes != nullptr ? nodes[t] : t];
+        for (int i = threadIdx.x; i < half; i += blockDim.x) {
+            double inv_freq = pow((double)rope_base, -2.0 * (double)i / (double)hd);
+            double s, c;
+            sincos((double)p * inv_freq, &s, &c);
+            rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
+        }
+    }
+    const float4* r4 = reinterpret_cast<const float4*>((copy_from ? copy_from : resid) + (size_t)t * H);
+    float4 a[NC];
+    float4 pv[NC][kMaxPartSlots / 2];
+    // all loads first: the row, then the partial sums of the previous projection (slots 0..3 of every column)
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        const int cl = threadIdx.x + 256 * j;
+        a[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (cl < cols_cta) a[j] = r4[col0 + cl];
+    }
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        const int cl = threadIdx.x + 256 * j;
+#pragma unroll
+        for (int s = 0; s < kMaxPartSlots / 2; ++s)
+            if (s < n_part && cl < cols_cta)
+                pv[j][s] = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + col0 + cl);
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        const int cl = threadIdx.x + 256 * j;
+        if (cl >= cols_cta) continue;
+        float4 v = a[j];
+#pragma unroll
+        for (int s = 0; s < kMaxPartSlots / 2; ++s)
+            if (s < n_part) { v.x += pv[j][s].x; v.y += pv[j][s].y; v.z += pv[j][s].z; v.w += pv[j][s].w; }
+        for (int s = kMaxPartSlots / 2; s < n_part; ++s) {     // more than four slots: rare (small matrices), in order
+            const float4 q = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + col0 + cl);
+            v.x += q.x; v.y += q.y; v.z += q.z; v.w += q.w;
+        }
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        a[j] = v;
+    }
+    if (threadIdx.x == 0) TR(1, 2);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    if (cs > 1) {
+        // every CTA sends its partial sum to slot [rank] of every CTA of the cluster (itself included); the store
+        // signals the receiver's barrier, so one one-way trip through distributed shared memory is all that is waited for
+        if (threadIdx.x == 0) {
+            for (int r = 0; r < cs; ++r) {
+                uint32_t rslot, rbar;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rslot) : "r"(smem_u32(&slots[rank])), "r"(r));
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_u32(&xbar)), "r"(r));
+                asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                             ::"r"(rslot), "r"(__float_as_uint(tot)), "r"(rbar) : "memory");
+            }
+        }
+        if (!mbar_wait(&xbar, 0, &wait_expired)) {
+            if (threadIdx.x == 0) report(d_status, CATS_ERR_TIMEOUT);
+        }
+        tot = 0.f;
+        for (int r = 0; r < cs; ++r) tot += slots[r];    // rank order: every CTA of the cluster gets the same bits
+    }
+    if (threadIdx.x == 0) TR(1, 3);
+    const float rs = rsqrtf(tot / (float)H + eps);
+    const bool write_resid = n_part > 0 || copy_from != nullptr;
+    float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
+#pragma unroll
+    for (int j = 0; j < NC; ++j) {
+        const int cl = threadIdx.x + 256 * j;
+        if (cl >= cols_cta) continue;
+        const int c = col0 + cl;
+        const float4 x = a[j];
+        if (write_resid) out4[c] = x;
+        if (xn != nullptr) {
+            uint2 o;
+            o.x = pack_bf16x2(__uint_as_float(g[j].x << 16) * (x.x * rs), __uint_as_float(g[j].x & 0xFFFF0000u) * (x.y * rs));
+            o.y = pack_bf16x2(__uint_as_float(g[j].y << 16) * (x.z * rs), __uint_as_float(g[j].y & 0xFFFF0000u) * (x.w * rs));
+            *reinterpret_cast<uint2*>(xn + packed_act_offset(t, c >> 1, n_pad) + (size_t)(c & 1) * 8) = o;
+        }
+    }
+    if (threadIdx.x == 0) TR(1, 4);
+}
+
+template <typename Kern, typename... Args>
+static cudaError_t launch_cluster_pdl(Kern kernel, dim3 grid, dim3 block, int cs, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (cs > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cs;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (!g_call_boundary) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    g_call_boundary = false;
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    ++g_launch_count;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 cudaError_t launch_mask_pos(const int32_t* parent, int T, int prefix_len, uint64_t* mask, int32_t* pos, int32_t* depth,
                             int32_t* d_status, cudaStream_t st) {
     return launch_pdl(k_mask_pos, dim3(1), dim3(kMaxTree), 0, st, parent, T, prefix_len, mask, pos, depth, d_status);
@@ -420,9 +584,31 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
-                           float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st) {
+                           float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st,
+                           int32_t* d_status) {
+    const int n_pad = (T + 15) / 16 * 16;
+#define CATS_NORM_REG(NC)                                                                                                   \
+    return launch_cluster_pdl(k_rmsnorm_reg<NC>, dim3(T * cs), dim3(256), cs, st, resid, copy_from, part, n_part, part_stride, \
+                              (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, n_pad, pos, nodes, rope, hd, rope_base,    \
+                              zero_flags, n_flags, cs, d_status)
+#ifndef CATS_NORM_SMEM
+    {
+        // as many CTAs per row as keep the grid within one wave and leave every CTA at least 256 columns
+        const int n_cols = H / 4;
+        int cs = 1;
+        for (int c = 4; c >= 2; c >>= 1)
+            if (T * c <= 148 && n_cols % c == 0 && n_cols / c >= 256) { cs = c; break; }
+        const int nc = (n_cols / cs + 255) / 256;
+        if (nc <= 1) CATS_NORM_REG(1);
+        if (nc <= 2) CATS_NORM_REG(2);
+        if (nc <= 4) CATS_NORM_REG(4);
+        if (nc <= 5) CATS_NORM_REG(5);
+        if (nc <= 8) CATS_NORM_REG(8);
+    }
+#endif
+#undef CATS_NORM_REG
     return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
-                      part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, (T + 15) / 16 * 16, pos, nodes, rope,
+                      part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, n_pad, pos, nodes, rope,
                       hd, rope_base, zero_flags, n_flags);
 }
 
