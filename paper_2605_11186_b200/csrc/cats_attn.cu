@@ -52,6 +52,8 @@ struct AttnDev {
     const uint64_t* mask;
     const int32_t* nodes;   // null, or the tree node of each query row (selects its mask row)
     int Tk;                 // tree rows in the cache after the prefix
+    int rpr;                // query rows each CTA of a cluster merges (contiguous block)
+    int32_t* d_status;
     int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split, blk, kv_area;   // blk: cache rows per pipeline block (multiple of 16*kvg); kv_area: bytes of the K/V buffers
     long long kv_stride;
     float scale_log2;
@@ -90,6 +92,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     uint8_t* q_s = sm;                                           // [n_mt*16][HD]
     uint8_t* kv_s = q_s + (size_t)p.n_mt * 16 * ROWB;            // 2 buffers x (K [64][HD], V [64][HD])
     uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + p.kv_area);   // [n_mt*16][2]
+    float* recv = reinterpret_cast<float*>(mask_s + (size_t)p.n_mt * 16 * 2);   // [csize][kvg][rpr][HD + 4]: partials pushed by the cluster
+    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (size_t)p.csize * p.kvg * p.rpr * (HD + 4));
+    volatile int* wait_expired = reinterpret_cast<volatile int*>(rbar + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, h = blockIdx.y;
@@ -126,6 +131,18 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     const bool early = (c_begin + p.blk <= p.P);
     if (threadIdx.x == 0) TR(2, 0);
     if (early) load_kv(0, 0);
+    if (p.csize > 1) {
+        // the barrier the cluster's pushed partials complete on; visible to the peers before anybody can send
+        if (threadIdx.x == 0) {
+            const int rank_ = split % p.csize;
+            const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
+            *wait_expired = 0;
+            mbar_init(rbar, 1);
+            mbar_fence_init();
+            mbar_expect_tx(rbar, (uint32_t)(r1 - r0) * (HD + 4) * 4u * (uint32_t)(p.csize * p.kvg));
+        }
+        cluster_sync_all();
+    }
     pdl_wait();
     if (threadIdx.x == 0) TR(2, 1);
     for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
@@ -247,43 +264,74 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     }
 
     // ---- every warp deposits its partial (m, l, O); the cluster merges all partials of the head ----
+    // Record of one (partial, query row): HD floats of O, then m, l and two pad floats (a multiple of 16 bytes).
+    // The query rows are divided among the CTAs of the cluster in contiguous blocks of rpr rows; every CTA PUSHES, for
+    // every destination CTA, the slab of records that CTA will merge, with bulk copies through distributed shared
+    // memory that complete on the destination's mbarrier.  The merge then reads local shared memory only.
+    constexpr int REC = HD + 4;
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
     l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
     l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
     cp_async_wait<0>();                                  // a CTA without rows still has its Q copy in flight
     __syncthreads();
-    float* loc_o = reinterpret_cast<float*>(kv_s);      // [kvg][Tpad][HD], aliases the KV buffers
-    float* loc_ml = reinterpret_cast<float*>(q_s);      // [kvg][Tpad][2], aliases Q (no longer needed)
+    float* loc = reinterpret_cast<float*>(kv_s);        // [kvg][Tpad][REC], aliases the KV buffers
     if (active) {
-        float* wo = loc_o + ((size_t)g * Tpad) * HD;
+        float* wo = loc + ((size_t)g * Tpad) * REC;
 #pragma unroll
         for (int j = 0; j < NT; ++j) {
             int col = j * 8 + (lane & 3) * 2;
-            *reinterpret_cast<float2*>(wo + (size_t)row_a * HD + col) = make_float2(o[j][0], o[j][1]);
-            *reinterpret_cast<float2*>(wo + (size_t)row_b * HD + col) = make_float2(o[j][2], o[j][3]);
+            *reinterpret_cast<float2*>(wo + (size_t)row_a * REC + col) = make_float2(o[j][0], o[j][1]);
+            *reinterpret_cast<float2*>(wo + (size_t)row_b * REC + col) = make_float2(o[j][2], o[j][3]);
         }
         if ((lane & 3) == 0) {
-            float* wm = loc_ml + ((size_t)g * Tpad) * 2;
-            wm[row_a * 2] = m_run[0]; wm[row_a * 2 + 1] = l_run[0];
-            wm[row_b * 2] = m_run[1]; wm[row_b * 2 + 1] = l_run[1];
+            *reinterpret_cast<float2*>(wo + (size_t)row_a * REC + HD) = make_float2(m_run[0], l_run[0]);
+            *reinterpret_cast<float2*>(wo + (size_t)row_b * REC + HD) = make_float2(m_run[1], l_run[1]);
         }
     }
-    __syncthreads();
-    const int csize = p.csize;
+    const int csize = p.csize, rpr = p.rpr;
     const int rank = split % csize, outer = split / csize;
-    if (csize > 1) cluster_sync_all();
     const int n_parts = csize * p.kvg;                         // <= 32
-    const uint32_t ml_base = smem_u32(loc_ml), o_base = smem_u32(loc_o);
-    for (int row = rank + csize * warp; row < p.T; row += csize * 8) {
+    const float* src_parts = loc;                              // csize == 1: merge straight from the deposit
+    int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
+    if (csize > 1) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the deposit is read by bulk copies
+        __syncthreads();
+        // one thread per (destination, g) sends slab g of the rows that destination owns; a bulk copy occupies its
+        // issuing thread for about half a microsecond, so the senders are spread over the warps
+        const int pi = lane * 8 + warp;
+        if (lane < 4 && pi < n_parts) {
+            const int dest = pi / p.kvg, gg = pi - dest * p.kvg;
+            const int r0 = min(Tpad, dest * rpr), r1 = min(Tpad, r0 + rpr);
+            if (r1 > r0) {
+                const uint32_t bytes = (uint32_t)(r1 - r0) * REC * 4;
+                const uint32_t src = smem_u32(loc + ((size_t)gg * Tpad + r0) * REC);
+                const uint32_t dst_local = smem_u32(recv + ((size_t)(rank * p.kvg + gg) * rpr) * REC);
+                const uint32_t dst = cluster_map(dst_local, dest), bar = cluster_map(smem_u32(rbar), dest);
+                asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(dst), "r"(src), "r"(bytes), "r"(bar) : "memory");
+            }
+        }
+        row0 = min(Tpad, rank * rpr);
+        n_my = min(Tpad, row0 + rpr) - row0;
+        if (n_my > 0 && !mbar_wait(rbar, 0, wait_expired)) {
+            if (threadIdx.x == 0) report(p.d_status, CATS_ERR_TIMEOUT);
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // this CTA holds everything it needs
+        src_parts = recv;
+        part_stride = rpr * REC;
+    } else {
+        __syncthreads();
+    }
+    for (int rl = warp; rl < n_my; rl += 8) {
+        const int row = row0 + rl;
+        if (row >= p.T) break;
         float mp = -INFINITY, lp = 0.f;
-        uint32_t my_o = 0;
+        const float* my_rec = src_parts;
         if (lane < n_parts) {
-            const int c = lane / p.kvg, gg = lane - c * p.kvg;
-            const uint32_t off = (uint32_t)((gg * Tpad + row) * 2 * 4);
-            float2 ml = ld_cluster_f2(cluster_map(ml_base + off, c));
+            my_rec = src_parts + (size_t)lane * part_stride + (size_t)(csize > 1 ? rl : row) * REC;
+            const float2 ml = *reinterpret_cast<const float2*>(my_rec + HD);
             mp = ml.x; lp = ml.y;
-            my_o = cluster_map(o_base + (uint32_t)((gg * Tpad + row) * HD * 4), c);
         }
         float M = mp;
 #pragma unroll
@@ -295,18 +343,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         for (int ofs = 16; ofs > 0; ofs >>= 1) L += __shfl_xor_sync(0xffffffffu, L, ofs);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         const bool col_ok = lane < HD / 4;
-        for (int p0 = 0; p0 < n_parts; p0 += 8) {      // eight remote loads in flight at a time
-            float4 v[8];
-            float w[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int pp = (p0 + i) & 31;
-                w[i] = (p0 + i < n_parts) ? __shfl_sync(0xffffffffu, wp, pp) : 0.f;
-                const uint32_t oa = __shfl_sync(0xffffffffu, my_o, pp);
-                v[i] = (col_ok && w[i] != 0.f) ? ld_cluster_f4(oa + (uint32_t)lane * 16) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* base = src_parts + (size_t)(csize > 1 ? rl : row) * REC + lane * 4;
+        for (int pp = 0; pp < n_parts; ++pp) {                 // partials in a fixed order
+            const float w = __shfl_sync(0xffffffffu, wp, pp);
+            if (col_ok && w != 0.f) {
+                const float4 v = *reinterpret_cast<const float4*>(base + (size_t)pp * part_stride);
+                acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
             }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) { acc.x += v[i].x * w[i]; acc.y += v[i].y * w[i]; acc.z += v[i].z * w[i]; acc.w += v[i].w * w[i]; }
         }
         if (p.n_outer == 1) {
             if (col_ok) {
@@ -319,13 +362,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
                 *reinterpret_cast<uint2*>(ob + off) = pk;
             }
         } else {
-            const size_t base = ((size_t)h * p.n_outer + outer) * Tpad + row;
-            if (col_ok) *reinterpret_cast<float4*>(p.part_o + base * HD + lane * 4) = acc;
-            if (lane == 0) { p.part_ml[base * 2] = M; p.part_ml[base * 2 + 1] = L; }
+            const size_t gbase = ((size_t)h * p.n_outer + outer) * Tpad + row;
+            if (col_ok) *reinterpret_cast<float4*>(p.part_o + gbase * HD + lane * 4) = acc;
+            if (lane == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
-    if (csize > 1) cluster_sync_all();   // nobody leaves while a peer may still read its shared memory
-    if (threadIdx.x == 0) TR(2, 4);
+    // nobody leaves while a peer's copy may still be reading this CTA's deposit
+    if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
@@ -408,8 +451,8 @@ static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t sme
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -430,7 +473,11 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.out_npad = p.out_packed_npad;
     d.part_o = p.part_o; d.part_ml = p.part_ml;
     int tpad = d.n_mt * 16;
-    size_t merge = (size_t)d.kvg * tpad * p.hd * 4;                 // aliases the KV buffers
+    const int rec = p.hd + 4;
+    size_t merge = (size_t)d.kvg * tpad * rec * 4;                  // the deposit aliases the KV buffers
+    d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;     // rows per CTA of the cluster, even
+    d.d_status = p.d_status;
+    const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.kvg * d.rpr * rec * 4 + 16 : 16;
     // Block size of the KV pipeline: a CTA whose whole share fits two or three 64-row blocks takes it in one block
     // instead (one wait and one barrier round instead of three); long shares stream 64-row blocks.
     int blk = kKvBlock;
@@ -446,7 +493,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     if (qbytes < (size_t)d.kvg * tpad * 8) qbytes = (size_t)d.kvg * tpad * 8;
     if (kv < merge) kv = merge;
     d.kv_area = (int)kv;
-    size_t smem = qbytes + kv + (size_t)tpad * 16;
+    size_t smem = qbytes + kv + (size_t)tpad * 16 + recv;
     cudaError_t e;
     dim3 grid(p.cluster * p.n_splits, p.nh);
     if (p.hd == 128) e = launch_cluster(k_tree_attn<128>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
