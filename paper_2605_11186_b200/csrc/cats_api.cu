@@ -61,8 +61,8 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     w.pidx = (int32_t*)take((size_t)vt * 128 * 4);
     w.psum = (float*)take((size_t)vt * 128 * 4);
     w.ps1 = (float*)take((size_t)vt * 128 * 4);
-    w.fix_part = (float*)take((size_t)kGemmCtas * tpad * 128 * 4);
-    w.fix_flags = (int*)take((size_t)kGemmCtas * sizeof(int));
+    w.fix_part = (float*)take((size_t)kFixSlots * tpad * 128 * 4);
+    w.fix_flags = (int*)take((size_t)kFixSlots * sizeof(int));
     w.scratch = (float*)take((size_t)T * c->hidden * 4);
     w.nodes = (int32_t*)take((size_t)CATS_MAX_TREE * sizeof(int32_t));
     w.bytes = off;
@@ -99,7 +99,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st, d_status));
+                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -162,7 +162,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               const TypicalOut* ty = nullptr) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kGemmCtas, st, d_status));
+                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;

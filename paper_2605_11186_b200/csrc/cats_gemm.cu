@@ -42,11 +42,14 @@ constexpr int kStagingCols = 32;      // epilogue staging tile: 32 nodes x 128 f
 struct GemmDev {
     int epi, T, n_pad, n_out, n_kb, n_ku, n_tiles, tiles_per_mat, units_per_cta, n_stages, max_pieces, split_s;
     long long total_units;
+    int head_units;       // > 0: "owners + helpers" split (see gemm_plan): CTA t < n_tiles runs units [0, head_units) of tile t
+    int help_upc;         //   units per helper CTA in the space of the tiles' remaining units
+    int total_rem;        //   n_tiles * (n_ku - head_units)
     uint32_t x_chunk_bytes, stage_bytes, tmem_cols;
     const uint8_t* Wp;
     const uint8_t* Xp;
-    float* fix_part;      // [n_ctas][n_pad][128] fp32 partial tiles of split tiles
-    int* fix_flags;       // [n_ctas]
+    float* fix_part;      // [slots][n_pad][128] fp32 partial tiles of split tiles (slot = CTA, or 2 * tile + i with helpers)
+    int* fix_flags;       // [slots]
     float* part;
     size_t part_stride;
     uint16_t *q_out, *kcache, *vcache;
@@ -121,9 +124,28 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
     const int S = p.n_stages;
-    // split_s == 0: even contiguous shares of all (tile, K) units; split_s > 0: every tile cut into split_s aligned pieces
+    // The CTA's work is a range [u0, u1) of a unit space in which every tile owns vlen consecutive units, unit v of a
+    // tile being its K unit koff + v.
+    //   split_s == 0, head_units == 0: all (tile, K) units, even contiguous shares ("stream-K"); vlen = n_ku.
+    //   split_s > 0: every tile cut into split_s aligned pieces.
+    //   head_units > 0: CTA t < n_tiles owns tile t and runs its first head_units K units; the CTAs after them
+    //     ("helpers") share the remaining units of all tiles evenly and only contribute partial tiles.
     long long u0, u1;
-    if (p.split_s > 0) {
+    int vlen = p.n_ku, koff = 0;
+    bool helper = false;
+    if (p.head_units > 0) {
+        if (cta < p.n_tiles) {
+            vlen = p.head_units;
+            u0 = (long long)cta * vlen;
+            u1 = u0 + vlen;
+        } else {
+            helper = true;
+            vlen = p.n_ku - p.head_units;
+            koff = p.head_units;
+            u0 = min((long long)p.total_rem, (long long)(cta - p.n_tiles) * p.help_upc);
+            u1 = min((long long)p.total_rem, u0 + p.help_upc);
+        }
+    } else if (p.split_s > 0) {
         const long long t0 = (long long)(cta / p.split_s) * p.n_ku;
         u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
         u1 = min(t0 + p.n_ku, u0 + (long long)p.units_per_cta);
@@ -168,8 +190,8 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             auto issue = [&](int i) {
                 const int s = i % S;
                 const long long u = u0 + i;
-                const int tile = (int)(u / p.n_ku);
-                const int kb = (int)(u - (long long)tile * p.n_ku) * kUnitKb;
+                const int tile = (int)(u / vlen);
+                const int kb = (koff + (int)(u - (long long)tile * vlen)) * kUnitKb;
                 const int nk = min(kUnitKb, p.n_kb - kb);
                 uint8_t* stage = stages + (size_t)s * p.stage_bytes;
                 if (is_w) {
@@ -220,7 +242,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             int i = 0, seg = 0;
             bool ok = true;
             for (long long u = u0; u < u1 && ok; ++seg) {
-                const long long tile_end = (u / p.n_ku + 1) * p.n_ku;
+                const long long tile_end = (u / vlen + 1) * vlen;
                 const long long seg_end = min(u1, tile_end);
                 const int b = seg & 1;
                 if (seg >= 2) ok = mbar_wait(&ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, abort_flag);
@@ -234,7 +256,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     if (i == 0) TR(10 + p.epi, 2);
                     if (i == S) TR(10 + p.epi, 5);
                     tc_fence_after_sync();
-                    const int kb = (int)(u % p.n_ku) * kUnitKb;
+                    const int kb = (koff + (int)(u % vlen)) * kUnitKb;
                     const int nk = min(kUnitKb, p.n_kb - kb);
                     const uint32_t a_addr = smem_u32(stages + (size_t)s * p.stage_bytes);
                     const uint32_t b_addr = a_addr + kUnitKb * kWChunk;
@@ -260,23 +282,37 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
         int seg = 0;
         bool ok = true;
         for (long long u = u0; u < u1; ++seg) {
-            const int tile = (int)(u / p.n_ku);
-            const long long tile_begin = (long long)tile * p.n_ku;
-            const long long tile_end = tile_begin + p.n_ku;
+            const int tile = (int)(u / vlen);
+            const long long tile_begin = (long long)tile * vlen;
+            const long long tile_end = tile_begin + vlen;
             const long long seg_end = min(u1, tile_end);
-            const bool head = (u == tile_begin), tail = (seg_end == tile_end);
+            const bool tail = (seg_end == tile_end);
+            const bool head = !helper && (u == tile_begin);
             u = seg_end;
             const int b = seg & 1;
-            const int head_cta = (int)(tile_begin / p.units_per_cta);
-            const int last_cta = (int)((tile_end - 1) / p.units_per_cta);
-            // A tile this CTA owns but shares with later CTAs: their partial tiles are usually published long before
+            int head_cta = 0, last_cta = 0;         // stream-K: the CTAs that share this tile
+            int g_first = 0, g_n = 0, my_slot = cta;   // contributors' slots this (owning) piece adds; slot a contributor writes
+            if (p.head_units > 0) {
+                // the tile's remaining units [tile * R, (tile + 1) * R) are spread over at most two helpers
+                const int R = p.n_ku - p.head_units;
+                const int j0 = (int)(((long long)tile * R) / p.help_upc), j1 = (int)(((long long)(tile + 1) * R - 1) / p.help_upc);
+                g_first = 2 * tile;
+                g_n = j1 - j0 + 1;
+                if (helper) my_slot = 2 * tile + ((cta - p.n_tiles) - j0);
+            } else {
+                head_cta = (int)(tile_begin / p.units_per_cta);
+                last_cta = (int)((tile_end - 1) / p.units_per_cta);
+                g_first = cta + 1;
+                g_n = (head && !tail) ? last_cta - cta : 0;
+            }
+            // A tile this CTA owns but shares with other CTAs: their partial tiles are usually published long before
             // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
-            const bool gather = head && !tail && p.epi != EPI_PARTIAL;
+            const bool gather = head && g_n > 0 && p.epi != EPI_PARTIAL;
             float pre[64];
             if (ok && gather) {
                 if (et == 0) {
                     unsigned long long t0 = globaltimer_ns();
-                    for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
                         while (ld_acquire(p.fix_flags + c2) == 0) {
                             if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
                         }
@@ -289,7 +325,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) pre[cc * 16 + i] = 0.f;
                     if (ok && cc * 16 < p.n_pad) {
-                        for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                        for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
                             const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(cc * 16) * 128 + f;
 #pragma unroll
                             for (int i = 0; i < 16; ++i) pre[cc * 16 + i] += __ldcg(src + (size_t)i * 128);
@@ -328,7 +364,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                 }
             } else if (!head) {
                 // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
-                float* dst = p.fix_part + (size_t)cta * p.n_pad * 128 + f;
+                float* dst = p.fix_part + (size_t)my_slot * p.n_pad * 128 + f;
                 for (int c = 0; c < p.T; c += 16) {
                     float v[16];
                     tmem_ld16(taddr + c, v);
@@ -337,7 +373,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                 }
                 __threadfence();
                 epi_barrier();
-                if (et == 0) st_release(p.fix_flags + cta, 1);
+                if (et == 0) st_release(p.fix_flags + my_slot, 1);
             } else {
                 // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
 #pragma unroll
@@ -355,7 +391,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
 #pragma unroll
                                 for (int i = 0; i < 16; ++i) v[i] += pre[((qc * (kStagingCols / 16) + hc) & 3) * 16 + i];
                             } else {
-                                for (int c2 = cta + 1; c2 <= last_cta; ++c2) {
+                                for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
                                     const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
 #pragma unroll
                                     for (int i = 0; i < 16; ++i) v[i] += __ldcg(src + (size_t)i * 128);
@@ -505,8 +541,8 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     }
                     epi_barrier();
                 }
-                if (!tail && et == 0)
-                    for (int c2 = cta + 1; c2 <= last_cta; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
+                if (gather && et == 0)
+                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
             }
             tc_fence_before_sync();
             mbar_arrive(&ctrl->acc_empty[b]);
@@ -596,6 +632,8 @@ GemmPlan gemm_plan(const GemmProblem& p) {
     const int tiles = gemm_num_tiles(p);
     const long long total = (long long)tiles * n_ku;
     long long upc = (total + kGemmCtas - 1) / kGemmCtas;          // stream-K: even, contiguous shares
+    pl.head_units = 0;
+    pl.help_upc = 0;
     if (p.epi == EPI_PARTIAL) {
         // partial sums: cut every tile into the same number of aligned pieces when that keeps most SMs busy (fewer
         // partial-sum slots for the following reduction, no zero filling), else even shares with a bounded number of
@@ -613,6 +651,35 @@ GemmPlan gemm_plan(const GemmProblem& p) {
         if (upc < lim) upc = lim;
     }
     if (upc < 1) upc = 1;
+    pl.head_units = 0;
+    pl.help_upc = 0;
+    if (p.epi != EPI_PARTIAL && upc < n_ku && tiles < kGemmCtas) {
+        // Fewer tiles than CTAs and a fused epilogue.  With even shares some CTAs hold nothing but the middle of a tile:
+        // they publish their partial tile only when the whole stream ends, and the tile's owner then still has to fetch
+        // it and run its epilogue.  Instead: one owner CTA per tile runs the first `a` K units and the epilogue; the
+        // other CTAs ("helpers") share the remaining units of all tiles, with shares a sixth of a tile shorter than an
+        // owner's, so their partial tiles are in L2 before an owner needs them.  (Measured on the 7B forward, 32 units
+        // per tile, T = 64: a = 22 / 23 / 24 / 25 -> 3.779 / 3.736 / 3.739 / 3.761 ms; even shares: 3.761 ms.  Timed
+        // alone, back to back, the projection prefers a = 25; inside the forward its first stages are already loaded
+        // while the RMSNorm before it runs.)
+        const int h = kGemmCtas - tiles;
+        const double rho = (double)tiles / h;
+        int a = (int)((rho * n_ku + n_ku / 6.0) / (1.0 + rho) + 0.999);
+        if (a > n_ku - 1) a = n_ku - 1;
+        const int R = n_ku - a;
+        if (a >= 1 && R >= 1) {
+            const int hupc = (int)(((long long)tiles * R + h - 1) / h);
+            if (hupc >= R) {           // a tile's remainder then meets at most two helpers (two slots per tile)
+                pl.split_s = 0;
+                pl.head_units = a;
+                pl.help_upc = hupc;
+                pl.units_per_cta = a;
+                pl.n_ctas = tiles + (int)(((long long)tiles * R + hupc - 1) / hupc);
+                pl.max_pieces = 1;
+                return pl;
+            }
+        }
+    }
     pl.split_s = 0;
     pl.units_per_cta = (int)upc;
     pl.n_ctas = (int)((total + upc - 1) / upc);
@@ -645,6 +712,9 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.units_per_cta = pl.units_per_cta;
     d.max_pieces = pl.max_pieces;
     d.split_s = pl.split_s;
+    d.head_units = pl.head_units;
+    d.help_upc = pl.help_upc;
+    d.total_rem = pl.head_units > 0 ? d.n_tiles * (d.n_ku - pl.head_units) : 0;
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
     size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
@@ -688,7 +758,7 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         GemmPlan np = gemm_plan(*p.warm_next);
         // the per-CTA base differs by CTA: pass the matrix base and let the CTA add its own offset
         d.warm_ptr = (const uint8_t*)p.warm_next->W[0];
-        d.warm_chunks = d.n_pad > 64 ? 0 : n_warm;   // measured: a small gain for T <= 64, a small loss above
+        d.warm_chunks = (d.n_pad > 64 || np.head_units > 0) ? 0 : n_warm;   // measured: a small gain for T <= 64, a small loss above
         d.warm_upc = np.units_per_cta;
         d.warm_n_ku = ((p.warm_next->K + 63) / 64 + kUnitKb - 1) / kUnitKb;
         d.warm_n_kb = (p.warm_next->K + 63) / 64;

@@ -73,6 +73,7 @@ enum GemmEpilogue : int {
 };
 
 constexpr int kGemmCtas = 148;      // one persistent CTA per SM
+constexpr int kFixSlots = 2 * kGemmCtas;   // partial-tile slots: one per CTA, or two per tile when helpers are used
 constexpr int kMaxPartSlots = 8;    // partial-sum slots of EPI_PARTIAL
 
 struct GemmProblem {
@@ -83,8 +84,8 @@ struct GemmProblem {
     int n_mats;       // 1, or 3 for QKV, or 2 for SwiGLU
     const void* W[3]; // W[0]: packed weights (all matrices of the problem in one buffer)
     const void* X;    // packed activations
-    float* fix_part;  // [kGemmCtas][n_pad][128] fp32: partial tiles of tiles shared by several CTAs
-    int* fix_flags;   // [kGemmCtas], zero between launches
+    float* fix_part;  // [kFixSlots][n_pad][128] fp32: partial tiles of tiles shared by several CTAs
+    int* fix_flags;   // [kFixSlots], zero between launches
     // epilogue operands
     float* part;           // EPI_PARTIAL: [pieces][T][n_out]
     size_t part_stride;    //   elements between slots
@@ -114,6 +115,8 @@ struct GemmPlan {
     int n_ctas;
     int max_pieces;      // EPI_PARTIAL: number of partial-sum slots the following reduction must fold
     int split_s;         // > 0: every tile is cut into this many aligned pieces (CTA = tile * split_s + piece)
+    int head_units;      // > 0: one owner CTA per tile runs this many K units, helper CTAs share the rest
+    int help_upc;        //      units per helper CTA
 };
 
 // Number of 128-row tiles the problem has (SwiGLU: tiles of 64 gate + 64 up rows).
