@@ -53,6 +53,7 @@ struct AttnDev {
     const int32_t* nodes;   // null, or the tree node of each query row (selects its mask row)
     int Tk;                 // tree rows in the cache after the prefix
     int rpr;                // query rows each CTA of a cluster merges (contiguous block)
+    int qsplit;             // > 0: the CTAs of a head split the QUERY tiles (n_mt tiles each) and every CTA reads all rows
     int32_t* d_status;
     int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split, blk, kv_area;   // blk: cache rows per pipeline block (multiple of 16*kvg); kv_area: bytes of the K/V buffers
     long long kv_stride;
@@ -97,7 +98,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     volatile int* wait_expired = reinterpret_cast<volatile int*>(rbar + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int split = blockIdx.x, h = blockIdx.y;
+    const int split = p.qsplit > 0 ? 0 : (int)blockIdx.x, h = blockIdx.y;
+    const int row_base = p.qsplit > 0 ? (int)blockIdx.x * p.n_mt * 16 : 0;   // first query row of this CTA
     const int S = p.P + p.Tk;
     const int c_begin = min(S, split * p.rows_per_split);
     const int c_end = min(S, c_begin + p.rows_per_split);
@@ -148,12 +150,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
         int r = e / NCH, ch = e % NCH;
         uint32_t off = tile_off<HD>(r, ch);
-        if (r < p.T) cp_async16(q_s + off, p.q + ((size_t)r * p.nh + h) * HD + ch * 8);
+        if (row_base + r < p.T) cp_async16(q_s + off, p.q + ((size_t)(row_base + r) * p.nh + h) * HD + ch * 8);
         else *reinterpret_cast<uint4*>(q_s + off) = make_uint4(0, 0, 0, 0);
     }
     for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) {
         uint64_t w = 0ull;
-        if (e < p.T * 2) w = p.nodes != nullptr ? p.mask[(size_t)p.nodes[e >> 1] * 2 + (e & 1)] : p.mask[e];
+        const int gr = row_base + (e >> 1);
+        if (gr < p.T) w = p.mask[(size_t)(p.nodes != nullptr ? p.nodes[gr] : gr) * 2 + (e & 1)];
         mask_s[e] = w;
     }
     if (!early && nb > 0) load_kv(0, 0);
@@ -324,12 +327,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         __syncthreads();
     }
     for (int rl = warp; rl < n_my; rl += 8) {
-        const int row = row0 + rl;
+        const int row = row_base + row0 + rl;      // global query row
         if (row >= p.T) break;
         float mp = -INFINITY, lp = 0.f;
         const float* my_rec = src_parts;
         if (lane < n_parts) {
-            my_rec = src_parts + (size_t)lane * part_stride + (size_t)(csize > 1 ? rl : row) * REC;
+            my_rec = src_parts + (size_t)lane * part_stride + (size_t)(csize > 1 ? rl : row0 + rl) * REC;
             const float2 ml = *reinterpret_cast<const float2*>(my_rec + HD);
             mp = ml.x; lp = ml.y;
         }
@@ -343,7 +346,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         for (int ofs = 16; ofs > 0; ofs >>= 1) L += __shfl_xor_sync(0xffffffffu, L, ofs);
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         const bool col_ok = lane < HD / 4;
-        const float* base = src_parts + (size_t)(csize > 1 ? rl : row) * REC + lane * 4;
+        const float* base = src_parts + (size_t)(csize > 1 ? rl : row0 + rl) * REC + lane * 4;
         for (int pp = 0; pp < n_parts; ++pp) {                 // partials in a fixed order
             const float w = __shfl_sync(0xffffffffu, wp, pp);
             if (col_ok && w != 0.f) {
@@ -415,6 +418,24 @@ size_t attn_plan(AttnProblem& p) {
         if (n_outer > rows / 128) n_outer = rows / 128;
         if (n_outer < 1) n_outer = 1;
     }
+    // Trees of four or more query tiles over a short cache: split the QUERY tiles over the CTAs of a head instead.
+    // Every CTA then reads all cache rows of its head (the copies after the first come from L2), its eight warps
+    // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
+    p.qsplit = 0;
+    p.mt_per_cta = 0;
+    const int n_mt = tpad / 16;
+    if (n_mt >= 4 && S <= 4096) {
+        int mpc = 1, groups = n_mt;
+        if (p.nh * groups > 148) { mpc = 2; groups = (n_mt + 1) / 2; }
+        if (p.nh * groups <= 148 && p.nh * groups >= 96) {
+            p.qsplit = groups;
+            p.mt_per_cta = mpc;
+            p.n_splits = 1;
+            p.cluster = 1;
+            p.rows_per_split = units16 * 16;
+            return 0;
+        }
+    }
     const int splits = csize * n_outer;
     p.n_splits = n_outer;
     p.cluster = csize;
@@ -466,6 +487,11 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.kvg = 8 / d.n_mt;
     if (d.kvg > 4) d.kvg = 4;
     if (d.kvg == 3) d.kvg = 2;
+    d.qsplit = p.qsplit;
+    if (p.qsplit > 0) {
+        d.n_mt = p.mt_per_cta;       // query tiles per CTA
+        d.kvg = 8 / d.n_mt;          // all eight warps split every block of cache rows
+    }
     d.csize = p.cluster; d.n_outer = p.n_splits; d.rows_per_split = p.rows_per_split;
     d.kv_stride = p.kv_stride;
     d.scale_log2 = p.scale * 1.4426950408889634f;
@@ -485,6 +511,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
         const int gran = 16 * d.kvg;
         const int whole = (p.rows_per_split + gran - 1) / gran * gran;
         if (whole <= 192) blk = whole;
+        if (p.qsplit > 0) blk = 128;   // one 16-row step per warp and block, double-buffered
     }
     d.blk = blk;
     const int n_buf = (p.rows_per_split <= blk) ? 1 : 2;            // a single block needs no second buffer
@@ -495,7 +522,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     d.kv_area = (int)kv;
     size_t smem = qbytes + kv + (size_t)tpad * 16 + recv;
     cudaError_t e;
-    dim3 grid(p.cluster * p.n_splits, p.nh);
+    dim3 grid(p.qsplit > 0 ? p.qsplit : p.cluster * p.n_splits, p.nh);
     if (p.hd == 128) e = launch_cluster(k_tree_attn<128>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
     else e = launch_cluster(k_tree_attn<64>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
     if (e != cudaSuccess || p.n_splits == 1) return e;

@@ -91,6 +91,34 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
         : "memory");
 }
 
+// The accumulator tile of this CTA (thread = feature row f, columns = nodes) to global rows of 128 consecutive features
+// per node: dst + node * row_stride + [0, 128).  Transposed through the staging tile, 32 nodes at a time, so that every
+// store instruction of a warp writes 512 contiguous bytes (a quarter of the store instructions of the direct way, which
+// was measured to be what the partial-sum epilogues were waiting for).  n_valid nodes, feat_limit: features that exist.
+__device__ __forceinline__ void store_tile_transposed(uint32_t taddr, int n_pad, int n_valid, float* acc_s, int f, int et,
+                                                      float* dst, size_t row_stride, int feat_limit) {
+    for (int c0 = 0; c0 < n_valid; c0 += kStagingCols) {
+#pragma unroll
+        for (int hc = 0; hc < kStagingCols / 16; ++hc) {
+            if (c0 + hc * 16 >= n_pad) break;
+            float v[16];
+            tmem_ld16(taddr + c0 + hc * 16, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc_s[(hc * 16 + i) * 128 + f] = v[i];
+        }
+        epi_barrier();
+        const int l4 = et & 31;
+#pragma unroll
+        for (int k = 0; k < kStagingCols / 4; ++k) {
+            const int nl = (et >> 5) + 4 * k;
+            if (c0 + nl < n_valid && l4 * 4 < feat_limit)
+                *reinterpret_cast<float4*>(dst + (size_t)(c0 + nl) * row_stride + l4 * 4) =
+                    *reinterpret_cast<const float4*>(acc_s + nl * 128 + l4 * 4);
+        }
+        epi_barrier();
+    }
+}
+
 __device__ __forceinline__ int ld_acquire(const int* p) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -346,16 +374,8 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             } else if (p.epi == EPI_PARTIAL) {
                 const int feat = row0 + f;
                 const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
-                float* dst = p.part + (size_t)piece * p.part_stride + feat;
-                for (int c = 0; c < p.T; c += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + c, v);
-                    if (feat < p.n_out) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            if (c + i < p.T) dst[(size_t)(c + i) * p.n_out] = v[i];
-                    }
-                }
+                store_tile_transposed(taddr, p.n_pad, p.T, acc_s, f, et, p.part + (size_t)piece * p.part_stride + row0,
+                                      (size_t)p.n_out, p.n_out - row0);
                 if (head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
                     for (int sl = last_cta - head_cta + 1; sl < p.max_pieces; ++sl) {
                         float* z = p.part + (size_t)sl * p.part_stride + feat;
@@ -364,13 +384,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                 }
             } else if (!head) {
                 // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
-                float* dst = p.fix_part + (size_t)my_slot * p.n_pad * 128 + f;
-                for (int c = 0; c < p.T; c += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + c, v);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) dst[(size_t)(c + i) * 128] = v[i];
-                }
+                store_tile_transposed(taddr, p.n_pad, p.n_pad, acc_s, f, et, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
                 __threadfence();
                 epi_barrier();
                 if (et == 0) st_release(p.fix_flags + my_slot, 1);
@@ -411,40 +425,48 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     epi_barrier();
                     const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
                     if (p.epi == EPI_QKV) {
-                        // thread -> feature pair (2j, 2j+1), every other node.  All loads of the thread are issued
-                        // before the first store, so their latencies overlap.
-                        const int j2 = (et & 63) * 2;
-                        const int feat = row0 + j2;
+                        // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
+                        // the thread are issued before the first store, so their latencies overlap.
+                        const int j8 = (et & 15) * 8;
+                        const int feat = row0 + j8;
                         const int hd = p.head_dim, half = hd >> 1;
                         const int in_head = feat % hd;
                         const bool first_half = in_head < half;
-                        const int partner = first_half ? j2 + half : j2 - half;
+                        const int partner = first_half ? j8 + half : j8 - half;
                         const int ri = in_head % half;
                         const float sgn = first_half ? -1.f : 1.f;
-                        constexpr int NI = kStagingCols / 2;
+                        constexpr int NI = kStagingCols / 8;
                         if (feat < p.n_out) {
-                            uint32_t packed[NI];
+                            uint4 packed[NI];
                             if (mat < 2) {
-                                float4 cs[NI];
+                                float4 cs[NI][4];     // (cos, sin) of the 8 feature pairs
 #pragma unroll
                                 for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 6) + 2 * it;
-                                    cs[it] = nl < n_hi ? __ldg(reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * half + ri))
-                                                       : make_float4(1.f, 0.f, 1.f, 0.f);
+                                    const int nl = (et >> 4) + 8 * it;
+                                    const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * half + ri);
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q) cs[it][q] = nl < n_hi ? __ldg(src + q) : make_float4(1.f, 0.f, 1.f, 0.f);
                                 }
 #pragma unroll
                                 for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 6) + 2 * it;
-                                    float2 x = *reinterpret_cast<const float2*>(acc_s + nl * 128 + j2);
-                                    float2 y = *reinterpret_cast<const float2*>(acc_s + nl * 128 + partner);
-                                    packed[it] = pack_bf16x2(x.x * cs[it].x + sgn * y.x * cs[it].y, x.y * cs[it].z + sgn * y.y * cs[it].w);
+                                    const int nl = (et >> 4) + 8 * it;
+                                    const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                                    const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
+                                    const float4 y0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner);
+                                    const float4 y1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner + 4);
+                                    packed[it].x = pack_bf16x2(x0.x * cs[it][0].x + sgn * y0.x * cs[it][0].y, x0.y * cs[it][0].z + sgn * y0.y * cs[it][0].w);
+                                    packed[it].y = pack_bf16x2(x0.z * cs[it][1].x + sgn * y0.z * cs[it][1].y, x0.w * cs[it][1].z + sgn * y0.w * cs[it][1].w);
+                                    packed[it].z = pack_bf16x2(x1.x * cs[it][2].x + sgn * y1.x * cs[it][2].y, x1.y * cs[it][2].z + sgn * y1.y * cs[it][2].w);
+                                    packed[it].w = pack_bf16x2(x1.z * cs[it][3].x + sgn * y1.z * cs[it][3].y, x1.w * cs[it][3].z + sgn * y1.w * cs[it][3].w);
                                 }
                             } else {
 #pragma unroll
                                 for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 6) + 2 * it;
-                                    float2 x = *reinterpret_cast<const float2*>(acc_s + nl * 128 + j2);
-                                    packed[it] = pack_bf16x2(x.x, x.y);
+                                    const int nl = (et >> 4) + 8 * it;
+                                    const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                                    const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
+                                    packed[it] = make_uint4(pack_bf16x2(x0.x, x0.y), pack_bf16x2(x0.z, x0.w), pack_bf16x2(x1.x, x1.y),
+                                                            pack_bf16x2(x1.z, x1.w));
                                 }
                             }
                             if (mat == 0 || p.kv_rows == nullptr) {
@@ -452,40 +474,40 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                                                           : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
 #pragma unroll
                                 for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 6) + 2 * it;
-                                    if (nl < n_hi) *reinterpret_cast<uint32_t*>(base + (size_t)nl * p.n_out + feat) = packed[it];
+                                    const int nl = (et >> 4) + 8 * it;
+                                    if (nl < n_hi) *reinterpret_cast<uint4*>(base + (size_t)nl * p.n_out + feat) = packed[it];
                                 }
                             } else {
                                 // a subset of the tree: row t of the batch is tree node kv_rows[t]
                                 uint16_t* base = (mat == 1 ? p.kcache : p.vcache) + (size_t)p.prefix_len * p.n_out;
 #pragma unroll
                                 for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 6) + 2 * it;
+                                    const int nl = (et >> 4) + 8 * it;
                                     if (nl < n_hi)
-                                        *reinterpret_cast<uint32_t*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
+                                        *reinterpret_cast<uint4*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
                                 }
                             }
                         }
                     } else if (p.epi == EPI_SWIGLU) {
                         // features beyond n_out come out as silu(0)*0 = 0 (zero-padded weights): they are stored too,
-                        // so that the padded K block of the down projection's input reads as zeros
-                        const int j2 = (et & 31) * 2;
-                        const int feat = row0 + j2;
-                        constexpr int NI = kStagingCols / 4;
-                        uint32_t packed[NI];
+                        // so that the padded K block of the down projection's input reads as zeros.
+                        // thread -> 8 consecutive features = one 16-byte group of the packed layout, every 16th node
+                        const int j8 = (et & 7) * 8;
+                        const int feat = row0 + j8;
+                        constexpr int NI = kStagingCols / 16;
 #pragma unroll
                         for (int it = 0; it < NI; ++it) {
-                            const int nl = (et >> 5) + 4 * it;
-                            float2 g = *reinterpret_cast<const float2*>(acc_s + nl * 128 + j2);
-                            float2 u = *reinterpret_cast<const float2*>(acc_s + nl * 128 + 64 + j2);
-                            packed[it] = pack_bf16x2(__fdividef(g.x, 1.f + __expf(-g.x)) * u.x, __fdividef(g.y, 1.f + __expf(-g.y)) * u.y);
-                        }
-#pragma unroll
-                        for (int it = 0; it < NI; ++it) {
-                            const int nl = (et >> 5) + 4 * it;
-                            if (nl < n_hi)
-                                *reinterpret_cast<uint32_t*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad) +
-                                                             (size_t)(feat & 7) * 2) = packed[it];
+                            const int nl = (et >> 3) + 16 * it;
+                            const float4 g0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                            const float4 g1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
+                            const float4 u0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8);
+                            const float4 u1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8 + 4);
+                            uint4 o;
+                            o.x = pack_bf16x2(__fdividef(g0.x, 1.f + __expf(-g0.x)) * u0.x, __fdividef(g0.y, 1.f + __expf(-g0.y)) * u0.y);
+                            o.y = pack_bf16x2(__fdividef(g0.z, 1.f + __expf(-g0.z)) * u0.z, __fdividef(g0.w, 1.f + __expf(-g0.w)) * u0.w);
+                            o.z = pack_bf16x2(__fdividef(g1.x, 1.f + __expf(-g1.x)) * u1.x, __fdividef(g1.y, 1.f + __expf(-g1.y)) * u1.y);
+                            o.w = pack_bf16x2(__fdividef(g1.z, 1.f + __expf(-g1.z)) * u1.z, __fdividef(g1.w, 1.f + __expf(-g1.w)) * u1.w);
+                            if (nl < n_hi) *reinterpret_cast<uint4*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad)) = o;
                         }
                     } else if (p.epi == EPI_LMHEAD) {
                         for (int nl = warp - 2; nl < n_hi; nl += 4) {

@@ -144,6 +144,8 @@ struct AttnProblem {
     int n_splits;       // filled by attn_plan: clusters per head (> 1 only for long prefixes with few heads)
     int cluster;        //   CTAs per cluster
     int rows_per_split; //   cache rows per CTA (multiple of 16)
+    int qsplit;         //   > 0: CTAs per head that split the query tiles instead (every CTA reads all cache rows)
+    int mt_per_cta;     //   query tiles per CTA in that case
     int32_t* d_status;
 };
 // Chooses the KV split; returns bytes of partial storage needed.
