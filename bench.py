@@ -32,7 +32,7 @@ METRIC = "verified tree tokens/sec per forward (7B-shape)"
 UNIT = "tree tokens/s"
 PREFIX = 512
 SWEEP = (16, 32, 64, 128)
-NCU_TRAFFIC_PER_LAUNCH = (32 * (113.5e6 + 42.5e6 + 194.1e6 + 103.6e6) + 272e6) / 129
+NCU_TRAFFIC_PER_LAUNCH = (32 * (113.7e6 + 42.5e6 + 195.5e6 + 95.6e6) + 272e6) / 129
 
 
 # --------------------------------------------------------------------------------------------------
@@ -283,7 +283,7 @@ def run_ours(args, rank, world, local_rank):
                      "achieved": wb / n_gemm / (gemm_sec / n_gemm) / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": wb / gemm_sec / 1e9 / peak, "peak_kind": peak_kind,
                      # dram__bytes_read + write per launch from the ncu capture of a 2-layer stack (profiles/k_gemm_sk_7b_T64.md),
-                     # scaled to the 129 launches of a forward: 32 x (113.5 + 42.5 + 194.1 + 103.6) MB + LM head
+                     # scaled to the 129 launches of a forward: 32 x (113.7 + 42.5 + 195.5 + 95.6) MB + LM head
                      "traffic": NCU_TRAFFIC_PER_LAUNCH if T == 64 else None,
                      "bytes_per_launch": wb / n_gemm, "us_per_launch": gemm_sec / n_gemm * 1e6,
                      "forward_achieved": fb / sec_step / 1e9, "forward_frac": fb / sec_step / 1e9 / peak,

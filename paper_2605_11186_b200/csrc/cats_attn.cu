@@ -17,7 +17,6 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
-CATS_TRACE_DEFINE(attn)
 
 constexpr int kAttnThreads = 256;
 constexpr int kKvBlock = 64;
@@ -131,7 +130,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     pdl_launch_dependents();
     // the first block can be requested before the previous kernel has finished if it lies in the prefix
     const bool early = (c_begin + p.blk <= p.P);
-    if (threadIdx.x == 0) TR(2, 0);
     if (early) load_kv(0, 0);
     if (p.csize > 1) {
         // the barrier the cluster's pushed partials complete on; visible to the peers before anybody can send
@@ -146,7 +144,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
         cluster_sync_all();
     }
     pdl_wait();
-    if (threadIdx.x == 0) TR(2, 1);
     for (int e = threadIdx.x; e < Tpad * NCH; e += kAttnThreads) {
         int r = e / NCH, ch = e % NCH;
         uint32_t off = tile_off<HD>(r, ch);

@@ -23,38 +23,6 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     return t;
 }
 
-#ifdef CATS_TRACE
-// Bring-up timeline: (tag, event, cta, sm, time) entries in a per-translation-unit device buffer.
-#define CATS_TRACE_CAP (1u << 18)
-#define CATS_TRACE_DEFINE(name)                                                                          \
-    static __device__ unsigned long long g_tr[2 * CATS_TRACE_CAP];                                       \
-    static __device__ unsigned g_trn;                                                                    \
-    extern "C" int cats_trace_##name(unsigned long long* out, unsigned cap) {                            \
-        unsigned n = 0;                                                                                  \
-        cudaMemcpyFromSymbol(&n, g_trn, sizeof(n));                                                      \
-        if (n > CATS_TRACE_CAP) n = CATS_TRACE_CAP;                                                      \
-        if (n > cap) n = cap;                                                                            \
-        cudaMemcpyFromSymbol(out, g_tr, (size_t)n * 16);                                                 \
-        unsigned z = 0;                                                                                  \
-        cudaMemcpyToSymbol(g_trn, &z, sizeof(z));                                                        \
-        return (int)n;                                                                                   \
-    }
-#define TR(tag, ev)                                                                                      \
-    do {                                                                                                 \
-        unsigned i_ = atomicAdd(&g_trn, 1u);                                                             \
-        if (i_ < CATS_TRACE_CAP) {                                                                       \
-            unsigned sm_;                                                                                \
-            asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_));                                             \
-            g_tr[2 * i_] = ((unsigned long long)(tag) << 48) | ((unsigned long long)(ev) << 40) |        \
-                           ((unsigned long long)blockIdx.x << 16) | sm_;                                 \
-            g_tr[2 * i_ + 1] = globaltimer_ns();                                                         \
-        }                                                                                                \
-    } while (0)
-#else
-#define CATS_TRACE_DEFINE(name)
-#define TR(tag, ev) do { } while (0)
-#endif
-
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

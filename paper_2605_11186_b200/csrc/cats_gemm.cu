@@ -30,7 +30,6 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
-CATS_TRACE_DEFINE(gemm)
 
 constexpr int kGemmThreads = 224;
 constexpr int kCtrlBytes = 512;
@@ -204,7 +203,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
     __syncthreads();
     tc_fence_after_sync();
     pdl_launch_dependents();
-    if (threadIdx.x == 0) TR(10 + p.epi, 0);
     const uint32_t tmem_acc = ctrl->tmem_base;
 
     if (warp == 0 || warp == 6) {
@@ -232,7 +230,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &ctrl->full[s], pol);
                 }
             };
-            if (!is_w) { pdl_wait(); TR(10 + p.epi, 1); }    // activations come from the previous kernel; weights never do
+            if (!is_w) pdl_wait();    // activations come from the previous kernel; weights never do
             int issued = 0;
             for (int i = 0; i < n_units; ++i) {
                 if (i >= S && !mbar_wait(&ctrl->empty[i % S], ((i / S) - 1) & 1, abort_flag)) break;
@@ -281,8 +279,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     int s = i % S;
                     ok = mbar_wait(&ctrl->full[s], (i / S) & 1, abort_flag);
                     if (!ok) break;
-                    if (i == 0) TR(10 + p.epi, 2);
-                    if (i == S) TR(10 + p.epi, 5);
                     tc_fence_after_sync();
                     const int kb = (koff + (int)(u % vlen)) * kUnitKb;
                     const int nk = min(kUnitKb, p.n_kb - kb);
@@ -299,7 +295,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                 }
                 umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
             }
-            TR(10 + p.epi, 3);
         }
     } else if (warp < 6) {
         // ---------------- epilogue warps ----------------
@@ -572,7 +567,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (threadIdx.x == 0) TR(10 + p.epi, 4);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();

@@ -4,7 +4,6 @@
 #include "cats_kernels.cuh"
 
 namespace cats {
-CATS_TRACE_DEFINE(small)
 
 // ---------------------------------------------------------------------------------------------
 // Ancestor mask, depth, position ids.  One CTA of 128 threads; thread i walks from node i to the
@@ -431,7 +430,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
     const int t = blockIdx.x / cs, rank = blockIdx.x - t * cs;
     const int cols_cta = H / 4 / cs;          // float4 columns of this CTA
     const int col0 = rank * cols_cta;
-    if (threadIdx.x == 0) TR(1, 0);
     // everything that does not depend on the previous kernel: the exchange barrier and the gains
     if (cs > 1) {
         if (threadIdx.x == 0) {
@@ -450,7 +448,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         if (xn != nullptr && cl < cols_cta) g[j] = __ldg(reinterpret_cast<const uint2*>(gain) + col0 + cl);
     }
     pdl_wait();
-    if (threadIdx.x == 0) TR(1, 1);
     if (zero_flags != nullptr && blockIdx.x == 0)
         for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
     if (rope != nullptr && rank == cs - 1) {
@@ -497,7 +494,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         a[j] = v;
     }
-    if (threadIdx.x == 0) TR(1, 2);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -523,7 +519,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         tot = 0.f;
         for (int r = 0; r < cs; ++r) tot += slots[r];    // rank order: every CTA of the cluster gets the same bits
     }
-    if (threadIdx.x == 0) TR(1, 3);
     const float rs = rsqrtf(tot / (float)H + eps);
     const bool write_resid = n_part > 0 || copy_from != nullptr;
     float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
@@ -541,7 +536,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
             *reinterpret_cast<uint2*>(xn + packed_act_offset(t, c >> 1, n_pad) + (size_t)(c & 1) * 8) = o;
         }
     }
-    if (threadIdx.x == 0) TR(1, 4);
 }
 
 template <typename Kern, typename... Args>
