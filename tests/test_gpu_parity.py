@@ -211,6 +211,10 @@ ATTN_CASES = [
     ("rand77_P333_hd64", gen.tree_random(77, 2), 333, 4, 64), ("b4211_P128_hd64", gen.tree_branching([4, 2, 1, 1], 16), 128, 4, 64),
     ("chain5_P0", gen.tree_chain(5), 0, 2, 128), ("single_P1", gen.tree_chain(1), 1, 3, 64), ("rand40_P7", gen.tree_random(40, 3), 7, 5, 128),
     ("rand100_P63", gen.tree_random(100, 4), 63, 6, 64),
+    # 32 heads, five and seven query tiles: two tiles per CTA with a ragged last group; 49 nodes: the smallest such tree
+    ("rand77_P300_h32", gen.tree_random(77, 2), 300, 32, 128), ("rand100_P63_h32", gen.tree_random(100, 4), 63, 32, 128),
+    ("rand49_P200_h32", gen.tree_random(49, 6), 200, 32, 128), ("rand48_P200_h32", gen.tree_random(48, 6), 200, 32, 128),
+    ("rand128_P3968_h32", gen.tree_random(128, 9), 3968, 32, 128), ("rand128_P3969_h32", gen.tree_random(128, 9), 3969, 32, 128),
 ]
 
 
