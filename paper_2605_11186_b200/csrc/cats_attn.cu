@@ -190,15 +190,22 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
             // 16 rows of the slice at a time: S = Q K^T (16 x 16), mask, online softmax, O += P V
             for (int sub = 0; sub < R; sub += 16) {
                 if (cbase + sub >= c_end) break;
+                // two accumulator pairs (even and odd k-steps): the chain of dependent MMAs is half as long
                 float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    uint32_t b0, b1, b2, b3;
-                    int r = rbase + sub + (lane & 7) + ((lane >> 4) << 3), ch = ks * 2 + ((lane >> 3) & 1);
+                for (int ks = 0; ks < KS; ks += 2) {
+                    uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+                    const int r = rbase + sub + (lane & 7) + ((lane >> 4) << 3), ch = ks * 2 + ((lane >> 3) & 1);
                     ldmatrix_x4(smem_u32(ks_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
+                    ldmatrix_x4(smem_u32(ks_s + tile_off<HD>(r, ch + 2)), c0, c1, c2, c3);
                     mma_bf16_16816(s0, qf[ks], b0, b1);
                     mma_bf16_16816(s1, qf[ks], b2, b3);
+                    mma_bf16_16816(t0, qf[ks + 1], c0, c1);
+                    mma_bf16_16816(t1, qf[ks + 1], c2, c3);
                 }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) { s0[e] += t0[e]; s1[e] += t1[e]; }
                 // visibility of the 4+4 scores this thread holds
                 float sc[8];
                 {
