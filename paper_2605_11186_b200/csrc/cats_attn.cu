@@ -1,17 +1,19 @@
 // Tree-masked attention of the T draft-tree nodes against the KV prefix plus their own ancestors.
 //
-// Split-KV inside a thread-block cluster: the cache rows [0, prefix + T) of one head are divided
-// among the CTAs of a cluster (up to 8).  Each CTA streams its rows in blocks of 64 through a double
-// buffered cp.async pipeline (128-bit loads), keeps Q [T_pad][hd] in shared memory, and computes
-// S = Q K^T and O += P V with bf16 tensor-core MMAs (fp32 accumulation, online softmax in fp32 with
-// warp-shuffle row reductions).  Prefix rows need no mask; rows >= prefix_len test bit (row - prefix)
-// of the node's 128-bit ancestor mask held in shared memory.  Warps are laid out as (16-row query
-// tile) x (slice of the 64-row block), so small trees still use every warp.  Every warp leaves its
-// partial (m, l, O) in its CTA's shared memory; after a cluster barrier the CTAs merge all partials of
-// the head by log-sum-exp, reading each other's shared memory (distributed shared memory), each CTA
-// finishing a share of the rows, and write the bf16 result.  Only when a head has far more rows than a
-// cluster can cover with few heads (long prefixes, few heads) are several clusters used per head; their
-// merged partials then go to the caller's workspace and k_attn_combine merges them.
+// Q [T_pad][hd] sits in shared memory; the cache rows stream through a double-buffered cp.async pipeline
+// (128-bit loads); S = Q K^T and O += P V run on bf16 tensor-core MMAs (fp32 accumulation, online softmax in
+// fp32 with warp-shuffle row reductions, the probabilities as a bf16 pair hi + lo).  Prefix rows need no mask;
+// rows >= prefix_len test bit (row - prefix) of the node's 128-bit ancestor mask held in shared memory.
+// Warps are laid out as (16-row query tile) x (slice of the block of rows), so small trees still use every
+// warp; every warp leaves its partial (m, l, O) in its CTA's shared memory.  Two ways of dividing a head:
+//   * query split (trees of four or more query tiles over a short cache): the CTAs of a head take different
+//     query tiles, every CTA reads all rows and merges its warps' partials alone;
+//   * split-KV inside a thread-block cluster (up to 8 CTAs): the rows are divided among the CTAs; each CTA
+//     pushes, per destination, the records of the query rows that destination merges, with bulk copies through
+//     distributed shared memory completing on the destination's mbarrier; the merge reads local memory only.
+// The merge is by log-sum-exp in a fixed order; the result is written as bf16.  Only when a head has far more
+// rows than a cluster can cover with few heads (long prefixes, few heads) are several clusters used per head;
+// their merged partials then go to the caller's workspace and k_attn_combine merges them.
 #include <mutex>
 
 #include "cats_kernels.cuh"

@@ -9,19 +9,22 @@
 //     128-byte swizzle).  Chunks of a tile are consecutive, tiles are consecutive.
 //   * X (the T tree nodes, padded to a multiple of 16) is kept by its producers in the same layout, one
 //     chunk of n_pad x 128 bytes per K block.
-//   * The (tile, K block) pairs are split evenly and contiguously over the CTAs ("stream-K"): CTA c
-//     copies bytes [c, c+1) * units_per_cta * 16 KB of the packed matrix with plain bulk copies, a
-//     pattern that reaches the HBM copy rate with one CTA per SM.
-// Warp 0 is the copy producer (ring of shared-memory stages, mbarrier completion), warp 1 issues
-// tcgen05.mma into one of two TMEM accumulators, warps 2-5 drain the other accumulator and run the
-// epilogue.  A tile whose K range is shared by several CTAs is finished by the CTA that owns its
-// first K block: the others publish fp32 partial tiles and a flag; the owner adds them in CTA order
-// (deterministic) and runs the epilogue.  Split-K partial sums of the O and down projections are
+//   * One persistent CTA per SM copies its share of the packed matrix with plain contiguous bulk copies, a
+//     pattern that reaches the HBM copy rate.  How the (tile, K unit) pairs are shared out depends on the
+//     projection (gemm_plan): aligned K pieces of every tile for the partial-sum projections, even contiguous
+//     shares ("stream-K") when there are more tiles than SMs, one owner CTA per tile plus helper CTAs when
+//     there are fewer.
+// Warp 0 (one thread) copies W, warp 6 (one thread) copies X, both into a ring of shared-memory stages with
+// mbarrier completion; warp 1 issues tcgen05.mma into one of two TMEM accumulators; warps 2-5 drain the other
+// accumulator and run the epilogue.  A tile whose K range is shared by several CTAs is finished by the CTA
+// that owns its first K units: the others publish fp32 partial tiles and a flag; the owner adds them in a fixed
+// order (deterministic) and runs the epilogue.  Split-K partial sums of the O and down projections are
 // not reduced here at all: the following RMSNorm kernel folds them into the residual stream.
 //   EPI_PARTIAL  fp32 partial sums, one slot per piece of a tile
 //   EPI_QKV      rotary embedding, bf16 q, k/v appended to the KV cache
 //   EPI_SWIGLU   silu(gate) * up from a tile holding 64 gate rows and the matching 64 up rows
-//   EPI_LMHEAD   fp32 logits and per-tile argmax candidates
+//   EPI_LMHEAD   fp32 logits, per-tile argmax candidates and (optionally) per-tile softmax statistics
+// All epilogues go through a 32-node staging tile in shared memory so that every thread stores 16 bytes.
 // Weight chunks of the first stages are requested before griddepcontrol.wait (weights never depend on
 // an earlier kernel).  Every wait (mbarrier or flag) is bounded; on expiry the CTA reports
 // CATS_ERR_TIMEOUT, lets its copies land, frees its TMEM and returns.
