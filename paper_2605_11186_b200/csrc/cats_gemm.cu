@@ -138,6 +138,7 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 #ifndef CATS_GEMM_MAXREG
 #define CATS_GEMM_MAXREG 192
 #endif
+template <int EPI>
 __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* stages = smem_raw;                                                             // 1024-byte aligned (checked)
@@ -333,7 +334,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             }
             // A tile this CTA owns but shares with other CTAs: their partial tiles are usually published long before
             // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
-            const bool gather = head && g_n > 0 && p.epi != EPI_PARTIAL;
+            const bool gather = head && g_n > 0 && EPI != EPI_PARTIAL;
             float pre[64];
             if (ok && gather) {
                 if (et == 0) {
@@ -364,12 +365,12 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             tc_fence_after_sync();
             const uint32_t taddr = tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * p.n_pad);
             int mat = 0, row0;
-            if (p.epi == EPI_SWIGLU) row0 = tile * 64;
+            if (EPI == EPI_SWIGLU) row0 = tile * 64;
             else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
 
             if (!ok) {
                 // nothing: fall through to the arrive below so that nobody waits on this accumulator
-            } else if (p.epi == EPI_PARTIAL) {
+            } else if (EPI == EPI_PARTIAL) {
                 const int feat = row0 + f;
                 const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
                 store_tile_transposed(taddr, p.n_pad, p.T, acc_s, f, et, p.part + (size_t)piece * p.part_stride + row0,
@@ -410,7 +411,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                                 }
                             }
                         }
-                        if (p.epi == EPI_LMHEAD && p.logits != nullptr && row0 + f < p.n_out) {
+                        if (EPI == EPI_LMHEAD && p.logits != nullptr && row0 + f < p.n_out) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i) {
                                 int n = c0 + c + i;
@@ -422,7 +423,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     }
                     epi_barrier();
                     const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
-                    if (p.epi == EPI_QKV) {
+                    if (EPI == EPI_QKV) {
                         // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
                         // the thread are issued before the first store, so their latencies overlap.
                         const int j8 = (et & 15) * 8;
@@ -486,7 +487,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                                 }
                             }
                         }
-                    } else if (p.epi == EPI_SWIGLU) {
+                    } else if (EPI == EPI_SWIGLU) {
                         // features beyond n_out come out as silu(0)*0 = 0 (zero-padded weights): they are stored too,
                         // so that the padded K block of the down projection's input reads as zeros.
                         // thread -> 8 consecutive features = one 16-byte group of the packed layout, every 16th node
@@ -507,7 +508,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                             o.w = pack_bf16x2(__fdividef(g1.z, 1.f + __expf(-g1.z)) * u1.z, __fdividef(g1.w, 1.f + __expf(-g1.w)) * u1.w);
                             if (nl < n_hi) *reinterpret_cast<uint4*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad)) = o;
                         }
-                    } else if (p.epi == EPI_LMHEAD) {
+                    } else if (EPI == EPI_LMHEAD) {
                         for (int nl = warp - 2; nl < n_hi; nl += 4) {
                             float best = -INFINITY;
                             int bi = 0x7fffffff;
@@ -713,7 +714,10 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     const int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_sk, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_sk<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_LMHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -783,7 +787,13 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         d.warm_n_kb = (p.warm_next->K + 63) / 64;
         d.warm_total_chunks = (long long)gemm_num_tiles(*p.warm_next) * d.warm_n_kb;
     }
-    return launch_pdl(k_gemm_sk, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
+    switch (p.epi) {
+        case EPI_PARTIAL: return launch_pdl(k_gemm_sk<EPI_PARTIAL>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
+        case EPI_QKV: return launch_pdl(k_gemm_sk<EPI_QKV>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
+        case EPI_SWIGLU: return launch_pdl(k_gemm_sk<EPI_SWIGLU>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
+        case EPI_LMHEAD: return launch_pdl(k_gemm_sk<EPI_LMHEAD>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
+        default: return cudaErrorInvalidValue;
+    }
 }
 
 }  // namespace cats
