@@ -210,7 +210,11 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
                 for (int e = 0; e < 4; ++e) { s0[e] += t0[e]; s1[e] += t1[e]; }
                 // visibility of the 4+4 scores this thread holds
                 float sc[8];
-                {
+                if (cbase + sub + 16 <= p.P) {
+                    // 16 prefix rows: every one visible to every node
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) sc[e] = ((e >> 2) ? s1[e & 3] : s0[e & 3]) * p.scale_log2;
+                } else {
                     const uint64_t ma0 = mask_s[row_a * 2], ma1 = mask_s[row_a * 2 + 1];
                     const uint64_t mb0 = mask_s[row_b * 2], mb1 = mask_s[row_b * 2 + 1];
 #pragma unroll
@@ -245,8 +249,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
                 for (int e = 0; e < 8; ++e) pr[e] = exp2f(sc[e] - (((e & 3) >> 1) ? ref_b : ref_a));
                 l_run[0] = l_run[0] * corr_a + pr[0] + pr[1] + pr[4] + pr[5];
                 l_run[1] = l_run[1] * corr_b + pr[2] + pr[3] + pr[6] + pr[7];
+                if (__any_sync(0xffffffffu, corr_a != 1.f || corr_b != 1.f)) {   // a running maximum moved: rescale O
 #pragma unroll
-                for (int j = 0; j < NT; ++j) { o[j][0] *= corr_a; o[j][1] *= corr_a; o[j][2] *= corr_b; o[j][3] *= corr_b; }
+                    for (int j = 0; j < NT; ++j) { o[j][0] *= corr_a; o[j][1] *= corr_a; o[j][2] *= corr_b; o[j][3] *= corr_b; }
+                }
                 // The probabilities enter the P V product as bf16 pairs hi + lo (hi = bf16(p), lo = bf16(p - hi)),
                 // so the product carries ~16 mantissa bits of p instead of 8; V is bf16 exactly.
                 uint32_t pa[4], pl[4];
