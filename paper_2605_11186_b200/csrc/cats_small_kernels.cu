@@ -450,16 +450,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
     pdl_wait();
     if (zero_flags != nullptr && blockIdx.x == 0)
         for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
-    if (rope != nullptr && rank == cs - 1) {
-        int half = hd / 2;
-        int p = pos[nodes != nullptr ? nodes[t] : t];
-        for (int i = threadIdx.x; i < half; i += blockDim.x) {
-            double inv_freq = pow((double)rope_base, -2.0 * (double)i / (double)hd);
-            double s, c;
-            sincos((double)p * inv_freq, &s, &c);
-            rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
-        }
-    }
     const float4* r4 = reinterpret_cast<const float4*>((copy_from ? copy_from : resid) + (size_t)t * H);
     float4 a[NC];
     float4 pv[NC][kMaxPartSlots / 2];
@@ -477,6 +467,17 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         for (int s = 0; s < kMaxPartSlots / 2; ++s)
             if (s < n_part && cl < cols_cta)
                 pv[j][s] = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + col0 + cl);
+    }
+    // the rotary table of this node (fp64 so that large positions lose no accuracy): computed while the loads are in flight
+    if (rope != nullptr && rank == cs - 1) {
+        int half = hd / 2;
+        int p = pos[nodes != nullptr ? nodes[t] : t];
+        for (int i = threadIdx.x; i < half; i += blockDim.x) {
+            double inv_freq = pow((double)rope_base, -2.0 * (double)i / (double)hd);
+            double s, c;
+            sincos((double)p * inv_freq, &s, &c);
+            rope[(size_t)t * half + i] = make_float2((float)c, (float)s);
+        }
     }
     float ss = 0.f;
 #pragma unroll
@@ -501,6 +502,15 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
+    const bool write_resid = n_part > 0 || copy_from != nullptr;
+    float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
+    if (write_resid) {      // the new residual does not depend on the other CTAs' sums
+#pragma unroll
+        for (int j = 0; j < NC; ++j) {
+            const int cl = threadIdx.x + 256 * j;
+            if (cl < cols_cta) out4[col0 + cl] = a[j];
+        }
+    }
     if (cs > 1) {
         // every CTA sends its partial sum to slot [rank] of every CTA of the cluster (itself included); the store
         // signals the receiver's barrier, so one one-way trip through distributed shared memory is all that is waited for
@@ -520,15 +530,12 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         for (int r = 0; r < cs; ++r) tot += slots[r];    // rank order: every CTA of the cluster gets the same bits
     }
     const float rs = rsqrtf(tot / (float)H + eps);
-    const bool write_resid = n_part > 0 || copy_from != nullptr;
-    float4* out4 = reinterpret_cast<float4*>(resid + (size_t)t * H);
 #pragma unroll
     for (int j = 0; j < NC; ++j) {
         const int cl = threadIdx.x + 256 * j;
         if (cl >= cols_cta) continue;
         const int c = col0 + cl;
         const float4 x = a[j];
-        if (write_resid) out4[c] = x;
         if (xn != nullptr) {
             uint2 o;
             o.x = pack_bf16x2(__uint_as_float(g[j].x << 16) * (x.x * rs), __uint_as_float(g[j].x & 0xFFFF0000u) * (x.y * rs));
