@@ -677,14 +677,18 @@ GemmPlan gemm_plan(const GemmProblem& p) {
         // Fewer tiles than CTAs and a fused epilogue.  With even shares some CTAs hold nothing but the middle of a tile:
         // they publish their partial tile only when the whole stream ends, and the tile's owner then still has to fetch
         // it and run its epilogue.  Instead: one owner CTA per tile runs the first `a` K units and the epilogue; the
-        // other CTAs ("helpers") share the remaining units of all tiles, with shares a sixth of a tile shorter than an
-        // owner's, so their partial tiles are in L2 before an owner needs them.  (Measured on the 7B forward, 32 units
-        // per tile, T = 64: a = 22 / 23 / 24 / 25 -> 3.779 / 3.736 / 3.739 / 3.761 ms; even shares: 3.761 ms.  Timed
-        // alone, back to back, the projection prefers a = 25; inside the forward its first stages are already loaded
-        // while the RMSNorm before it runs.)
+        // other CTAs ("helpers") share the remaining units of all tiles, with shorter shares than an owner's, so their
+        // partial tiles are in L2 before an owner needs them.  How much shorter grows with the tree (the published tiles
+        // and the owner's epilogue grow with it).  Measured on the 7B forward, 32 units per tile, owner units a:
+        //   T = 16:  a = 22 / 23 / 24 / 25 -> 3.136 / 3.115 / 3.128 / 3.151 ms
+        //   T = 64:  a = 23 / 24 / 25 / 26 -> 3.539 / 3.506 / 3.484 / 3.503 ms
+        //   T = 128: a = 25 / 26 / 27 / 28 -> 4.199 / 4.144 / 4.163 / 4.187 ms
         const int h = kGemmCtas - tiles;
         const double rho = (double)tiles / h;
-        int a = (int)((rho * n_ku + n_ku / 6.0) / (1.0 + rho) + 0.999);
+        int lg = 0;                                    // log2(n_pad / 16): 0, 1, 2, 3 for trees of up to 16, 32, 64, 128 nodes
+        for (int n = ((p.T + 15) / 16) * 16; n > 16; n = (n + 1) / 2) ++lg;
+        const double lead = (5.0 + 3.0 * lg) * n_ku / 32.0;
+        int a = (int)((rho * n_ku + lead) / (1.0 + rho) + 0.999);
         if (a > n_ku - 1) a = n_ku - 1;
         const int R = n_ku - a;
         if (a >= 1 && R >= 1) {
