@@ -93,7 +93,7 @@ inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintp
 // sums this layer's down projection left pending (>0) or a negative status.
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               const void* next_w, size_t next_w_bytes, bool next_is_head, int32_t* d_status, cudaStream_t st,
+               const void* next_w, bool next_is_head, int32_t* d_status, cudaStream_t st,
                const int32_t* nodes = nullptr, int T_tree = 0) {
     const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
     const int tpad = (T + 15) / 16 * 16;
@@ -298,7 +298,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     Workspace ws = carve(cfg, T, d_ws);
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, nullptr, 0,
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, nullptr,
                              false, d_status, st);
     if (pending < 0) return pending;
     if (stage_on(6))
@@ -327,7 +327,7 @@ int cats_verify_layer_nodes(const cats_model_cfg* cfg, const cats_layer_weights*
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     CATS_CUDA(launch_check_nodes(d_nodes, m, T, ws.nodes, d_status, st));
-    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, m, prefix_len, ws, 0, nullptr, 0,
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, m, prefix_len, ws, 0, nullptr,
                              false, d_status, st, ws.nodes, T);
     if (pending < 0) return pending;
     CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, m, cfg->hidden, cfg->rms_eps, nullptr,
@@ -472,10 +472,8 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     for (int l = 0; l < c->n_layers; ++l) {
         const bool last = (l + 1 == c->n_layers);
         const void* next_w = last ? a->d_w_lm : a->layers[l + 1].wqkv;
-        const size_t next_b = last ? packed_weight_bytes(1, 0, c->vocab, c->hidden)
-                                   : packed_weight_bytes(3, 0, c->n_heads * c->head_dim, c->hidden);
         pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
-                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, next_w, next_b,
+                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, next_w,
                              last, a->d_status, st);
         if (pending < 0) return pending;
     }

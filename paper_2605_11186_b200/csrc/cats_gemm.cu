@@ -28,8 +28,6 @@
 // Weight chunks of the first stages are requested before griddepcontrol.wait (weights never depend on
 // an earlier kernel).  Every wait (mbarrier or flag) is bounded; on expiry the CTA reports
 // CATS_ERR_TIMEOUT, lets its copies land, frees its TMEM and returns.
-#include <cstdlib>
-
 #include "cats_kernels.cuh"
 
 namespace cats {
