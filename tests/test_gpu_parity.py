@@ -214,7 +214,7 @@ ATTN_CASES = [
     # 32 heads, five and seven query tiles: two tiles per CTA with a ragged last group; 49 nodes: the smallest such tree
     ("rand77_P300_h32", gen.tree_random(77, 2), 300, 32, 128), ("rand100_P63_h32", gen.tree_random(100, 4), 63, 32, 128),
     ("rand49_P200_h32", gen.tree_random(49, 6), 200, 32, 128), ("rand48_P200_h32", gen.tree_random(48, 6), 200, 32, 128),
-    ("rand128_P3968_h32", gen.tree_random(128, 9), 3968, 32, 128), ("rand128_P3969_h32", gen.tree_random(128, 9), 3969, 32, 128),
+    ("rand128_P896_h32", gen.tree_random(128, 9), 896, 32, 128), ("rand128_P897_h32", gen.tree_random(128, 9), 897, 32, 128),
     # 40 heads: clusters of three CTAs (row blocks of 44, 44 and 40 query rows), and a 17-node tree on them
     ("rand128_P2048_h40", gen.tree_random(128, 11), 2048, 40, 128), ("rand17_P700_h40", gen.tree_random(17, 12), 700, 40, 128),
 ]
