@@ -133,6 +133,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     // the first block can be requested before the previous kernel has finished if it lies in the prefix
     const bool early = (c_begin + p.blk <= p.P);
     if (early) load_kv(0, 0);
+    // with a second buffer and a second block inside the prefix, that one too
+    const bool early2 = early && nb > 1 && p.kv_area >= 4 * p.blk * ROWB && c_begin + 2 * p.blk <= p.P;
+    if (early2) load_kv(1, 1);
     if (p.csize > 1) {
         // the barrier the cluster's pushed partials complete on; visible to the peers before anybody can send
         if (threadIdx.x == 0) {
@@ -170,7 +173,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 
     for (int b = 0; b < nb; ++b) {
         if (b + 1 < nb) {
-            load_kv(b + 1, (b + 1) & 1);
+            if (!(b == 0 && early2)) load_kv(b + 1, (b + 1) & 1);
             cp_async_commit();
             cp_async_wait<1>();
         } else {
