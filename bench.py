@@ -154,6 +154,65 @@ def time_steps(fn, steps, warmup, stream):
 # our arm
 # --------------------------------------------------------------------------------------------------
 
+def bench_attention(cats, dev):
+    """Config 5: cats_tree_attention alone, 32 heads x 128, trees chain-16 / heap-64 / random-128, prefixes 256..16384.
+    K/V sets rotate (8 sets up to prefix 4096, 2 above) so that consecutive launches read different memory."""
+    nh, hd = 32, 128
+    D = nh * hd
+    out = {}
+    for P in (256, 1024, 4096, 16384):
+        n_sets = 8 if P <= 4096 else 2
+        S_max = P + 128
+        ks = [gen.normal_bf16((S_max, D), 1.0, dev, "cfg5", P, i, "k") for i in range(n_sets)]
+        vs = [gen.normal_bf16((S_max, D), 1.0, dev, "cfg5", P, i, "v") for i in range(n_sets)]
+        for name, parent in (("chain16", gen.tree_chain(16)), ("heap64", gen.tree_heap(64)), ("rand128", gen.tree_random(128, 5))):
+            T = len(parent)
+            q = gen.normal_bf16((T, nh, hd), 1.0, dev, "cfg5", P, name, "q")
+            mask = torch.zeros((T, 2), dtype=torch.int64, device=dev)
+            pos = torch.zeros(T, dtype=torch.int32, device=dev)
+            st = cats.new_status(dev)
+            cats.cats_build_tree_mask(torch.from_numpy(parent).to(dev), P, mask, pos, None, st)
+            o = torch.zeros((T, nh, hd), dtype=torch.bfloat16, device=dev)
+            cfg = cats.model_cfg(gen.ModelShape(hidden=D, n_heads=nh, head_dim=hd, ffn=64, vocab=128, n_layers=1), S_max)
+            ws = cats.new_workspace(cfg, T, P)
+            scale = 1.0 / float(np.sqrt(hd))
+
+            def run(i):
+                cats.cats_tree_attention(q, ks[i % n_sets], vs[i % n_sets], mask, T, P, nh, hd, D, scale, o, ws, st)
+            for i in range(4):
+                run(i)
+            torch.cuda.synchronize()
+            reps = 4 * n_sets
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(reps):
+                run(i)
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / reps * 1e3
+            b = roofline.attention_bytes(nh, hd, P, T)
+            out["P%d_%s" % (P, name)] = {"us": us, "gbs": b / us / 1e3, "status": int(st.item())}
+    return out
+
+
+def bench_13b(cats, dev, graph_of, time_steps, stream):
+    """Config 4: 40-layer 13B-shaped forward + LM head, prefix 2048, 64-node tree [6,3,2,2,1,1], graph replay."""
+    shape = gen.LLAMA_13B
+    P, T = 2048, 64
+    model = cats.pack_model(make_device_model(shape, "bench13b", dev), free_source=True)
+    torch.cuda.empty_cache()
+    kc, vc = gen.make_kv_prefix(shape, shape.n_layers, P + 128, P, "bench13b", device=dev)
+    parent = gen.tree_branching([6, 3, 2, 2, 1, 1], T)
+    tokens = gen.uniform_tokens(T, shape.vocab, "bench13b", T)
+    fwd = cats.VerifyForward(shape, model, kc, vc, T, P, want_logits=False, compact=True)
+    d_parent, d_tokens = torch.from_numpy(parent).to(dev), torch.from_numpy(tokens).to(dev)
+    g = graph_of(fwd, d_parent, d_tokens)
+    sec = time_steps(g.replay, 5, 3, stream) / 5
+    b = roofline.forward_bytes(shape, P, T)
+    return {"tree_nodes": T, "prefix_len": P, "ms": sec * 1e3, "tok_s": T / sec, "gbs": b / sec / 1e9,
+            "status": int(fwd.status.item())}
+
+
 def run_ours(args, rank, world, local_rank):
     from paper_2605_11186_b200 import binding as cats
     dev = torch.device("cuda", local_rank)
@@ -260,6 +319,16 @@ def run_ours(args, rank, world, local_rank):
         b1 = roofline.forward_bytes(shape, PREFIX, 1)
         widening["one_token_pass"] = {"tree_nodes": 1, "ms": r["sec_per_step"] * 1e3, "gbs": b1 / r["sec_per_step"] / 1e9}
 
+    # the other configurations of the workload table, reported beside the headline (rank 0, with the sweep):
+    # config 5, tree attention alone over prefixes 256..16384 with rotating K/V sets (so that short prefixes do not
+    # simply sit in L2), and config 4, the 40-layer 13B-shaped forward at prefix 2048
+    other = {}
+    if rank == 0 and not args.no_sweep and world == 1:
+        other["cfg5_attention"] = bench_attention(cats, dev)
+        del fwd
+        torch.cuda.empty_cache()
+        other["cfg4_13b"] = bench_13b(cats, dev, graph_of, time_steps, stream)
+
     sec_step, sec_e2e = max_over_ranks([main["sec_per_step"], e2e_sec / args.steps], dev)
     if rank != 0:
         return None
@@ -291,6 +360,7 @@ def run_ours(args, rank, world, local_rank):
         "breakdown_ms": {k: v * 1e3 for k, v in main["breakdown"].items()},
         "sweep": sweep,
         "widening": widening,
+        "other_configs": other,
     }
     return out
 
