@@ -84,7 +84,7 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
     return v;
 }
 
-template <int HD>
+template <int HD, bool K32>
 __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) {
     extern __shared__ __align__(128) uint8_t sm[];
     constexpr int ROWB = HD * 2;                 // bytes per tile row
@@ -195,6 +195,77 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
             // 16 rows of the slice at a time: S = Q K^T (16 x 16), mask, online softmax, O += P V
             for (int sub = 0; sub < R; sub += 16) {
                 if (cbase + sub >= c_end) break;
+                if (K32 && sub + 32 <= R && cbase + sub + 32 <= min(p.P, c_end)) {
+                    // 32 prefix rows at once (all visible): the softmax bookkeeping is paid once for twice the keys and
+                    // the four score tiles are four independent chains of MMAs
+                    float s[4][4];
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+                        const int r = rbase + sub + (lane & 7) + ((lane >> 4) << 3), ch = ks * 2 + ((lane >> 3) & 1);
+                        ldmatrix_x4(smem_u32(ks_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
+                        ldmatrix_x4(smem_u32(ks_s + tile_off<HD>(r + 16, ch)), c0, c1, c2, c3);
+                        mma_bf16_16816(s[0], qf[ks], b0, b1);
+                        mma_bf16_16816(s[1], qf[ks], b2, b3);
+                        mma_bf16_16816(s[2], qf[ks], c0, c1);
+                        mma_bf16_16816(s[3], qf[ks], c2, c3);
+                    }
+                    float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) s[n][e] *= p.scale_log2;
+                        mx_a = fmaxf(mx_a, fmaxf(s[n][0], s[n][1]));
+                        mx_b = fmaxf(mx_b, fmaxf(s[n][2], s[n][3]));
+                    }
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
+                    const float mn_a = fmaxf(m_run[0], mx_a), mn_b = fmaxf(m_run[1], mx_b);   // finite: prefix rows are visible
+                    const float corr_a = exp2f(m_run[0] - mn_a), corr_b = exp2f(m_run[1] - mn_b);
+                    m_run[0] = mn_a; m_run[1] = mn_b;
+                    float la = 0.f, lb = 0.f;
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) {
+                        s[n][0] = exp2f(s[n][0] - mn_a); s[n][1] = exp2f(s[n][1] - mn_a);
+                        s[n][2] = exp2f(s[n][2] - mn_b); s[n][3] = exp2f(s[n][3] - mn_b);
+                        la += s[n][0] + s[n][1];
+                        lb += s[n][2] + s[n][3];
+                    }
+                    l_run[0] = l_run[0] * corr_a + la;
+                    l_run[1] = l_run[1] * corr_b + lb;
+                    if (__any_sync(0xffffffffu, corr_a != 1.f || corr_b != 1.f)) {
+#pragma unroll
+                        for (int j = 0; j < NT; ++j) { o[j][0] *= corr_a; o[j][1] *= corr_a; o[j][2] *= corr_b; o[j][3] *= corr_b; }
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {            // the two 16-key halves of the P V product
+                        uint32_t pa[4], pl[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float x0 = s[2 * kk + (e >> 1)][(e & 1) * 2], x1 = s[2 * kk + (e >> 1)][(e & 1) * 2 + 1];
+                            const float h0 = bf16_bits_to_float(float_to_bf16_bits(x0));
+                            const float h1 = bf16_bits_to_float(float_to_bf16_bits(x1));
+                            pa[e] = pack_bf16x2(h0, h1);
+                            pl[e] = pack_bf16x2(x0 - h0, x1 - h1);
+                        }
+#pragma unroll
+                        for (int j = 0; j < NT; j += 2) {
+                            uint32_t b0, b1, b2, b3;
+                            const int r = rbase + sub + kk * 16 + (lane & 15), ch = j + (lane >> 4);
+                            ldmatrix_x4_trans(smem_u32(vs_s + tile_off<HD>(r, ch)), b0, b1, b2, b3);
+                            mma_bf16_16816(o[j], pa, b0, b1);
+                            mma_bf16_16816(o[j], pl, b0, b1);
+                            mma_bf16_16816(o[j + 1], pa, b2, b3);
+                            mma_bf16_16816(o[j + 1], pl, b2, b3);
+                        }
+                    }
+                    sub += 16;      // the loop adds the other 16
+                    continue;
+                }
                 // two accumulator pairs (even and odd k-steps): the chain of dependent MMAs is half as long
                 float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
                 float t0[4] = {0.f, 0.f, 0.f, 0.f}, t1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -487,8 +558,10 @@ static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t sme
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -538,8 +611,13 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     size_t smem = qbytes + kv + (size_t)tpad * 16 + recv;
     cudaError_t e;
     dim3 grid(p.qsplit > 0 ? p.qsplit : p.cluster * p.n_splits, p.nh);
-    if (p.hd == 128) e = launch_cluster(k_tree_attn<128>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
-    else e = launch_cluster(k_tree_attn<64>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
+    // a warp whose slice of a block has 32 rows or more takes prefix rows 32 at a time; the variant is compiled apart so
+    // that the 16-row kernel keeps its register allocation
+    const bool k32 = d.blk / d.kvg >= 32 && d.P >= 32;
+    if (p.hd == 128) e = k32 ? launch_cluster(k_tree_attn<128, true>, grid, dim3(kAttnThreads), smem, p.cluster, st, d)
+                             : launch_cluster(k_tree_attn<128, false>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
+    else e = k32 ? launch_cluster(k_tree_attn<64, true>, grid, dim3(kAttnThreads), smem, p.cluster, st, d)
+                 : launch_cluster(k_tree_attn<64, false>, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
