@@ -460,6 +460,329 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
     if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The same attention on the 5th-generation tensor cores (head_dim 128).
+//
+// One CTA per (head, share of the cache rows).  Q (128 rows, zero beyond T) and the blocks of K and V sit in shared
+// memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of 128-byte rows with the
+// 128-byte swizzle.  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache row) and as the MN-major
+// operand of O += P V (row = K index).  S lives in tensor memory, one query row per lane: thread r of warps 0-3 owns
+// row r, so the row maximum and sum are thread-local.  The probabilities go back to tensor memory as two bf16
+// operands hi + lo (hi over the columns S occupied) and enter P V as the A operand from tensor memory; O accumulates
+// in tensor memory and is rescaled (load, multiply, store) only by warps in which a running maximum moved.  The
+// partial (m, l, O) of the CTA is then merged across the cluster exactly as in the kernel above.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kTcCols = 512;          // tensor-memory columns: S / P_hi [0,256), P_lo [256,384), O [384,512)
+
+// byte offset of 16-byte chunk ch (0..15) of row r in a [2 halves][rows][128 B] tile with the 128-byte swizzle
+__device__ __forceinline__ uint32_t tc_off(int r, int ch, int rows) {
+    return (uint32_t)((ch >> 3) * rows * 128 + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ bool tc_visible(int col, int P, int c_end, uint64_t m0, uint64_t m1) {
+    if (col >= c_end) return false;
+    if (col < P) return true;
+    const int j = col - P;
+    return (((j < 64) ? m0 : m1) >> (j & 63)) & 1ull;
+}
+
+__global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn_tc(const AttnDev p) {
+    extern __shared__ __align__(128) uint8_t sm_raw[];
+    constexpr int HD = 128, REC = HD + 4;
+    uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
+    const int Tpad = p.n_mt * 16;
+    uint8_t* q_s = sm;                                                           // [2][128][128 B]
+    uint8_t* kv_s = q_s + 128 * 256;                                             // K and V blocks
+    uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + p.kv_area);           // [Tpad][2]
+    float* recv = reinterpret_cast<float*>(mask_s + (size_t)Tpad * 2);          // [csize][rpr][REC]
+    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // a lone CTA receives nothing
+    uint64_t* bar_s = rbar + 1;
+    uint64_t* bar_o = rbar + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 3);
+    volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = (int)blockIdx.x, h = blockIdx.y;
+    const int S = p.P + p.Tk;
+    const int c_begin = min(S, split * p.rows_per_split);
+    const int c_end = min(S, c_begin + p.rows_per_split);
+    const int NB = p.blk;
+    const int nb = (c_end - c_begin + NB - 1) / NB;
+    const uint32_t half = (uint32_t)NB * 128u;                                   // bytes between the two head-dim halves
+
+    // part 0: rows below the prefix length only; 1: the others (zero beyond the share); 2: all
+    auto load_kv = [&](int b, int buf, int part) {
+        uint8_t* ks = kv_s + (size_t)buf * 2 * NB * 256;
+        uint8_t* vs = ks + (size_t)NB * 256;
+        const int r0 = c_begin + b * NB;
+        const int n16 = min(NB, (c_end - r0 + 15) & ~15);
+        for (int e = threadIdx.x; e < n16 * 16; e += kAttnThreads) {
+            const int r = e >> 4, ch = e & 15, row = r0 + r;
+            if (part == 0 && row >= p.P) continue;
+            if (part == 1 && row < p.P) continue;
+            const uint32_t off = tc_off(r, ch, NB);
+            if (row < c_end) {
+                const size_t gofs = (size_t)row * p.kv_stride + (size_t)h * HD + ch * 8;
+                cp_async16(ks + off, p.k + gofs);
+                cp_async16(vs + off, p.v + gofs);
+            } else {
+                *reinterpret_cast<uint4*>(ks + off) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(vs + off) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+
+    pdl_launch_dependents();
+    if (nb > 0) load_kv(0, 0, 0);                       // prefix rows do not depend on the previous kernel
+    if (warp == 7) {
+        tmem_alloc(tmem_slot, kTcCols);
+        tmem_relinquish();
+    }
+    if (threadIdx.x == 0) {
+        *wait_expired = 0;
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        if (p.csize > 1) {
+            const int rank_ = split % p.csize;
+            const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
+            mbar_init(rbar, 1);
+            mbar_fence_init();
+            mbar_expect_tx(rbar, (uint32_t)(r1 - r0) * REC * 4u * (uint32_t)p.csize);
+        } else {
+            mbar_fence_init();
+        }
+    }
+    if (p.csize > 1) cluster_sync_all();
+    pdl_wait();
+    for (int e = threadIdx.x; e < 128 * 16; e += kAttnThreads) {
+        const int r = e >> 4, ch = e & 15;
+        const uint32_t off = tc_off(r, ch, 128);
+        if (r < p.T) cp_async16(q_s + off, p.q + ((size_t)r * p.nh + h) * HD + ch * 8);
+        else *reinterpret_cast<uint4*>(q_s + off) = make_uint4(0, 0, 0, 0);
+    }
+    for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) {
+        uint64_t w = 0ull;
+        const int gr = e >> 1;
+        if (gr < p.T) w = p.mask[(size_t)(p.nodes != nullptr ? p.nodes[gr] : gr) * 2 + (e & 1)];
+        mask_s[e] = w;
+    }
+    if (nb > 0) load_kv(0, 0, 1);
+    cp_async_commit();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tbase = *tmem_slot;
+    const uint32_t tS = tbase, tPlo = tbase + 256, tO = tbase + 384;
+    const uint32_t q_u32 = smem_u32(q_s);
+
+    const int row = (warp & 3) * 32 + lane;                          // the query row (= TMEM lane) of a softmax thread
+    const bool sm_warp = warp < 4 && warp * 32 < Tpad;             // warps that own query rows
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    uint64_t mk0 = 0ull, mk1 = 0ull;
+    if (sm_warp && row < Tpad) { mk0 = mask_s[row * 2]; mk1 = mask_s[row * 2 + 1]; }
+    float m_run = -INFINITY, l_run = 0.f;
+    uint32_t ph = 0;
+
+    for (int b = 0; b < nb; ++b) {
+        const int buf = b & 1;
+        if (b + 1 < nb) {
+            load_kv(b + 1, (b + 1) & 1, 2);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the tiles are read by the tensor core
+        __syncthreads();
+        const int r0 = c_begin + b * NB;
+        const int n16 = min(NB, (c_end - r0 + 15) & ~15);
+        const uint32_t ks_u32 = smem_u32(kv_s + (size_t)buf * 2 * NB * 256), vs_u32 = ks_u32 + (uint32_t)NB * 256u;
+        if (threadIdx.x == 0) {
+            tc_fence_after_sync();
+            const uint32_t idesc = umma_idesc_bf16_m128(n16);
+#pragma unroll
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                const uint64_t da = umma_desc_sw128(q_u32 + (uint32_t)(ks >> 2) * (128u * 128u) + (uint32_t)(ks & 3) * 32u);
+                const uint64_t db = umma_desc_sw128(ks_u32 + (uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u);
+                umma_bf16(tS, da, db, idesc, ks > 0);
+            }
+            umma_commit(bar_s);
+        }
+        if (sm_warp) {
+            mbar_wait(bar_s, ph, wait_expired);
+            tc_fence_after_sync();
+            const int lim = min(p.P, c_end);
+            // pass 1: the row maximum
+            float mx = -INFINITY;
+            for (int c = 0; c < n16; c += 16) {
+                float v[16];
+                tmem_ld16(tS + lane_base + (uint32_t)c, v);
+                if (r0 + c + 16 <= lim) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) mx = fmaxf(mx, v[e] * p.scale_log2);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (tc_visible(r0 + c + e, p.P, c_end, mk0, mk1)) mx = fmaxf(mx, v[e] * p.scale_log2);
+                }
+            }
+            const float mn = fmaxf(m_run, mx);
+            const float ref = (mn == -INFINITY) ? 0.f : mn;
+            const float corr = exp2f(m_run - ref);
+            m_run = mn;
+            // O of the earlier blocks follows the maximum (their P V products have completed)
+            if (b > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+                for (int c = 0; c < HD; c += 16) {
+                    float v[16];
+                    tmem_ld16(tO + lane_base + (uint32_t)c, v);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] *= corr;
+                    tmem_st16(tO + lane_base + (uint32_t)c, v);
+                }
+            }
+            // pass 2: probabilities, their sum, and the two bf16 operands
+            float ls = 0.f;
+            for (int c = 0; c < n16; c += 16) {
+                float v[16];
+                tmem_ld16(tS + lane_base + (uint32_t)c, v);
+                const bool all_vis = r0 + c + 16 <= lim;
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int e = 0; e < 16; e += 2) {
+                    float x0 = exp2f(v[e] * p.scale_log2 - ref), x1 = exp2f(v[e + 1] * p.scale_log2 - ref);
+                    if (!all_vis) {
+                        if (!tc_visible(r0 + c + e, p.P, c_end, mk0, mk1)) x0 = 0.f;
+                        if (!tc_visible(r0 + c + e + 1, p.P, c_end, mk0, mk1)) x1 = 0.f;
+                    }
+                    ls += x0 + x1;
+                    const float h0 = bf16_bits_to_float(float_to_bf16_bits(x0));
+                    const float h1 = bf16_bits_to_float(float_to_bf16_bits(x1));
+                    hi[e >> 1] = pack_bf16x2(h0, h1);
+                    lo[e >> 1] = pack_bf16x2(x0 - h0, x1 - h1);
+                }
+                tmem_st8(tS + lane_base + (uint32_t)(c >> 1), hi);
+                tmem_st8(tPlo + lane_base + (uint32_t)(c >> 1), lo);
+            }
+            l_run = l_run * corr + ls;
+            tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            tc_fence_after_sync();
+            const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
+            for (int kk = 0; kk < n16 / 16; ++kk)
+                umma_bf16_ts(tO, tS + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, b > 0 || kk > 0);
+            for (int kk = 0; kk < n16 / 16; ++kk)
+                umma_bf16_ts(tO, tPlo + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, true);
+            umma_commit(bar_o);
+        }
+        // the block's buffers and the S / P columns are free once its P V product has completed
+        mbar_wait(bar_o, ph, wait_expired);
+        tc_fence_after_sync();
+        ph ^= 1u;
+    }
+
+    // ---- deposit the CTA's partial (m, l, O), then the cluster merge ----
+    cp_async_wait<0>();                                  // a CTA without rows still has its Q copy in flight
+    __syncthreads();
+    float* loc = reinterpret_cast<float*>(kv_s);        // [Tpad][REC], aliases the K/V buffers
+    if (sm_warp) {
+        float* wo = loc + (size_t)row * REC;
+        for (int c = 0; c < HD; c += 16) {
+            float v[16];
+            if (nb > 0) {
+                tmem_ld16(tO + lane_base + (uint32_t)c, v);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = 0.f;
+            }
+            if (row < Tpad) {
+#pragma unroll
+                for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(wo + c + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+            }
+        }
+        if (row < Tpad) *reinterpret_cast<float2*>(wo + HD) = make_float2(m_run, l_run);
+    }
+    tc_fence_before_sync();
+    const int csize = p.csize, rpr = p.rpr;
+    const int rank = split % csize, outer = split / csize;
+    const int n_parts = csize;
+    const float* src_parts = loc;
+    int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
+    if (csize > 1) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the deposit is read by bulk copies
+        __syncthreads();
+        if (warp == 7) { tc_fence_after_sync(); tmem_dealloc(tbase, kTcCols); }
+        const int pi = lane * 8 + warp;                 // senders spread over the warps
+        if (lane < 4 && pi < n_parts) {
+            const int dest = pi;
+            const int r0 = min(Tpad, dest * rpr), r1 = min(Tpad, r0 + rpr);
+            if (r1 > r0) {
+                const uint32_t bytes = (uint32_t)(r1 - r0) * REC * 4;
+                const uint32_t src = smem_u32(loc + (size_t)r0 * REC);
+                const uint32_t dst_local = smem_u32(recv + ((size_t)rank * rpr) * REC);
+                const uint32_t dst = cluster_map(dst_local, dest), bar = cluster_map(smem_u32(rbar), dest);
+                asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(dst), "r"(src), "r"(bytes), "r"(bar) : "memory");
+            }
+        }
+        row0 = min(Tpad, rank * rpr);
+        n_my = min(Tpad, row0 + rpr) - row0;
+        if (n_my > 0 && !mbar_wait(rbar, 0, wait_expired)) {
+            if (threadIdx.x == 0) report(p.d_status, CATS_ERR_TIMEOUT);
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        src_parts = recv;
+        part_stride = rpr * REC;
+    } else {
+        __syncthreads();
+        if (warp == 7) { tc_fence_after_sync(); tmem_dealloc(tbase, kTcCols); }
+    }
+    if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
+    for (int rl = warp; rl < n_my; rl += 8) {
+        const int grow = row0 + rl;                    // global query row
+        if (grow >= p.T) break;
+        float mp = -INFINITY, lp = 0.f;
+        if (lane < n_parts) {
+            const float* my_rec = src_parts + (size_t)lane * part_stride + (size_t)(csize > 1 ? rl : grow) * REC;
+            const float2 ml = *reinterpret_cast<const float2*>(my_rec + HD);
+            mp = ml.x; lp = ml.y;
+        }
+        float M = mp;
+#pragma unroll
+        for (int ofs = 16; ofs > 0; ofs >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, ofs));
+        const float ref = (M == -INFINITY) ? 0.f : M;
+        const float wp = exp2f(mp - ref);
+        float L = lp * wp;
+#pragma unroll
+        for (int ofs = 16; ofs > 0; ofs >>= 1) L += __shfl_xor_sync(0xffffffffu, L, ofs);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* base = src_parts + (size_t)(csize > 1 ? rl : grow) * REC + lane * 4;
+        for (int pp = 0; pp < n_parts; ++pp) {                 // partials in a fixed order
+            const float w = __shfl_sync(0xffffffffu, wp, pp);
+            if (w != 0.f) {
+                const float4 v = *reinterpret_cast<const float4*>(base + (size_t)pp * part_stride);
+                acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+            }
+        }
+        if (p.n_outer == 1) {
+            const float inv = 1.f / L;
+            uint2 pk = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+            uint8_t* ob = reinterpret_cast<uint8_t*>(p.out);
+            const int col = lane * 4;
+            size_t off = p.out_npad > 0 ? packed_act_offset(grow, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2
+                                        : (((size_t)grow * p.nh + h) * HD + col) * 2;
+            *reinterpret_cast<uint2*>(ob + off) = pk;
+        } else {
+            const size_t gbase = ((size_t)h * p.n_outer + outer) * Tpad + grow;
+            *reinterpret_cast<float4*>(p.part_o + gbase * HD + lane * 4) = acc;
+            if (lane == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
+        }
+    }
+    // nobody leaves while a peer's copy may still be reading this CTA's deposit
+    if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
 __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                       int n_splits, int Tpad, int nh, int hd, uint16_t* __restrict__ out,
@@ -488,6 +811,11 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
 
 // Chooses the cluster size (CTAs per head that share one merge through distributed shared memory) and, for long
 // prefixes with few heads, the number of clusters per head.  Returns the bytes of workspace the outer merge needs.
+static bool attn_tc_enabled() {
+    static const bool on = [] { const char* e = getenv("CATS_ATTN_TC"); return e != nullptr && e[0] == '1'; }();
+    return on;
+}
+
 size_t attn_plan(AttnProblem& p) {
     const int S = p.prefix_len + (p.T_tree > 0 ? p.T_tree : p.T);
     const int units16 = (S + 15) / 16;
@@ -509,8 +837,9 @@ size_t attn_plan(AttnProblem& p) {
     // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
     p.qsplit = 0;
     p.mt_per_cta = 0;
+    p.use_tc = (p.hd == 128 && attn_tc_enabled()) ? 1 : 0;
     const int n_mt = tpad / 16;
-    if (n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
+    if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
         int mpc = 1, groups = n_mt;
         if (p.nh * groups > 148) { mpc = 2; groups = (n_mt + 1) / 2; }
         if (p.nh * groups <= 148 && p.nh * groups >= 96) {
@@ -555,6 +884,47 @@ static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t sme
     return cudaLaunchKernelEx(&cfg, kernel, d);
 }
 
+static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    AttnDev d;
+    d.q = (const uint16_t*)p.q; d.k = (const uint16_t*)p.k; d.v = (const uint16_t*)p.v;
+    d.mask = p.mask;
+    d.nodes = p.nodes;
+    d.Tk = p.T_tree > 0 ? p.T_tree : p.T;
+    d.T = p.T; d.P = p.prefix_len; d.nh = p.nh;
+    d.n_mt = (p.T + 15) / 16;
+    d.kvg = 1;
+    d.qsplit = 0;
+    d.csize = p.cluster; d.n_outer = p.n_splits; d.rows_per_split = p.rows_per_split;
+    d.kv_stride = p.kv_stride;
+    d.scale_log2 = p.scale * 1.4426950408889634f;
+    d.out = (uint16_t*)p.out;
+    d.out_npad = p.out_packed_npad;
+    d.part_o = p.part_o; d.part_ml = p.part_ml;
+    d.d_status = p.d_status;
+    const int tpad = d.n_mt * 16, rec = p.hd + 4;
+    d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
+    const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
+    const size_t fixed = 1024 + 128 * 256 + (size_t)tpad * 16 + recv + 64;     // alignment slack, Q, masks, received partials, barriers
+    // rows per block of the streaming pipeline: two buffers of K and V (1024 bytes per row) in what is left
+    int nbs = (int)((227 * 1024 - fixed) / 1024) / 16 * 16;
+    if (nbs > 128) nbs = 128;
+    if ((size_t)4 * nbs * 256 < (size_t)tpad * rec * 4) return cudaErrorInvalidConfiguration;   // the deposit aliases the buffers
+    d.blk = p.rows_per_split <= 2 * nbs ? p.rows_per_split : nbs;     // a share of up to two blocks is taken as one
+    d.kv_area = 4 * nbs * 256;
+    const size_t smem = fixed + (size_t)d.kv_area;
+    dim3 grid(p.cluster * p.n_splits, p.nh);
+    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
+    if (e != cudaSuccess || p.n_splits == 1) return e;
+    return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
+                      p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
+}
+
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
@@ -565,6 +935,7 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
+    if (p.use_tc) return launch_tree_attention_tc(p, st);
     AttnDev d;
     d.q = (const uint16_t*)p.q; d.k = (const uint16_t*)p.k; d.v = (const uint16_t*)p.v;
     d.mask = p.mask;

@@ -146,6 +146,7 @@ struct AttnProblem {
     int rows_per_split; //   cache rows per CTA (multiple of 16)
     int qsplit;         //   > 0: CTAs per head that split the query tiles instead (every CTA reads all cache rows)
     int mt_per_cta;     //   query tiles per CTA in that case
+    int use_tc;         //   1: the tcgen05 kernel (head_dim 128)
     int32_t* d_status;
 };
 // Chooses the KV split; returns bytes of partial storage needed.
