@@ -55,6 +55,7 @@ struct AttnDev {
     int Tk;                 // tree rows in the cache after the prefix
     int rpr;                // query rows each CTA of a cluster merges (contiguous block)
     int qsplit;             // > 0: the CTAs of a head split the QUERY tiles (n_mt tiles each) and every CTA reads all rows
+    int stages;             // tcgen05 kernel: stages of the K/V ring
     int32_t* d_status;
     int T, P, nh, n_mt, kvg, csize, n_outer, rows_per_split, blk, kv_area;   // blk: cache rows per pipeline block (multiple of 16*kvg); kv_area: bytes of the K/V buffers
     long long kv_stride;
@@ -463,16 +464,25 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // ---------------------------------------------------------------------------------------------------
 // The same attention on the 5th-generation tensor cores (head_dim 128).
 //
-// One CTA per (head, share of the cache rows).  Q (128 rows, zero beyond T) and the blocks of K and V sit in shared
-// memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of 128-byte rows with the
-// 128-byte swizzle.  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache row) and as the MN-major
-// operand of O += P V (row = K index).  S lives in tensor memory, one query row per lane: thread r of warps 0-3 owns
-// row r, so the row maximum and sum are thread-local.  The probabilities go back to tensor memory as two bf16
-// operands hi + lo (hi over the columns S occupied) and enter P V as the A operand from tensor memory; O accumulates
-// in tensor memory and is rescaled (load, multiply, store) only by warps in which a running maximum moved.  The
-// partial (m, l, O) of the CTA is then merged across the cluster exactly as in the kernel above.
+// One CTA per (head, share of the cache rows), nine warps.  Q (128 rows, zero beyond T) and a ring of K/V blocks
+// sit in shared memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of
+// 128-byte rows with the 128-byte swizzle.  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache
+// row) and as the MN-major operand of O += P V (row = K index).  Warp 8 issues the MMAs: S(b+1) = Q K(b+1)^T is
+// issued before P(b) V(b), so the tensor core works on the next block while warps 0-7 take the softmax of this one.
+// S has two buffers in tensor memory, one query row per lane; warps w and w+4 share the 32 rows of lane quadrant
+// w and split the block's columns, so a row's maximum and sum need one exchange between two threads.  The
+// probabilities go back to tensor memory over the columns S occupied, as two bf16 operands hi + lo, and enter
+// P V as the A operand from tensor memory.  O accumulates in tensor memory and is rescaled (load, multiply, store)
+// only by warps in which a running maximum moved.  Warps 0-7 also refill the ring: cp.async into the stage the last
+// P V product released, completion counted on that stage's mbarrier.  The CTA's partial (m, l, O) is then merged
+// across the cluster exactly as in the kernel above.
 // ---------------------------------------------------------------------------------------------------
-constexpr int kTcCols = 512;          // tensor-memory columns: S / P_hi [0,256), P_lo [256,384), O [384,512)
+constexpr int kTcThreads = 288;       // warps 0-7: softmax and loads; warp 8: MMA issue, tensor-memory allocation
+constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
+constexpr int kTcSStride = 192;
+constexpr int kTcStream = 64;         // cache rows per block when a share is streamed
+constexpr int kTcOneShot = 192;       // a share of at most this many rows is one block
+constexpr int kTcMaxStages = 4;
 
 // byte offset of 16-byte chunk ch (0..15) of row r in a [2 halves][rows][128 B] tile with the 128-byte swizzle
 __device__ __forceinline__ uint32_t tc_off(int r, int ch, int rows) {
@@ -484,20 +494,51 @@ __device__ __forceinline__ bool tc_visible(int col, int P, int c_end, uint64_t m
     const int j = col - P;
     return (((j < 64) ? m0 : m1) >> (j & 63)) & 1ull;
 }
+// 16 bytes global -> shared, or 16 zero bytes when !valid (the source address is not read then)
+__device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, bool valid) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(valid ? 16u : 0u) : "memory");
+}
+// The mbarrier receives one arrival from this thread once all cp.async it has issued so far have landed.
+__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+// Completes the loads above; the values may be used only after the empty statements that tie them to this point.
+template <int N>
+__device__ __forceinline__ void tmem_wait_ld(float* v) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < N; ++i) asm volatile("" : "+f"(v[i]));
+}
+__device__ __forceinline__ void pair_barrier(int quadrant) {     // the two warps that share a lane quadrant
+    asm volatile("bar.sync %0, 64;" ::"r"(quadrant + 1) : "memory");
+}
 
-__global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn_tc(const AttnDev p) {
+__global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
-    constexpr int HD = 128, REC = HD + 4;
+    constexpr int HD = 128, REC = HD + 4, CPT = kTcOneShot / 2;    // CPT: most columns of S one thread holds
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
     const int Tpad = p.n_mt * 16;
     uint8_t* q_s = sm;                                                           // [2][128][128 B]
-    uint8_t* kv_s = q_s + 128 * 256;                                             // K and V blocks
-    uint64_t* mask_s = reinterpret_cast<uint64_t*>(kv_s + p.kv_area);           // [Tpad][2]
-    float* recv = reinterpret_cast<float*>(mask_s + (size_t)Tpad * 2);          // [csize][rpr][REC]
-    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // a lone CTA receives nothing
-    uint64_t* bar_s = rbar + 1;
-    uint64_t* bar_o = rbar + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 3);
+    uint8_t* kv_s = q_s + 128 * 256;                                             // ring of K and V blocks
+    float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][2][128] row maxima (by block parity), [2][128] row sums
+    float* recv = xch + 768;                                                     // [csize][rpr][REC]
+    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));
+    uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete
+    uint64_t* bar_o = rbar + 3;           //      P(b) V(b) complete
+    uint64_t* bar_p = rbar + 4;           //      P(b) written (256 arrivals)
+    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  block landed (256 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 5 + kTcMaxStages);
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -505,221 +546,263 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn_tc(const AttnDev 
     const int S = p.P + p.Tk;
     const int c_begin = min(S, split * p.rows_per_split);
     const int c_end = min(S, c_begin + p.rows_per_split);
-    const int NB = p.blk;
+    const int NB = p.blk;                                  // rows per block, a multiple of 32
+    const int NST = p.stages;                              // stages of the ring
     const int nb = (c_end - c_begin + NB - 1) / NB;
-    const uint32_t half = (uint32_t)NB * 128u;                                   // bytes between the two head-dim halves
+    const uint32_t half = (uint32_t)NB * 128u;             // bytes between the two head-dim halves of a block
+    const size_t stage_bytes = (size_t)NB * 512;           // K block, then V block
 
-    // part 0: rows below the prefix length only; 1: the others (zero beyond the share); 2: all
-    auto load_kv = [&](int b, int buf, int part) {
-        uint8_t* ks = kv_s + (size_t)buf * 2 * NB * 256;
+    // part 0: rows below the prefix length only; 1: the others (zeros beyond the share); 2: all
+    auto load_kv = [&](int b, int part) {
+        uint8_t* ks = kv_s + (size_t)(b % NST) * stage_bytes;
         uint8_t* vs = ks + (size_t)NB * 256;
         const int r0 = c_begin + b * NB;
         const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-        for (int e = threadIdx.x; e < n16 * 16; e += kAttnThreads) {
+        for (int e = threadIdx.x; e < n16 * 16; e += 256) {
             const int r = e >> 4, ch = e & 15, row = r0 + r;
             if (part == 0 && row >= p.P) continue;
             if (part == 1 && row < p.P) continue;
             const uint32_t off = tc_off(r, ch, NB);
-            if (row < c_end) {
-                const size_t gofs = (size_t)row * p.kv_stride + (size_t)h * HD + ch * 8;
-                cp_async16(ks + off, p.k + gofs);
-                cp_async16(vs + off, p.v + gofs);
-            } else {
-                *reinterpret_cast<uint4*>(ks + off) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(vs + off) = make_uint4(0, 0, 0, 0);
-            }
+            const bool valid = row < c_end;
+            const size_t gofs = valid ? (size_t)row * p.kv_stride + (size_t)h * HD + ch * 8 : 0;
+            cp_async16_zfill(ks + off, p.k + gofs, valid);
+            cp_async16_zfill(vs + off, p.v + gofs, valid);
         }
     };
 
     pdl_launch_dependents();
-    if (nb > 0) load_kv(0, 0, 0);                       // prefix rows do not depend on the previous kernel
-    if (warp == 7) {
+    if (warp == 8) {
         tmem_alloc(tmem_slot, kTcCols);
         tmem_relinquish();
-    }
-    if (threadIdx.x == 0) {
-        *wait_expired = 0;
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
-        if (p.csize > 1) {
-            const int rank_ = split % p.csize;
-            const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
-            mbar_init(rbar, 1);
-            mbar_fence_init();
-            mbar_expect_tx(rbar, (uint32_t)(r1 - r0) * REC * 4u * (uint32_t)p.csize);
-        } else {
-            mbar_fence_init();
+        if (lane == 0) {
+            *wait_expired = 0;
+            mbar_init(bar_s, 1);
+            mbar_init(bar_s + 1, 1);
+            mbar_init(bar_o, 1);
+            mbar_init(bar_p, 256);
+            for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 256);
+            if (p.csize > 1) {
+                const int rank_ = split % p.csize;
+                const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
+                mbar_init(rbar, 1);
+                mbar_fence_init();
+                mbar_expect_tx(rbar, (uint32_t)(r1 - r0) * REC * 4u * (uint32_t)p.csize);
+            } else {
+                mbar_fence_init();
+            }
         }
+    } else {
+        // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
+        for (int b = 0; b < NST && b < nb; ++b) load_kv(b, 0);
     }
-    if (p.csize > 1) cluster_sync_all();
-    pdl_wait();
-    for (int e = threadIdx.x; e < 128 * 16; e += kAttnThreads) {
-        const int r = e >> 4, ch = e & 15;
-        const uint32_t off = tc_off(r, ch, 128);
-        if (r < p.T) cp_async16(q_s + off, p.q + ((size_t)r * p.nh + h) * HD + ch * 8);
-        else *reinterpret_cast<uint4*>(q_s + off) = make_uint4(0, 0, 0, 0);
-    }
-    for (int e = threadIdx.x; e < Tpad * 2; e += kAttnThreads) {
-        uint64_t w = 0ull;
-        const int gr = e >> 1;
-        if (gr < p.T) w = p.mask[(size_t)(p.nodes != nullptr ? p.nodes[gr] : gr) * 2 + (e & 1)];
-        mask_s[e] = w;
-    }
-    if (nb > 0) load_kv(0, 0, 1);
-    cp_async_commit();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    if (p.csize > 1) cluster_sync_all();                   // every receiving barrier is armed before anybody can send
+    pdl_wait();
     const uint32_t tbase = *tmem_slot;
-    const uint32_t tS = tbase, tPlo = tbase + 256, tO = tbase + 384;
+    const uint32_t tO = tbase + 384;
     const uint32_t q_u32 = smem_u32(q_s);
 
-    const int row = (warp & 3) * 32 + lane;                          // the query row (= TMEM lane) of a softmax thread
-    const bool sm_warp = warp < 4 && warp * 32 < Tpad;             // warps that own query rows
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    uint64_t mk0 = 0ull, mk1 = 0ull;
-    if (sm_warp && row < Tpad) { mk0 = mask_s[row * 2]; mk1 = mask_s[row * 2 + 1]; }
-    float m_run = -INFINITY, l_run = 0.f;
-    uint32_t ph = 0;
-
-    for (int b = 0; b < nb; ++b) {
-        const int buf = b & 1;
-        if (b + 1 < nb) {
-            load_kv(b + 1, (b + 1) & 1, 2);
-            cp_async_commit();
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the tiles are read by the tensor core
-        __syncthreads();
-        const int r0 = c_begin + b * NB;
-        const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-        const uint32_t ks_u32 = smem_u32(kv_s + (size_t)buf * 2 * NB * 256), vs_u32 = ks_u32 + (uint32_t)NB * 256u;
-        if (threadIdx.x == 0) {
-            tc_fence_after_sync();
-            const uint32_t idesc = umma_idesc_bf16_m128(n16);
+    if (warp == 8) {
+        // ---- MMA issue: QK(0); then per block QK(b+1) ahead of PV(b) ----
+        if (lane == 0 && nb > 0) {
+            const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
+            auto issue_qk = [&](int b) {
+                const int r0 = c_begin + b * NB;
+                const int n16 = min(NB, (c_end - r0 + 15) & ~15);
+                const uint32_t ks_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes);
+                const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
+                const uint32_t idesc = umma_idesc_bf16_m128(n16);
 #pragma unroll
-            for (int ks = 0; ks < HD / 16; ++ks) {
-                const uint64_t da = umma_desc_sw128(q_u32 + (uint32_t)(ks >> 2) * (128u * 128u) + (uint32_t)(ks & 3) * 32u);
-                const uint64_t db = umma_desc_sw128(ks_u32 + (uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u);
-                umma_bf16(tS, da, db, idesc, ks > 0);
+                for (int ks = 0; ks < HD / 16; ++ks) {
+                    const uint64_t da = umma_desc_sw128(q_u32 + (uint32_t)(ks >> 2) * (128u * 128u) + (uint32_t)(ks & 3) * 32u);
+                    const uint64_t db = umma_desc_sw128(ks_u32 + (uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u);
+                    umma_bf16(tS, da, db, idesc, ks > 0);
+                }
+                umma_commit(bar_s + (b & 1));
+            };
+            bool ok = mbar_wait(bar_kv, 0, wait_expired);          // Q and block 0
+            if (ok) {
+                tc_fence_after_sync();
+                issue_qk(0);
             }
-            umma_commit(bar_s);
+            for (int b = 0; b < nb && ok; ++b) {
+                if (b + 1 < nb) {
+                    ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_qk(b + 1);
+                }
+                ok = mbar_wait(bar_p, (uint32_t)b & 1u, wait_expired);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const int r0 = c_begin + b * NB;
+                const int n16 = min(NB, (c_end - r0 + 15) & ~15);
+                const uint32_t vs_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes) + (uint32_t)NB * 256u;
+                const uint32_t tP = tbase + (uint32_t)(b & 1) * kTcSStride;
+                for (int kk = 0; kk < n16 / 16; ++kk)
+                    umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, b > 0 || kk > 0);
+                for (int kk = 0; kk < n16 / 16; ++kk)
+                    umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, true);
+                umma_commit(bar_o);
+            }
         }
-        if (sm_warp) {
-            mbar_wait(bar_s, ph, wait_expired);
+    } else {
+        // ---- warps 0-7: Q and the rows that depend on the previous kernel, then softmax and refills ----
+        for (int e = threadIdx.x; e < 128 * 16; e += 256) {
+            const int r = e >> 4, ch = e & 15;
+            const bool valid = r < p.T;
+            cp_async16_zfill(q_s + tc_off(r, ch, 128), p.q + (valid ? ((size_t)r * p.nh + h) * HD + ch * 8 : 0), valid);
+        }
+        for (int b = 0; b < NST && b < nb; ++b) {
+            load_kv(b, 1);
+            cp_async_arrive(bar_kv + b);
+        }
+        const int quad = warp & 3, hf = warp >> 2;
+        const int row = quad * 32 + lane;                       // the query row (= TMEM lane) of this thread
+        const bool act = quad * 32 < Tpad;                      // the warp owns query rows
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const int ncol = NB / 2, c0 = hf * ncol;                // this thread's columns of a block
+        uint64_t mk0 = 0ull, mk1 = 0ull;
+        if (row < p.T) {
+            const size_t node = p.nodes != nullptr ? p.nodes[row] : row;
+            mk0 = p.mask[node * 2];
+            mk1 = p.mask[node * 2 + 1];
+        }
+        float m_run = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int b = 0; b < nb; ++b) {
+            const int r0 = c_begin + b * NB;
+            const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
+            float v[CPT];
+            float corr = 1.f, ref = 0.f;
+            if (ok) ok = mbar_wait(bar_s + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
             tc_fence_after_sync();
-            const int lim = min(p.P, c_end);
-            // pass 1: the row maximum
-            float mx = -INFINITY;
-            for (int c = 0; c < n16; c += 16) {
-                float v[16];
-                tmem_ld16(tS + lane_base + (uint32_t)c, v);
-                if (r0 + c + 16 <= lim) {
+            if (act) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) mx = fmaxf(mx, v[e] * p.scale_log2);
+                for (int c = 0; c < CPT; c += 16)
+                    if (c < ncol) tmem_ld16_nowait(tS + lane_base + (uint32_t)(c0 + c), v + c);
+                tmem_wait_ld<CPT>(v);
+                const int lim = min(p.P, c_end);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < CPT; c += 16) {
+                    if (c < ncol) {
+                        const int g0 = r0 + c0 + c;
+                        if (g0 + 16 <= lim) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) { v[c + e] *= p.scale_log2; mx = fmaxf(mx, v[c + e]); }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) {
+                                v[c + e] = tc_visible(g0 + e, p.P, c_end, mk0, mk1) ? v[c + e] * p.scale_log2 : -INFINITY;
+                                mx = fmaxf(mx, v[c + e]);
+                            }
+                        }
+                    }
+                }
+                xch[((b & 1) * 2 + hf) * 128 + row] = mx;
+                pair_barrier(quad);                              // both halves are in registers; maxima exchanged
+                mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
+                const float mn = fmaxf(m_run, mx);
+                ref = (mn == -INFINITY) ? 0.f : mn;
+                corr = exp2f(m_run - ref);
+                m_run = mn;
+            }
+            if (b > 0) {
+                // P(b-1) V(b-1) has completed: O is stable, and the stage it read can be refilled
+                if (ok) ok = mbar_wait(bar_o, (uint32_t)(b - 1) & 1u, wait_expired);
+                tc_fence_after_sync();
+                if (b - 1 + NST < nb) {
+                    load_kv(b - 1 + NST, 2);
+                    cp_async_arrive(bar_kv + (b - 1) % NST);
+                }
+                if (act && __any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+                    for (int c = 0; c < HD / 2; c += 16) {
+                        float o[16];
+                        tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) o[e] *= corr;
+                        tmem_st16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
+                    }
+                }
+            }
+            if (act) {
+                float ls = 0.f;
+#pragma unroll
+                for (int c = 0; c < CPT; c += 16) {
+                    if (c < ncol) {
+                        uint32_t hi[8], lo[8];
+#pragma unroll
+                        for (int e = 0; e < 16; e += 2) {
+                            const float x0 = exp2f(v[c + e] - ref), x1 = exp2f(v[c + e + 1] - ref);
+                            ls += x0 + x1;
+                            const float h0 = bf16_bits_to_float(float_to_bf16_bits(x0));
+                            const float h1 = bf16_bits_to_float(float_to_bf16_bits(x1));
+                            hi[e >> 1] = pack_bf16x2(h0, h1);
+                            lo[e >> 1] = pack_bf16x2(x0 - h0, x1 - h1);
+                        }
+                        tmem_st8(tS + lane_base + (uint32_t)((c0 + c) >> 1), hi);
+                        tmem_st8(tS + lane_base + (uint32_t)(ncol + ((c0 + c) >> 1)), lo);
+                    }
+                }
+                l_run = l_run * corr + ls;
+                tmem_wait_st();
+            }
+            tc_fence_before_sync();
+            mbar_arrive(bar_p);
+        }
+        // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
+        if (nb > 0) {
+            if (ok) ok = mbar_wait(bar_o, (uint32_t)(nb - 1) & 1u, wait_expired);
+            tc_fence_after_sync();
+        }
+        cp_async_wait<0>();
+        asm volatile("bar.sync 5, 256;" ::: "memory");          // warps 0-7: every MMA and copy that used the ring is done
+        float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
+        if (act) {
+            float* xl = xch + 512;                              // [2][128]
+            xl[hf * 128 + row] = l_run;
+            float* wo = loc + (size_t)row * REC + hf * (HD / 2);
+#pragma unroll
+            for (int c = 0; c < HD / 2; c += 16) {
+                float o[16];
+                if (nb > 0) {
+                    tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
                 } else {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e)
-                        if (tc_visible(r0 + c + e, p.P, c_end, mk0, mk1)) mx = fmaxf(mx, v[e] * p.scale_log2);
+                    for (int e = 0; e < 16; ++e) o[e] = 0.f;
+                }
+                if (row < Tpad) {
+#pragma unroll
+                    for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(wo + c + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
                 }
             }
-            const float mn = fmaxf(m_run, mx);
-            const float ref = (mn == -INFINITY) ? 0.f : mn;
-            const float corr = exp2f(m_run - ref);
-            m_run = mn;
-            // O of the earlier blocks follows the maximum (their P V products have completed)
-            if (b > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
-                for (int c = 0; c < HD; c += 16) {
-                    float v[16];
-                    tmem_ld16(tO + lane_base + (uint32_t)c, v);
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) v[e] *= corr;
-                    tmem_st16(tO + lane_base + (uint32_t)c, v);
-                }
-            }
-            // pass 2: probabilities, their sum, and the two bf16 operands
-            float ls = 0.f;
-            for (int c = 0; c < n16; c += 16) {
-                float v[16];
-                tmem_ld16(tS + lane_base + (uint32_t)c, v);
-                const bool all_vis = r0 + c + 16 <= lim;
-                uint32_t hi[8], lo[8];
-#pragma unroll
-                for (int e = 0; e < 16; e += 2) {
-                    float x0 = exp2f(v[e] * p.scale_log2 - ref), x1 = exp2f(v[e + 1] * p.scale_log2 - ref);
-                    if (!all_vis) {
-                        if (!tc_visible(r0 + c + e, p.P, c_end, mk0, mk1)) x0 = 0.f;
-                        if (!tc_visible(r0 + c + e + 1, p.P, c_end, mk0, mk1)) x1 = 0.f;
-                    }
-                    ls += x0 + x1;
-                    const float h0 = bf16_bits_to_float(float_to_bf16_bits(x0));
-                    const float h1 = bf16_bits_to_float(float_to_bf16_bits(x1));
-                    hi[e >> 1] = pack_bf16x2(h0, h1);
-                    lo[e >> 1] = pack_bf16x2(x0 - h0, x1 - h1);
-                }
-                tmem_st8(tS + lane_base + (uint32_t)(c >> 1), hi);
-                tmem_st8(tPlo + lane_base + (uint32_t)(c >> 1), lo);
-            }
-            l_run = l_run * corr + ls;
-            tmem_wait_st();
+            pair_barrier(quad);
+            if (hf == 0 && row < Tpad) *reinterpret_cast<float2*>(loc + (size_t)row * REC + HD) = make_float2(m_run, l_run + xl[128 + row]);
         }
-        tc_fence_before_sync();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            tc_fence_after_sync();
-            const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
-            for (int kk = 0; kk < n16 / 16; ++kk)
-                umma_bf16_ts(tO, tS + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, b > 0 || kk > 0);
-            for (int kk = 0; kk < n16 / 16; ++kk)
-                umma_bf16_ts(tO, tPlo + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, true);
-            umma_commit(bar_o);
-        }
-        // the block's buffers and the S / P columns are free once its P V product has completed
-        mbar_wait(bar_o, ph, wait_expired);
-        tc_fence_after_sync();
-        ph ^= 1u;
-    }
-
-    // ---- deposit the CTA's partial (m, l, O), then the cluster merge ----
-    cp_async_wait<0>();                                  // a CTA without rows still has its Q copy in flight
-    __syncthreads();
-    float* loc = reinterpret_cast<float*>(kv_s);        // [Tpad][REC], aliases the K/V buffers
-    if (sm_warp) {
-        float* wo = loc + (size_t)row * REC;
-        for (int c = 0; c < HD; c += 16) {
-            float v[16];
-            if (nb > 0) {
-                tmem_ld16(tO + lane_base + (uint32_t)c, v);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = 0.f;
-            }
-            if (row < Tpad) {
-#pragma unroll
-                for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(wo + c + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-            }
-        }
-        if (row < Tpad) *reinterpret_cast<float2*>(wo + HD) = make_float2(m_run, l_run);
     }
     tc_fence_before_sync();
     const int csize = p.csize, rpr = p.rpr;
     const int rank = split % csize, outer = split / csize;
     const int n_parts = csize;
-    const float* src_parts = loc;
+    const float* src_parts = reinterpret_cast<const float*>(kv_s);
+    const float* loc_c = src_parts;
     int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
     if (csize > 1) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the deposit is read by bulk copies
         __syncthreads();
-        if (warp == 7) { tc_fence_after_sync(); tmem_dealloc(tbase, kTcCols); }
-        const int pi = lane * 8 + warp;                 // senders spread over the warps
-        if (lane < 4 && pi < n_parts) {
-            const int dest = pi;
+        if (warp == 8) {
+            tc_fence_after_sync();
+            tmem_dealloc(tbase, kTcCols);
+        } else if (lane == 0 && warp < n_parts) {       // one sender per destination, spread over the warps
+            const int dest = warp;
             const int r0 = min(Tpad, dest * rpr), r1 = min(Tpad, r0 + rpr);
             if (r1 > r0) {
                 const uint32_t bytes = (uint32_t)(r1 - r0) * REC * 4;
-                const uint32_t src = smem_u32(loc + (size_t)r0 * REC);
+                const uint32_t src = smem_u32(loc_c + (size_t)r0 * REC);
                 const uint32_t dst_local = smem_u32(recv + ((size_t)rank * rpr) * REC);
                 const uint32_t dst = cluster_map(dst_local, dest), bar = cluster_map(smem_u32(rbar), dest);
                 asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -728,18 +811,19 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn_tc(const AttnDev 
         }
         row0 = min(Tpad, rank * rpr);
         n_my = min(Tpad, row0 + rpr) - row0;
-        if (n_my > 0 && !mbar_wait(rbar, 0, wait_expired)) {
-            if (threadIdx.x == 0) report(p.d_status, CATS_ERR_TIMEOUT);
-        }
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (n_my > 0) mbar_wait(rbar, 0, wait_expired);
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // this CTA holds everything it needs
         src_parts = recv;
         part_stride = rpr * REC;
     } else {
         __syncthreads();
-        if (warp == 7) { tc_fence_after_sync(); tmem_dealloc(tbase, kTcCols); }
+        if (warp == 8) {
+            tc_fence_after_sync();
+            tmem_dealloc(tbase, kTcCols);
+        }
     }
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
-    for (int rl = warp; rl < n_my; rl += 8) {
+    for (int rl = warp; rl < n_my && warp < 8; rl += 8) {
         const int grow = row0 + rl;                    // global query row
         if (grow >= p.T) break;
         float mp = -INFINITY, lp = 0.f;
@@ -910,16 +994,23 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
-    const size_t fixed = 1024 + 128 * 256 + (size_t)tpad * 16 + recv + 64;     // alignment slack, Q, masks, received partials, barriers
-    // rows per block of the streaming pipeline: two buffers of K and V (1024 bytes per row) in what is left
-    int nbs = (int)((227 * 1024 - fixed) / 1024) / 16 * 16;
-    if (nbs > 128) nbs = 128;
-    if ((size_t)4 * nbs * 256 < (size_t)tpad * rec * 4) return cudaErrorInvalidConfiguration;   // the deposit aliases the buffers
-    d.blk = p.rows_per_split <= 2 * nbs ? p.rows_per_split : nbs;     // a share of up to two blocks is taken as one
-    d.kv_area = 4 * nbs * 256;
+    const size_t fixed = 1024 + 128 * 256 + 3072 + recv + 128;     // alignment slack, Q, pair exchange, received partials, barriers
+    // the ring: stages of 64 rows of K and V (32 KB each), as many as fit, at least three (which also hold a one-block share)
+    int stages = (int)((227 * 1024 - fixed) / (kTcStream * 512));
+    if (stages > kTcMaxStages) stages = kTcMaxStages;
+    if (stages < 3) return cudaErrorInvalidConfiguration;
+    d.kv_area = stages * kTcStream * 512;
+    if ((size_t)d.kv_area < (size_t)tpad * rec * 4) return cudaErrorInvalidConfiguration;   // the deposit aliases the ring
+    if (p.rows_per_split <= kTcOneShot) {
+        d.blk = (p.rows_per_split + 31) / 32 * 32;
+        d.stages = 1;
+    } else {
+        d.blk = kTcStream;
+        d.stages = stages;
+    }
     const size_t smem = fixed + (size_t)d.kv_area;
     dim3 grid(p.cluster * p.n_splits, p.nh);
-    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kAttnThreads), smem, p.cluster, st, d);
+    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kTcThreads), smem, p.cluster, st, d);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
