@@ -477,6 +477,15 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // P V product released, completion counted on that stage's mbarrier.  The CTA's partial (m, l, O) is then merged
 // across the cluster exactly as in the kernel above.
 // ---------------------------------------------------------------------------------------------------
+#ifdef CATS_TC_TRACE
+__device__ long long g_tc_trace[1024];
+#define TCT(slot) do { if (blockIdx.x == TC_TRACE_X && blockIdx.y == 0 && (slot) < 1024) g_tc_trace[(slot)] = clock64(); } while (0)
+#ifndef TC_TRACE_X
+#define TC_TRACE_X 0
+#endif
+#else
+#define TCT(slot) do { } while (0)
+#endif
 constexpr int kTcThreads = 288;       // warps 0-7: softmax and loads; warp 8: MMA issue, tensor-memory allocation
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
@@ -520,6 +529,32 @@ __device__ __forceinline__ void tmem_wait_ld(float* v) {
 #pragma unroll
     for (int i = 0; i < N; ++i) asm volatile("" : "+f"(v[i]));
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {      // two roundings in one instruction
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// Bit e set iff cache row g0 + e is visible to the query whose ancestor mask is (m0, m1): prefix rows always, tree
+// rows by their mask bit, nothing from c_end on.
+__device__ __forceinline__ uint32_t tc_visible16(int g0, int P, int c_end, uint64_t m0, uint64_t m1) {
+    const int np = min(max(min(P, c_end) - g0, 0), 16);
+    uint32_t bits = (1u << np) - 1u;
+    const int e0 = max(P - g0, 0);
+    if (e0 < 16) {
+        const int j0 = g0 + e0 - P;                       // first tree row of the group, 0 <= j0
+        uint64_t w = 0ull;
+        if (j0 < 64) w = (m0 >> j0) | (j0 > 0 ? (m1 << (64 - j0)) : 0ull);
+        else if (j0 < 128) w = m1 >> (j0 - 64);
+        const int nv = min(max(c_end - (g0 + e0), 0), 16);
+        bits |= (((uint32_t)w & ((1u << nv) - 1u)) << e0) & 0xffffu;
+    }
+    return bits;
+}
 __device__ __forceinline__ void pair_barrier(int quadrant) {     // the two warps that share a lane quadrant
     asm volatile("bar.sync %0, 64;" ::"r"(quadrant + 1) : "memory");
 }
@@ -552,24 +587,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     const uint32_t half = (uint32_t)NB * 128u;             // bytes between the two head-dim halves of a block
     const size_t stage_bytes = (size_t)NB * 512;           // K block, then V block
 
-    // part 0: rows below the prefix length only; 1: the others (zeros beyond the share); 2: all
-    auto load_kv = [&](int b, int part) {
-        uint8_t* ks = kv_s + (size_t)(b % NST) * stage_bytes;
+    // part 0: rows below the prefix length only; 1: the others (zeros beyond the share); 2: all.
+    // Thread t of warps 0-7 copies 16-byte chunk t & 15 of rows (t >> 4) + 16 i: the swizzle term is the same for all i.
+    const int ld_ch = threadIdx.x & 15, ld_rr = (threadIdx.x >> 4) & 15;
+    const uint32_t ld_off0 = tc_off(ld_rr, ld_ch, NB);
+    const size_t ld_g0 = (size_t)h * HD + (size_t)ld_ch * 8;
+    auto load_kv = [&](int b, int stage, int part) {
+        uint8_t* ks = kv_s + (size_t)stage * stage_bytes + ld_off0;
         uint8_t* vs = ks + (size_t)NB * 256;
         const int r0 = c_begin + b * NB;
         const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-        for (int e = threadIdx.x; e < n16 * 16; e += 256) {
-            const int r = e >> 4, ch = e & 15, row = r0 + r;
+        for (int r = ld_rr; r < n16; r += 16, ks += 2048, vs += 2048) {
+            const int row = r0 + r;
             if (part == 0 && row >= p.P) continue;
             if (part == 1 && row < p.P) continue;
-            const uint32_t off = tc_off(r, ch, NB);
             const bool valid = row < c_end;
-            const size_t gofs = valid ? (size_t)row * p.kv_stride + (size_t)h * HD + ch * 8 : 0;
-            cp_async16_zfill(ks + off, p.k + gofs, valid);
-            cp_async16_zfill(vs + off, p.v + gofs, valid);
+            const size_t gofs = valid ? (size_t)row * p.kv_stride + ld_g0 : 0;
+            cp_async16_zfill(ks, p.k + gofs, valid);
+            cp_async16_zfill(vs, p.v + gofs, valid);
         }
     };
 
+    if (threadIdx.x == 0) TCT(0);
     pdl_launch_dependents();
     if (warp == 8) {
         tmem_alloc(tmem_slot, kTcCols);
@@ -593,13 +632,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
         }
     } else {
         // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
-        for (int b = 0; b < NST && b < nb; ++b) load_kv(b, 0);
+        for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 0);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     if (p.csize > 1) cluster_sync_all();                   // every receiving barrier is armed before anybody can send
+    if (threadIdx.x == 0) TCT(1);
     pdl_wait();
+    if (threadIdx.x == 0) TCT(2);
     const uint32_t tbase = *tmem_slot;
     const uint32_t tO = tbase + 384;
     const uint32_t q_u32 = smem_u32(q_s);
@@ -614,38 +655,47 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 const uint32_t ks_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes);
                 const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
                 const uint32_t idesc = umma_idesc_bf16_m128(n16);
+                const uint64_t da0 = umma_desc_sw128(q_u32), db0 = umma_desc_sw128(ks_u32);      // the address field takes plain additions
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
-                    const uint64_t da = umma_desc_sw128(q_u32 + (uint32_t)(ks >> 2) * (128u * 128u) + (uint32_t)(ks & 3) * 32u);
-                    const uint64_t db = umma_desc_sw128(ks_u32 + (uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u);
+                    const uint64_t da = da0 + (uint64_t)(((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4);
+                    const uint64_t db = db0 + (uint64_t)(((uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u) >> 4);
                     umma_bf16(tS, da, db, idesc, ks > 0);
                 }
                 umma_commit(bar_s + (b & 1));
             };
             bool ok = mbar_wait(bar_kv, 0, wait_expired);          // Q and block 0
+            TCT(3);
             if (ok) {
                 tc_fence_after_sync();
                 issue_qk(0);
             }
+            TCT(4);
             for (int b = 0; b < nb && ok; ++b) {
                 if (b + 1 < nb) {
                     ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
                     if (!ok) break;
+                    if (b < 8) TCT(512 + b * 8 + 0);
                     tc_fence_after_sync();
                     issue_qk(b + 1);
+                    if (b < 8) TCT(512 + b * 8 + 1);
                 }
                 ok = mbar_wait(bar_p, (uint32_t)b & 1u, wait_expired);
                 if (!ok) break;
+                if (b < 8) TCT(512 + b * 8 + 2);
                 tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
                 const int n16 = min(NB, (c_end - r0 + 15) & ~15);
                 const uint32_t vs_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes) + (uint32_t)NB * 256u;
                 const uint32_t tP = tbase + (uint32_t)(b & 1) * kTcSStride;
-                for (int kk = 0; kk < n16 / 16; ++kk)
-                    umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, b > 0 || kk > 0);
-                for (int kk = 0; kk < n16 / 16; ++kk)
-                    umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, umma_desc_sw128_mn(vs_u32 + (uint32_t)kk * 2048u, half), idv, true);
+                const uint64_t dv0 = umma_desc_sw128_mn(vs_u32, half);
+                const int nk = n16 / 16;
+                for (int kk = 0; kk < nk; ++kk)
+                    umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, b > 0 || kk > 0);
+                for (int kk = 0; kk < nk; ++kk)
+                    umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, true);
                 umma_commit(bar_o);
+                if (b < 8) TCT(512 + b * 8 + 3);
             }
         }
     } else {
@@ -656,7 +706,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             cp_async16_zfill(q_s + tc_off(r, ch, 128), p.q + (valid ? ((size_t)r * p.nh + h) * HD + ch * 8 : 0), valid);
         }
         for (int b = 0; b < NST && b < nb; ++b) {
-            load_kv(b, 1);
+            load_kv(b, b, 1);
             cp_async_arrive(bar_kv + b);
         }
         const int quad = warp & 3, hf = warp >> 2;
@@ -677,13 +727,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
             float v[CPT];
             float corr = 1.f, ref = 0.f;
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 0);
             if (ok) ok = mbar_wait(bar_s + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
             tc_fence_after_sync();
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 1);
             if (act) {
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16)
                     if (c < ncol) tmem_ld16_nowait(tS + lane_base + (uint32_t)(c0 + c), v + c);
                 tmem_wait_ld<CPT>(v);
+                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 2);
                 const int lim = min(p.P, c_end);
                 float mx = -INFINITY;
 #pragma unroll
@@ -692,11 +745,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                         const int g0 = r0 + c0 + c;
                         if (g0 + 16 <= lim) {
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) { v[c + e] *= p.scale_log2; mx = fmaxf(mx, v[c + e]); }
+                            for (int e = 0; e < 16; ++e) mx = fmaxf(mx, v[c + e]);
                         } else {
+                            const uint32_t vis = tc_visible16(g0, p.P, c_end, mk0, mk1);
 #pragma unroll
                             for (int e = 0; e < 16; ++e) {
-                                v[c + e] = tc_visible(g0 + e, p.P, c_end, mk0, mk1) ? v[c + e] * p.scale_log2 : -INFINITY;
+                                v[c + e] = ((vis >> e) & 1u) ? v[c + e] : -INFINITY;
                                 mx = fmaxf(mx, v[c + e]);
                             }
                         }
@@ -704,7 +758,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 }
                 xch[((b & 1) * 2 + hf) * 128 + row] = mx;
                 pair_barrier(quad);                              // both halves are in registers; maxima exchanged
-                mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
+                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 3);
+                mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]) * p.scale_log2;     // the scale is positive
                 const float mn = fmaxf(m_run, mx);
                 ref = (mn == -INFINITY) ? 0.f : mn;
                 corr = exp2f(m_run - ref);
@@ -714,10 +769,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 // P(b-1) V(b-1) has completed: O is stable, and the stage it read can be refilled
                 if (ok) ok = mbar_wait(bar_o, (uint32_t)(b - 1) & 1u, wait_expired);
                 tc_fence_after_sync();
-                if (b - 1 + NST < nb) {
-                    load_kv(b - 1 + NST, 2);
-                    cp_async_arrive(bar_kv + (b - 1) % NST);
-                }
+                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 4);
                 if (act && __any_sync(0xffffffffu, corr != 1.f)) {
 #pragma unroll
                     for (int c = 0; c < HD / 2; c += 16) {
@@ -729,6 +781,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                     }
                 }
             }
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 6);
             if (act) {
                 float ls = 0.f;
 #pragma unroll
@@ -737,12 +790,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                         uint32_t hi[8], lo[8];
 #pragma unroll
                         for (int e = 0; e < 16; e += 2) {
-                            const float x0 = exp2f(v[c + e] - ref), x1 = exp2f(v[c + e + 1] - ref);
+                            const float x0 = ex2_approx(fmaf(v[c + e], p.scale_log2, -ref));
+                            const float x1 = ex2_approx(fmaf(v[c + e + 1], p.scale_log2, -ref));
                             ls += x0 + x1;
-                            const float h0 = bf16_bits_to_float(float_to_bf16_bits(x0));
-                            const float h1 = bf16_bits_to_float(float_to_bf16_bits(x1));
-                            hi[e >> 1] = pack_bf16x2(h0, h1);
-                            lo[e >> 1] = pack_bf16x2(x0 - h0, x1 - h1);
+                            const uint32_t hh = cvt_bf16x2(x0, x1);
+                            hi[e >> 1] = hh;
+                            lo[e >> 1] = cvt_bf16x2(x0 - __uint_as_float(hh << 16), x1 - __uint_as_float(hh & 0xffff0000u));
                         }
                         tmem_st8(tS + lane_base + (uint32_t)((c0 + c) >> 1), hi);
                         tmem_st8(tS + lane_base + (uint32_t)(ncol + ((c0 + c) >> 1)), lo);
@@ -751,14 +804,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 l_run = l_run * corr + ls;
                 tmem_wait_st();
             }
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 7);
             tc_fence_before_sync();
             mbar_arrive(bar_p);
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 8);
+            if (b > 0 && b - 1 + NST < nb) {             // the stage P(b-1) V(b-1) released (waited for above)
+                load_kv(b - 1 + NST, (b - 1) % NST, 2);
+                cp_async_arrive(bar_kv + (b - 1) % NST);
+            }
+            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 5);
         }
         // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
         if (nb > 0) {
             if (ok) ok = mbar_wait(bar_o, (uint32_t)(nb - 1) & 1u, wait_expired);
             tc_fence_after_sync();
         }
+        if (threadIdx.x == 0) TCT(5);
         cp_async_wait<0>();
         asm volatile("bar.sync 5, 256;" ::: "memory");          // warps 0-7: every MMA and copy that used the ring is done
         float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
@@ -784,6 +845,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             if (hf == 0 && row < Tpad) *reinterpret_cast<float2*>(loc + (size_t)row * REC + HD) = make_float2(m_run, l_run + xl[128 + row]);
         }
     }
+    if (threadIdx.x == 0) TCT(6);
     tc_fence_before_sync();
     const int csize = p.csize, rpr = p.rpr;
     const int rank = split % csize, outer = split / csize;
@@ -822,6 +884,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             tmem_dealloc(tbase, kTcCols);
         }
     }
+    if (threadIdx.x == 0) TCT(7);
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
     for (int rl = warp; rl < n_my && warp < 8; rl += 8) {
         const int grow = row0 + rl;                    // global query row
@@ -863,8 +926,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             if (lane == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
+    if (threadIdx.x == 0) TCT(8);
     // nobody leaves while a peer's copy may still be reading this CTA's deposit
     if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (threadIdx.x == 0) TCT(9);
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
@@ -921,7 +986,7 @@ size_t attn_plan(AttnProblem& p) {
     // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
     p.qsplit = 0;
     p.mt_per_cta = 0;
-    p.use_tc = (p.hd == 128 && attn_tc_enabled()) ? 1 : 0;
+    p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_enabled()) ? 1 : 0;
     const int n_mt = tpad / 16;
     if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
         int mpc = 1, groups = n_mt;
@@ -1156,3 +1221,9 @@ extern "C" int cats_tree_attention_static(const void* d_q, const void* d_k, cons
     if (launch_tree_attention(a, (cudaStream_t)stream) != cudaSuccess) return CATS_ERR_CUDA;
     return CATS_OK;
 }
+
+#ifdef CATS_TC_TRACE
+extern "C" int cats_debug_read_tc_trace(long long* host, int n) {
+    return (int)cudaMemcpyFromSymbol(host, cats::g_tc_trace, sizeof(long long) * (size_t)n);
+}
+#endif
