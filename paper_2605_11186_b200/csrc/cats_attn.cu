@@ -486,7 +486,8 @@ __device__ long long g_tc_trace[1024];
 #else
 #define TCT(slot) do { } while (0)
 #endif
-constexpr int kTcThreads = 288;       // warps 0-7: softmax and loads; warp 8: MMA issue, tensor-memory allocation
+constexpr int kTcThreads = 384;       // warps 0-7: softmax; warp 8: MMA issue, tensor-memory allocation; warps 9-11: loads
+constexpr int kTcLoaders = 96;
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
 constexpr int kTcStream = 64;         // cache rows per block when a share is streamed
@@ -572,8 +573,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete
     uint64_t* bar_o = rbar + 3;           //      P(b) V(b) complete
     uint64_t* bar_p = rbar + 4;           //      P(b) written (256 arrivals)
-    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  block landed (256 arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(rbar + 5 + kTcMaxStages);
+    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  refill landed (one arrival per loader thread)
+    uint64_t* bar_kv0 = bar_kv + kTcMaxStages;   // [kTcMaxStages]  first fill landed (warps 0-7, 256 arrivals)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_kv0 + kTcMaxStages);
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -588,23 +590,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     const size_t stage_bytes = (size_t)NB * 512;           // K block, then V block
 
     // part 0: rows below the prefix length only; 1: the others (zeros beyond the share); 2: all.
-    // Thread t of warps 0-7 copies 16-byte chunk t & 15 of rows (t >> 4) + 16 i: the swizzle term is the same for all i.
-    const int ld_ch = threadIdx.x & 15, ld_rr = (threadIdx.x >> 4) & 15;
-    const uint32_t ld_off0 = tc_off(ld_rr, ld_ch, NB);
+    // The first fill of the ring is issued by warps 0-7 (which have nothing else to do until S(0) exists), the refills
+    // by the loader warps: thread t of the n issuing threads copies 16-byte chunk t & 15 of rows (t >> 4) + (n / 16) i.
+    const int ld_n = warp > 8 ? kTcLoaders : 256;
+    const int ld_t = warp > 8 ? (int)threadIdx.x - 288 : (int)threadIdx.x, ld_ch = ld_t & 15, ld_rr = ld_t >> 4;
     const size_t ld_g0 = (size_t)h * HD + (size_t)ld_ch * 8;
     auto load_kv = [&](int b, int stage, int part) {
-        uint8_t* ks = kv_s + (size_t)stage * stage_bytes + ld_off0;
+        uint8_t* ks = kv_s + (size_t)stage * stage_bytes;
         uint8_t* vs = ks + (size_t)NB * 256;
         const int r0 = c_begin + b * NB;
         const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-        for (int r = ld_rr; r < n16; r += 16, ks += 2048, vs += 2048) {
+        for (int r = ld_rr; r < n16; r += ld_n / 16) {
             const int row = r0 + r;
             if (part == 0 && row >= p.P) continue;
             if (part == 1 && row < p.P) continue;
             const bool valid = row < c_end;
             const size_t gofs = valid ? (size_t)row * p.kv_stride + ld_g0 : 0;
-            cp_async16_zfill(ks, p.k + gofs, valid);
-            cp_async16_zfill(vs, p.v + gofs, valid);
+            const uint32_t off = tc_off(r, ld_ch, NB);
+            cp_async16_zfill(ks + off, p.k + gofs, valid);
+            cp_async16_zfill(vs + off, p.v + gofs, valid);
         }
     };
 
@@ -619,7 +623,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             mbar_init(bar_s + 1, 1);
             mbar_init(bar_o, 1);
             mbar_init(bar_p, 256);
-            for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 256);
+            for (int i = 0; i < kTcMaxStages; ++i) { mbar_init(bar_kv + i, kTcLoaders); mbar_init(bar_kv0 + i, 256); }
             if (p.csize > 1) {
                 const int rank_ = split % p.csize;
                 const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
@@ -630,7 +634,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 mbar_fence_init();
             }
         }
-    } else {
+    } else if (warp < 8) {
         // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
         for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 0);
     }
@@ -664,7 +668,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 }
                 umma_commit(bar_s + (b & 1));
             };
-            bool ok = mbar_wait(bar_kv, 0, wait_expired);          // Q and block 0
+            bool ok = mbar_wait(bar_kv0, 0, wait_expired);         // Q and block 0
             TCT(3);
             if (ok) {
                 tc_fence_after_sync();
@@ -673,7 +677,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             TCT(4);
             for (int b = 0; b < nb && ok; ++b) {
                 if (b + 1 < nb) {
-                    ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
+                    ok = b + 1 < NST ? mbar_wait(bar_kv0 + (b + 1), 0, wait_expired)
+                                     : mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST - 1) & 1u, wait_expired);
                     if (!ok) break;
                     if (b < 8) TCT(512 + b * 8 + 0);
                     tc_fence_after_sync();
@@ -698,8 +703,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 if (b < 8) TCT(512 + b * 8 + 3);
             }
         }
+    } else if (warp > 8) {
+        // ---- loaders: a refill whenever a P V product frees a stage ----
+        for (int j = NST; j < nb; ++j) {
+            if (!mbar_wait(bar_o, (uint32_t)(j - NST) & 1u, wait_expired)) break;
+            load_kv(j, j % NST, 2);
+            cp_async_arrive(bar_kv + j % NST);
+        }
+        cp_async_wait<0>();
     } else {
-        // ---- warps 0-7: Q and the rows that depend on the previous kernel, then softmax and refills ----
+        // ---- warps 0-7: Q and the rows that depend on the previous kernel, then softmax ----
         for (int e = threadIdx.x; e < 128 * 16; e += 256) {
             const int r = e >> 4, ch = e & 15;
             const bool valid = r < p.T;
@@ -707,7 +720,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
         }
         for (int b = 0; b < NST && b < nb; ++b) {
             load_kv(b, b, 1);
-            cp_async_arrive(bar_kv + b);
+            cp_async_arrive(bar_kv0 + b);
         }
         const int quad = warp & 3, hf = warp >> 2;
         const int row = quad * 32 + lane;                       // the query row (= TMEM lane) of this thread
@@ -760,7 +773,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 pair_barrier(quad);                              // both halves are in registers; maxima exchanged
                 if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 3);
                 mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]) * p.scale_log2;     // the scale is positive
-                const float mn = fmaxf(m_run, mx);
+                // the old reference is kept while the maximum grows by less than 2^8 (probabilities then stay below 256 and
+                // nothing is rescaled); any reference gives the same merged result
+                const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
                 ref = (mn == -INFINITY) ? 0.f : mn;
                 corr = exp2f(m_run - ref);
                 m_run = mn;
@@ -808,10 +823,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             tc_fence_before_sync();
             mbar_arrive(bar_p);
             if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 8);
-            if (b > 0 && b - 1 + NST < nb) {             // the stage P(b-1) V(b-1) released (waited for above)
-                load_kv(b - 1 + NST, (b - 1) % NST, 2);
-                cp_async_arrive(bar_kv + (b - 1) % NST);
-            }
             if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 5);
         }
         // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
@@ -820,8 +831,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             tc_fence_after_sync();
         }
         if (threadIdx.x == 0) TCT(5);
-        cp_async_wait<0>();
-        asm volatile("bar.sync 5, 256;" ::: "memory");          // warps 0-7: every MMA and copy that used the ring is done
         float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
         if (act) {
             float* xl = xch + 512;                              // [2][128]
@@ -889,27 +898,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     for (int rl = warp; rl < n_my && warp < 8; rl += 8) {
         const int grow = row0 + rl;                    // global query row
         if (grow >= p.T) break;
-        float mp = -INFINITY, lp = 0.f;
-        if (lane < n_parts) {
-            const float* my_rec = src_parts + (size_t)lane * part_stride + (size_t)(csize > 1 ? rl : grow) * REC;
-            const float2 ml = *reinterpret_cast<const float2*>(my_rec + HD);
-            mp = ml.x; lp = ml.y;
+        // every lane reads the (m, l) of all partials itself (broadcast loads): no shuffles on the critical path
+        const float* rec0 = src_parts + (size_t)(csize > 1 ? rl : grow) * REC;
+        float mpv[8], lpv[8], M = -INFINITY;
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp) {
+            mpv[pp] = -INFINITY; lpv[pp] = 0.f;
+            if (pp < n_parts) {
+                const float2 ml = *reinterpret_cast<const float2*>(rec0 + (size_t)pp * part_stride + HD);
+                mpv[pp] = ml.x; lpv[pp] = ml.y;
+                M = fmaxf(M, ml.x);
+            }
         }
-        float M = mp;
-#pragma unroll
-        for (int ofs = 16; ofs > 0; ofs >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, ofs));
         const float ref = (M == -INFINITY) ? 0.f : M;
-        const float wp = exp2f(mp - ref);
-        float L = lp * wp;
-#pragma unroll
-        for (int ofs = 16; ofs > 0; ofs >>= 1) L += __shfl_xor_sync(0xffffffffu, L, ofs);
+        float L = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float* base = src_parts + (size_t)(csize > 1 ? rl : grow) * REC + lane * 4;
-        for (int pp = 0; pp < n_parts; ++pp) {                 // partials in a fixed order
-            const float w = __shfl_sync(0xffffffffu, wp, pp);
-            if (w != 0.f) {
-                const float4 v = *reinterpret_cast<const float4*>(base + (size_t)pp * part_stride);
-                acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp) {                       // partials in a fixed order
+            if (pp < n_parts) {
+                const float w = exp2f(mpv[pp] - ref);
+                L += lpv[pp] * w;
+                if (w != 0.f) {
+                    const float4 v = *reinterpret_cast<const float4*>(rec0 + (size_t)pp * part_stride + lane * 4);
+                    acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+                }
             }
         }
         if (p.n_outer == 1) {
