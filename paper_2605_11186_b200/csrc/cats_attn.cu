@@ -641,7 +641,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (p.csize > 1) cluster_sync_all();                   // every receiving barrier is armed before anybody can send
+    // every receiving barrier is armed before anybody can send: arrive here, wait just before the pushes
+    if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     if (threadIdx.x == 0) TCT(1);
     pdl_wait();
     if (threadIdx.x == 0) TCT(2);
@@ -751,24 +752,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 tmem_wait_ld<CPT>(v);
                 if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 2);
                 const int lim = min(p.P, c_end);
-                float mx = -INFINITY;
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // independent chains
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16) {
                     if (c < ncol) {
                         const int g0 = r0 + c0 + c;
-                        if (g0 + 16 <= lim) {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) mx = fmaxf(mx, v[c + e]);
-                        } else {
+                        if (g0 + 16 > lim) {
                             const uint32_t vis = tc_visible16(g0, p.P, c_end, mk0, mk1);
 #pragma unroll
-                            for (int e = 0; e < 16; ++e) {
-                                v[c + e] = ((vis >> e) & 1u) ? v[c + e] : -INFINITY;
-                                mx = fmaxf(mx, v[c + e]);
-                            }
+                            for (int e = 0; e < 16; ++e) v[c + e] = ((vis >> e) & 1u) ? v[c + e] : -INFINITY;
                         }
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[c + e]);
                     }
                 }
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 xch[((b & 1) * 2 + hf) * 128 + row] = mx;
                 pair_barrier(quad);                              // both halves are in registers; maxima exchanged
                 if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 3);
@@ -798,7 +796,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             }
             if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 6);
             if (act) {
-                float ls = 0.f;
+                float ls4[4] = {0.f, 0.f, 0.f, 0.f};                      // independent chains, summed in a fixed order
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16) {
                     if (c < ncol) {
@@ -807,16 +805,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                         for (int e = 0; e < 16; e += 2) {
                             const float x0 = ex2_approx(fmaf(v[c + e], p.scale_log2, -ref));
                             const float x1 = ex2_approx(fmaf(v[c + e + 1], p.scale_log2, -ref));
-                            ls += x0 + x1;
-                            const uint32_t hh = cvt_bf16x2(x0, x1);
-                            hi[e >> 1] = hh;
-                            lo[e >> 1] = cvt_bf16x2(x0 - __uint_as_float(hh << 16), x1 - __uint_as_float(hh & 0xffff0000u));
+                            ls4[(e >> 1) & 3] += x0 + x1;
+                            // hi = the upper 16 bits of x (exact in bf16), lo = the upper 16 bits of x - hi: integer and
+                            // byte-permute operations only, the conversion unit is left to the exponentials
+                            const uint32_t b0 = __float_as_uint(x0), b1 = __float_as_uint(x1);
+                            hi[e >> 1] = __byte_perm(b0, b1, 0x7632);
+                            const float l0 = x0 - __uint_as_float(b0 & 0xffff0000u), l1 = x1 - __uint_as_float(b1 & 0xffff0000u);
+                            lo[e >> 1] = __byte_perm(__float_as_uint(l0), __float_as_uint(l1), 0x7632);
                         }
                         tmem_st8(tS + lane_base + (uint32_t)((c0 + c) >> 1), hi);
                         tmem_st8(tS + lane_base + (uint32_t)(ncol + ((c0 + c) >> 1)), lo);
                     }
                 }
-                l_run = l_run * corr + ls;
+                l_run = l_run * corr + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
                 tmem_wait_st();
             }
             if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 7);
@@ -865,6 +866,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     if (csize > 1) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the deposit is read by bulk copies
         __syncthreads();
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // the peers' receiving barriers exist
         if (warp == 8) {
             tc_fence_after_sync();
             tmem_dealloc(tbase, kTcCols);
@@ -972,9 +974,10 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
 
 // Chooses the cluster size (CTAs per head that share one merge through distributed shared memory) and, for long
 // prefixes with few heads, the number of clusters per head.  Returns the bytes of workspace the outer merge needs.
-static bool attn_tc_enabled() {
-    static const bool on = [] { const char* e = getenv("CATS_ATTN_TC"); return e != nullptr && e[0] == '1'; }();
-    return on;
+// CATS_ATTN_TC=0 / 1 forces the mma.sync / the tcgen05 kernel (for measurements); unset: chosen by shape.
+static int attn_tc_override() {
+    static const int v = [] { const char* e = getenv("CATS_ATTN_TC"); return e == nullptr ? -1 : (e[0] == '1' ? 1 : 0); }();
+    return v;
 }
 
 size_t attn_plan(AttnProblem& p) {
@@ -998,7 +1001,11 @@ size_t attn_plan(AttnProblem& p) {
     // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
     p.qsplit = 0;
     p.mt_per_cta = 0;
-    p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_enabled()) ? 1 : 0;
+    // The tcgen05 kernel (head_dim 128, positive scale) is ahead except for one query tile over a short cache, where
+    // seven eighths of its 128 MMA rows are padding (measured in the 7B forward at prefix 512: 3.13 vs 3.12 ms at T = 16,
+    // 3.18 vs 3.22 at 32, 3.44 vs 3.48 at 64, 4.02 vs 4.14 at 128; over 16384 rows 106 vs 239 us at T = 128).
+    p.use_tc = (p.hd == 128 && p.scale > 0.f && (tpad > 16 || S > 2048)) ? 1 : 0;
+    if (attn_tc_override() >= 0) p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_override() == 1) ? 1 : 0;
     const int n_mt = tpad / 16;
     if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
         int mpc = 1, groups = n_mt;
