@@ -486,8 +486,8 @@ __device__ long long g_tc_trace[1024];
 #else
 #define TCT(slot) do { } while (0)
 #endif
-constexpr int kTcThreads = 384;       // warps 0-7: softmax; warp 8: MMA issue, tensor-memory allocation; warps 9-11: loads
-constexpr int kTcLoaders = 96;
+constexpr int kTcThreads = 320;       // warps 0-7: softmax; warp 8: MMA issue, tensor-memory allocation; warp 9: TMA loads
+constexpr int kTcBoxRows = 32;        // rows of one TMA box (64 head-dim elements wide)
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
 constexpr int kTcStream = 64;         // cache rows per block when a share is streamed
@@ -560,7 +560,9 @@ __device__ __forceinline__ void pair_barrier(int quadrant) {     // the two warp
     asm volatile("bar.sync %0, 64;" ::"r"(quadrant + 1) : "memory");
 }
 
-__global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p) {
+__global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
+                                                                const __grid_constant__ CUtensorMap tm_k,
+                                                                const __grid_constant__ CUtensorMap tm_v) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
     constexpr int HD = 128, REC = HD + 4, CPT = kTcOneShot / 2;    // CPT: most columns of S one thread holds
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
@@ -573,9 +575,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete
     uint64_t* bar_o = rbar + 3;           //      P(b) V(b) complete
     uint64_t* bar_p = rbar + 4;           //      P(b) written (256 arrivals)
-    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  refill landed (one arrival per loader thread)
-    uint64_t* bar_kv0 = bar_kv + kTcMaxStages;   // [kTcMaxStages]  first fill landed (warps 0-7, 256 arrivals)
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_kv0 + kTcMaxStages);
+    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  block landed (bytes counted)
+    uint64_t* bar_q = bar_kv + kTcMaxStages;     //      Q landed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 1);
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -589,26 +591,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
     const uint32_t half = (uint32_t)NB * 128u;             // bytes between the two head-dim halves of a block
     const size_t stage_bytes = (size_t)NB * 512;           // K block, then V block
 
-    // part 0: rows below the prefix length only; 1: the others (zeros beyond the share); 2: all.
-    // The first fill of the ring is issued by warps 0-7 (which have nothing else to do until S(0) exists), the refills
-    // by the loader warps: thread t of the n issuing threads copies 16-byte chunk t & 15 of rows (t >> 4) + (n / 16) i.
-    const int ld_n = warp > 8 ? kTcLoaders : 256;
-    const int ld_t = warp > 8 ? (int)threadIdx.x - 288 : (int)threadIdx.x, ld_ch = ld_t & 15, ld_rr = ld_t >> 4;
-    const size_t ld_g0 = (size_t)h * HD + (size_t)ld_ch * 8;
-    auto load_kv = [&](int b, int stage, int part) {
+    // One thread (warp 9) moves everything with TMA: boxes of 32 rows x 64 head-dim elements land as 32 swizzled
+    // 128-byte rows.  The tensor maps end at row P + T_tree (K, V) and T (Q): rows beyond read as zeros.  Rows between
+    // the end of this CTA's share and the end of the cache are another CTA's (finite values, masked in the softmax).
+    // part 0: boxes wholly below the prefix length (no dependence on the previous kernel); 1: the others; 2: all.
+    auto load_kv = [&](int b, int stage, int part, uint64_t policy) {
         uint8_t* ks = kv_s + (size_t)stage * stage_bytes;
         uint8_t* vs = ks + (size_t)NB * 256;
         const int r0 = c_begin + b * NB;
-        const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-        for (int r = ld_rr; r < n16; r += ld_n / 16) {
-            const int row = r0 + r;
-            if (part == 0 && row >= p.P) continue;
-            if (part == 1 && row < p.P) continue;
-            const bool valid = row < c_end;
-            const size_t gofs = valid ? (size_t)row * p.kv_stride + ld_g0 : 0;
-            const uint32_t off = tc_off(r, ld_ch, NB);
-            cp_async16_zfill(ks + off, p.k + gofs, valid);
-            cp_async16_zfill(vs + off, p.v + gofs, valid);
+        for (int rb = 0; rb < NB; rb += kTcBoxRows) {
+            const bool below = r0 + rb + kTcBoxRows <= p.P;
+            if ((part == 0 && !below) || (part == 1 && below)) continue;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                tma_load_2d(ks + (size_t)hh * half + (size_t)rb * 128, &tm_k, h * HD + hh * 64, r0 + rb, bar_kv + stage, policy);
+                tma_load_2d(vs + (size_t)hh * half + (size_t)rb * 128, &tm_v, h * HD + hh * 64, r0 + rb, bar_kv + stage, policy);
+            }
         }
     };
 
@@ -623,7 +621,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             mbar_init(bar_s + 1, 1);
             mbar_init(bar_o, 1);
             mbar_init(bar_p, 256);
-            for (int i = 0; i < kTcMaxStages; ++i) { mbar_init(bar_kv + i, kTcLoaders); mbar_init(bar_kv0 + i, 256); }
+            for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 1);
+            mbar_init(bar_q, 1);
             if (p.csize > 1) {
                 const int rank_ = split % p.csize;
                 const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
@@ -634,13 +633,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 mbar_fence_init();
             }
         }
-    } else if (warp < 8) {
-        // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
-        for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 0);
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    uint64_t ld_policy = 0;
+    if (warp == 9 && lane == 0) {
+        // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
+        ld_policy = l2_policy_evict_first();
+        for (int b = 0; b < NST && b < nb; ++b) {
+            mbar_expect_tx(bar_kv + b, (uint32_t)stage_bytes);
+            load_kv(b, b, 0, ld_policy);
+        }
+    }
     // every receiving barrier is armed before anybody can send: arrive here, wait just before the pushes
     if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     if (threadIdx.x == 0) TCT(1);
@@ -669,7 +674,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 }
                 umma_commit(bar_s + (b & 1));
             };
-            bool ok = mbar_wait(bar_kv0, 0, wait_expired);         // Q and block 0
+            bool ok = mbar_wait(bar_q, 0, wait_expired) && mbar_wait(bar_kv, 0, wait_expired);         // Q and block 0
             TCT(3);
             if (ok) {
                 tc_fence_after_sync();
@@ -678,8 +683,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
             TCT(4);
             for (int b = 0; b < nb && ok; ++b) {
                 if (b + 1 < nb) {
-                    ok = b + 1 < NST ? mbar_wait(bar_kv0 + (b + 1), 0, wait_expired)
-                                     : mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST - 1) & 1u, wait_expired);
+                    ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
                     if (!ok) break;
                     if (b < 8) TCT(512 + b * 8 + 0);
                     tc_fence_after_sync();
@@ -704,25 +708,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p)
                 if (b < 8) TCT(512 + b * 8 + 3);
             }
         }
-    } else if (warp > 8) {
-        // ---- loaders: a refill whenever a P V product frees a stage ----
-        for (int j = NST; j < nb; ++j) {
-            if (!mbar_wait(bar_o, (uint32_t)(j - NST) & 1u, wait_expired)) break;
-            load_kv(j, j % NST, 2);
-            cp_async_arrive(bar_kv + j % NST);
+    } else if (warp == 9) {
+        // ---- loader: Q and the boxes that depend on the previous kernel, then a refill whenever a P V product frees a stage ----
+        if (lane == 0) {
+            if (nb > 0) mbar_expect_tx(bar_q, 128u * 256u);
+            for (int rb = 0; rb < 128 && nb > 0; rb += kTcBoxRows) {
+                tma_load_2d(q_s + (size_t)rb * 128, &tm_q, h * HD, rb, bar_q, ld_policy);
+                tma_load_2d(q_s + 128 * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
+            }
+            for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 1, ld_policy);
+            for (int j = NST; j < nb; ++j) {
+                if (!mbar_wait(bar_o, (uint32_t)(j - NST) & 1u, wait_expired)) break;
+                mbar_expect_tx(bar_kv + j % NST, (uint32_t)stage_bytes);
+                load_kv(j, j % NST, 2, ld_policy);
+            }
         }
-        cp_async_wait<0>();
     } else {
-        // ---- warps 0-7: Q and the rows that depend on the previous kernel, then softmax ----
-        for (int e = threadIdx.x; e < 128 * 16; e += 256) {
-            const int r = e >> 4, ch = e & 15;
-            const bool valid = r < p.T;
-            cp_async16_zfill(q_s + tc_off(r, ch, 128), p.q + (valid ? ((size_t)r * p.nh + h) * HD + ch * 8 : 0), valid);
-        }
-        for (int b = 0; b < NST && b < nb; ++b) {
-            load_kv(b, b, 1);
-            cp_async_arrive(bar_kv0 + b);
-        }
+        // ---- warps 0-7: softmax ----
         const int quad = warp & 3, hf = warp >> 2;
         const int row = quad * 32 + lane;                       // the query row (= TMEM lane) of this thread
         const bool act = quad * 32 < Tpad;                      // the warp owns query rows
@@ -1026,8 +1028,9 @@ size_t attn_plan(AttnProblem& p) {
     return n_outer > 1 ? (size_t)p.nh * n_outer * tpad * (p.hd + 2) * sizeof(float) : 0;
 }
 
-template <typename Kern>
-static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t smem, int csize, cudaStream_t st, const AttnDev& d) {
+template <typename Kern, typename... Extra>
+static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t smem, int csize, cudaStream_t st, const AttnDev& d,
+                                  const Extra&... extra) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -1049,9 +1052,55 @@ static cudaError_t launch_cluster(Kern kernel, dim3 grid, dim3 block, size_t sme
     cfg.attrs = attr;
     cfg.numAttrs = n;
     ++g_launch_count;
-    return cudaLaunchKernelEx(&cfg, kernel, d);
+    return cudaLaunchKernelEx(&cfg, kernel, d, extra...);
 }
 
+// ---- tensor maps for the tcgen05 kernel ----------------------------------------------------------
+// A [rows][cols] bf16 matrix with a row pitch, read in boxes of kTcBoxRows rows x 64 columns with the 128-byte swizzle;
+// rows from `rows` on read as zeros.  The driver entry point is looked up once; the encoded maps are cached by
+// (pointer, shape), since a decoding loop asks for the same few maps again and again.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static TensorMapEncodeFn tensor_map_encoder() {
+    static const TensorMapEncodeFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (TensorMapEncodeFn)f;
+    }();
+    return fn;
+}
+static bool attn_tensor_map(const void* ptr, long long cols, long long rows, long long pitch_elems, CUtensorMap* out) {
+    struct Entry { const void* ptr; long long cols, rows, pitch; CUtensorMap map; bool used; };
+    constexpr int kSlots = 256;
+    static Entry cache[kSlots];
+    static std::mutex mu;
+    const size_t hsh = ((size_t)ptr >> 4) * 0x9E3779B97F4A7C15ull + (size_t)rows * 0xC2B2AE3D27D4EB4Full + (size_t)pitch_elems;
+    Entry& e = cache[(hsh >> 20) % kSlots];
+    std::lock_guard<std::mutex> lock(mu);
+    if (e.used && e.ptr == ptr && e.cols == cols && e.rows == rows && e.pitch == pitch_elems) {
+        *out = e.map;
+        return true;
+    }
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTcBoxRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+        e.used = false;
+        return false;
+    }
+    e.ptr = ptr; e.cols = cols; e.rows = rows; e.pitch = pitch_elems; e.used = true;
+    *out = e.map;
+    return true;
+}
+
+// Returns cudaErrorNotSupported when the tensor maps cannot be made (the caller then uses the mma.sync kernel).
 static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
@@ -1094,7 +1143,12 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     }
     const size_t smem = fixed + (size_t)d.kv_area;
     dim3 grid(p.cluster * p.n_splits, p.nh);
-    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kTcThreads), smem, p.cluster, st, d);
+    CUtensorMap tm_q, tm_k, tm_v;
+    const long long width = (long long)p.nh * p.hd;
+    if (!attn_tensor_map(p.q, width, p.T, width, &tm_q) || !attn_tensor_map(p.k, width, p.prefix_len + d.Tk, p.kv_stride, &tm_k) ||
+        !attn_tensor_map(p.v, width, p.prefix_len + d.Tk, p.kv_stride, &tm_v))
+        return cudaErrorNotSupported;
+    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
@@ -1110,7 +1164,10 @@ cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    if (p.use_tc) return launch_tree_attention_tc(p, st);
+    if (p.use_tc) {
+        const cudaError_t e = launch_tree_attention_tc(p, st);
+        if (e != cudaErrorNotSupported) return e;     // no tensor maps on this driver: the kernel below takes any split
+    }
     AttnDev d;
     d.q = (const uint16_t*)p.q; d.k = (const uint16_t*)p.k; d.v = (const uint16_t*)p.v;
     d.mask = p.mask;
