@@ -464,28 +464,21 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // ---------------------------------------------------------------------------------------------------
 // The same attention on the 5th-generation tensor cores (head_dim 128).
 //
-// One CTA per (head, share of the cache rows), nine warps.  Q (128 rows, zero beyond T) and a ring of K/V blocks
+// One CTA per (head, share of the cache rows), ten warps.  Q (128 rows, zero beyond T) and a ring of K/V blocks
 // sit in shared memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of
-// 128-byte rows with the 128-byte swizzle.  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache
+// 128-byte rows with the 128-byte swizzle, written by TMA (one thread of warp 9 issues every copy; a refill goes into
+// the stage the last P V product released).  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache
 // row) and as the MN-major operand of O += P V (row = K index).  Warp 8 issues the MMAs: S(b+1) = Q K(b+1)^T is
 // issued before P(b) V(b), so the tensor core works on the next block while warps 0-7 take the softmax of this one.
 // S has two buffers in tensor memory, one query row per lane; warps w and w+4 share the 32 rows of lane quadrant
-// w and split the block's columns, so a row's maximum and sum need one exchange between two threads.  The
-// probabilities go back to tensor memory over the columns S occupied, as two bf16 operands hi + lo, and enter
-// P V as the A operand from tensor memory.  O accumulates in tensor memory and is rescaled (load, multiply, store)
-// only by warps in which a running maximum moved.  Warps 0-7 also refill the ring: cp.async into the stage the last
-// P V product released, completion counted on that stage's mbarrier.  The CTA's partial (m, l, O) is then merged
-// across the cluster exactly as in the kernel above.
+// w and split the block's columns.  The reference of the exponentials moves only when a row's maximum outgrows it
+// by 2^8, which the two warps find out by a vote inside the barrier that orders their loads of S before their stores
+// of P; only then are maxima exchanged and O (in tensor memory) rescaled.  The probabilities go back to tensor
+// memory over the columns S occupied, as two bf16 operands hi + lo (the upper and the next 16 bits of the fp32
+// value), and enter P V as the A operand from tensor memory.  The CTA's partial (m, l, O) is then merged across the
+// cluster as in the kernel above (the receiving barrier is armed early, the cluster barrier completed just before
+// the pushes).  A share of at most 192 rows is one block: nothing is streamed then.
 // ---------------------------------------------------------------------------------------------------
-#ifdef CATS_TC_TRACE
-__device__ long long g_tc_trace[1024];
-#define TCT(slot) do { if (blockIdx.x == TC_TRACE_X && blockIdx.y == 0 && (slot) < 1024) g_tc_trace[(slot)] = clock64(); } while (0)
-#ifndef TC_TRACE_X
-#define TC_TRACE_X 0
-#endif
-#else
-#define TCT(slot) do { } while (0)
-#endif
 constexpr int kTcThreads = 320;       // warps 0-7: softmax; warp 8: MMA issue, tensor-memory allocation; warp 9: TMA loads
 constexpr int kTcBoxRows = 32;        // rows of one TMA box (64 head-dim elements wide)
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
@@ -497,20 +490,6 @@ constexpr int kTcMaxStages = 4;
 // byte offset of 16-byte chunk ch (0..15) of row r in a [2 halves][rows][128 B] tile with the 128-byte swizzle
 __device__ __forceinline__ uint32_t tc_off(int r, int ch, int rows) {
     return (uint32_t)((ch >> 3) * rows * 128 + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
-}
-__device__ __forceinline__ bool tc_visible(int col, int P, int c_end, uint64_t m0, uint64_t m1) {
-    if (col >= c_end) return false;
-    if (col < P) return true;
-    const int j = col - P;
-    return (((j < 64) ? m0 : m1) >> (j & 63)) & 1ull;
-}
-// 16 bytes global -> shared, or 16 zero bytes when !valid (the source address is not read then)
-__device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, bool valid) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(valid ? 16u : 0u) : "memory");
-}
-// The mbarrier receives one arrival from this thread once all cp.async it has issued so far have landed.
-__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v) {
     uint32_t r[16];
@@ -535,11 +514,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {      // two roundings in one instruction
-    uint32_t d;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-    return d;
-}
 // Bit e set iff cache row g0 + e is visible to the query whose ancestor mask is (m0, m1): prefix rows always, tree
 // rows by their mask bit, nothing from c_end on.
 __device__ __forceinline__ uint32_t tc_visible16(int g0, int P, int c_end, uint64_t m0, uint64_t m1) {
@@ -558,6 +532,18 @@ __device__ __forceinline__ uint32_t tc_visible16(int g0, int P, int c_end, uint6
 }
 __device__ __forceinline__ void pair_barrier(int quadrant) {     // the two warps that share a lane quadrant
     asm volatile("bar.sync %0, 64;" ::"r"(quadrant + 1) : "memory");
+}
+__device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     // the same barrier, returning the OR of pred
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, 64, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(quadrant + 1)
+        : "memory");
+    return r != 0;
 }
 
 __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
@@ -610,7 +596,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         }
     };
 
-    if (threadIdx.x == 0) TCT(0);
     pdl_launch_dependents();
     if (warp == 8) {
         tmem_alloc(tmem_slot, kTcCols);
@@ -648,9 +633,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     }
     // every receiving barrier is armed before anybody can send: arrive here, wait just before the pushes
     if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    if (threadIdx.x == 0) TCT(1);
     pdl_wait();
-    if (threadIdx.x == 0) TCT(2);
     const uint32_t tbase = *tmem_slot;
     const uint32_t tO = tbase + 384;
     const uint32_t q_u32 = smem_u32(q_s);
@@ -675,24 +658,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 umma_commit(bar_s + (b & 1));
             };
             bool ok = mbar_wait(bar_q, 0, wait_expired) && mbar_wait(bar_kv, 0, wait_expired);         // Q and block 0
-            TCT(3);
             if (ok) {
                 tc_fence_after_sync();
                 issue_qk(0);
             }
-            TCT(4);
             for (int b = 0; b < nb && ok; ++b) {
                 if (b + 1 < nb) {
                     ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
                     if (!ok) break;
-                    if (b < 8) TCT(512 + b * 8 + 0);
                     tc_fence_after_sync();
                     issue_qk(b + 1);
-                    if (b < 8) TCT(512 + b * 8 + 1);
                 }
                 ok = mbar_wait(bar_p, (uint32_t)b & 1u, wait_expired);
                 if (!ok) break;
-                if (b < 8) TCT(512 + b * 8 + 2);
                 tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
                 const int n16 = min(NB, (c_end - r0 + 15) & ~15);
@@ -705,7 +683,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 for (int kk = 0; kk < nk; ++kk)
                     umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, true);
                 umma_commit(bar_o);
-                if (b < 8) TCT(512 + b * 8 + 3);
             }
         }
     } else if (warp == 9) {
@@ -743,16 +720,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
             float v[CPT];
             float corr = 1.f, ref = 0.f;
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 0);
             if (ok) ok = mbar_wait(bar_s + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
             tc_fence_after_sync();
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 1);
             if (act) {
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16)
                     if (c < ncol) tmem_ld16_nowait(tS + lane_base + (uint32_t)(c0 + c), v + c);
                 tmem_wait_ld<CPT>(v);
-                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 2);
                 const int lim = min(p.P, c_end);
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // independent chains
 #pragma unroll
@@ -768,24 +742,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                         for (int e = 0; e < 16; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[c + e]);
                     }
                 }
-                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                xch[((b & 1) * 2 + hf) * 128 + row] = mx;
-                pair_barrier(quad);                              // both halves are in registers; maxima exchanged
-                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 3);
-                mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]) * p.scale_log2;     // the scale is positive
-                // the old reference is kept while the maximum grows by less than 2^8 (probabilities then stay below 256 and
-                // nothing is rescaled); any reference gives the same merged result
-                const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
-                ref = (mn == -INFINITY) ? 0.f : mn;
-                corr = exp2f(m_run - ref);
-                m_run = mn;
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;     // the scale is positive
+                // The old reference is kept while the maximum grows by less than 2^8 (probabilities then stay below 256 and
+                // nothing is rescaled); any reference gives the same merged result.  The two warps of a quadrant vote in the
+                // barrier that also orders their loads of S before their stores of P; only if some row of the 32 wants
+                // a new reference are the maxima exchanged.
+                const bool want = !(m_run != -INFINITY && mx <= m_run + 8.f);
+                if (pair_barrier_or(quad, want)) {
+                    xch[((b & 1) * 2 + hf) * 128 + row] = mx;
+                    pair_barrier(quad);
+                    mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
+                    const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
+                    ref = (mn == -INFINITY) ? 0.f : mn;
+                    corr = exp2f(m_run - ref);
+                    m_run = mn;
+                } else {
+                    ref = m_run;
+                }
             }
-            if (b > 0) {
-                // P(b-1) V(b-1) has completed: O is stable, and the stage it read can be refilled
+            if (b > 0 && act && __any_sync(0xffffffffu, corr != 1.f)) {
+                // O follows the reference; P(b-1) V(b-1) must have completed first
                 if (ok) ok = mbar_wait(bar_o, (uint32_t)(b - 1) & 1u, wait_expired);
                 tc_fence_after_sync();
-                if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 4);
-                if (act && __any_sync(0xffffffffu, corr != 1.f)) {
+                {
 #pragma unroll
                     for (int c = 0; c < HD / 2; c += 16) {
                         float o[16];
@@ -796,7 +775,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                     }
                 }
             }
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 6);
             if (act) {
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};                      // independent chains, summed in a fixed order
 #pragma unroll
@@ -822,18 +800,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 l_run = l_run * corr + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
                 tmem_wait_st();
             }
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 7);
             tc_fence_before_sync();
+            // no second arrival before every thread has made its first: the hand-off barrier counts one per thread and block
+            if (b > 0 && ok) ok = mbar_wait(bar_p, (uint32_t)(b - 1) & 1u, wait_expired);
             mbar_arrive(bar_p);
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 8);
-            if (threadIdx.x == 0 && b < 8) TCT(16 + b * 16 + 5);
         }
         // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
         if (nb > 0) {
             if (ok) ok = mbar_wait(bar_o, (uint32_t)(nb - 1) & 1u, wait_expired);
             tc_fence_after_sync();
         }
-        if (threadIdx.x == 0) TCT(5);
         float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
         if (act) {
             float* xl = xch + 512;                              // [2][128]
@@ -857,7 +833,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             if (hf == 0 && row < Tpad) *reinterpret_cast<float2*>(loc + (size_t)row * REC + HD) = make_float2(m_run, l_run + xl[128 + row]);
         }
     }
-    if (threadIdx.x == 0) TCT(6);
     tc_fence_before_sync();
     const int csize = p.csize, rpr = p.rpr;
     const int rank = split % csize, outer = split / csize;
@@ -897,7 +872,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             tmem_dealloc(tbase, kTcCols);
         }
     }
-    if (threadIdx.x == 0) TCT(7);
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
     for (int rl = warp; rl < n_my && warp < 8; rl += 8) {
         const int grow = row0 + rl;                    // global query row
@@ -942,10 +916,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             if (lane == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
-    if (threadIdx.x == 0) TCT(8);
     // nobody leaves while a peer's copy may still be reading this CTA's deposit
     if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    if (threadIdx.x == 0) TCT(9);
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
@@ -1298,8 +1270,3 @@ extern "C" int cats_tree_attention_static(const void* d_q, const void* d_k, cons
     return CATS_OK;
 }
 
-#ifdef CATS_TC_TRACE
-extern "C" int cats_debug_read_tc_trace(long long* host, int n) {
-    return (int)cudaMemcpyFromSymbol(host, cats::g_tc_trace, sizeof(long long) * (size_t)n);
-}
-#endif
