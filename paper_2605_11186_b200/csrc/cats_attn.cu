@@ -975,10 +975,10 @@ size_t attn_plan(AttnProblem& p) {
     // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
     p.qsplit = 0;
     p.mt_per_cta = 0;
-    // The tcgen05 kernel (head_dim 128, positive scale) is ahead except for one query tile over a short cache, where
-    // seven eighths of its 128 MMA rows are padding (measured in the 7B forward at prefix 512: 3.13 vs 3.12 ms at T = 16,
-    // 3.18 vs 3.22 at 32, 3.44 vs 3.48 at 64, 4.02 vs 4.14 at 128; over 16384 rows 106 vs 239 us at T = 128).
-    p.use_tc = (p.hd == 128 && p.scale > 0.f && (tpad > 16 || S > 2048)) ? 1 : 0;
+    // The tcgen05 kernel (head_dim 128, positive scale) is ahead except for a single query tile, where seven eighths of its
+    // 128 MMA rows are padding (measured in the 7B forward at prefix 512: 3.13 vs 3.12 ms at T = 16, 3.18 vs 3.22 at 32,
+    // 3.44 vs 3.48 at 64, 4.02 vs 4.14 at 128; alone over 16384 rows: 97 vs 82 us at T = 16, 100 vs 253 us at T = 128).
+    p.use_tc = (p.hd == 128 && p.scale > 0.f && tpad > 16) ? 1 : 0;
     if (attn_tc_override() >= 0) p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_override() == 1) ? 1 : 0;
     const int n_mt = tpad / 16;
     if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
