@@ -873,10 +873,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         }
     }
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
-    for (int rl = warp; rl < n_my && warp < 8; rl += 8) {
+    // One thread per (query row, 8 output columns): all rows of the CTA are merged at once, every load of a thread is
+    // independent of the others (the (m, l) pairs are broadcast reads), and the result leaves as one 16-byte store.
+    for (int it = threadIdx.x; it < n_my * (HD / 8) && warp < 8; it += 256) {
+        const int rl = it / (HD / 8), c8 = (it % (HD / 8)) * 8;
         const int grow = row0 + rl;                    // global query row
-        if (grow >= p.T) break;
-        // every lane reads the (m, l) of all partials itself (broadcast loads): no shuffles on the critical path
+        if (grow >= p.T) continue;
         const float* rec0 = src_parts + (size_t)(csize > 1 ? rl : grow) * REC;
         float mpv[8], lpv[8], M = -INFINITY;
 #pragma unroll
@@ -890,30 +892,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         }
         const float ref = (M == -INFINITY) ? 0.f : M;
         float L = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int pp = 0; pp < 8; ++pp) {                       // partials in a fixed order
             if (pp < n_parts) {
                 const float w = exp2f(mpv[pp] - ref);
                 L += lpv[pp] * w;
                 if (w != 0.f) {
-                    const float4 v = *reinterpret_cast<const float4*>(rec0 + (size_t)pp * part_stride + lane * 4);
-                    acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+                    const float4 v0 = *reinterpret_cast<const float4*>(rec0 + (size_t)pp * part_stride + c8);
+                    const float4 v1 = *reinterpret_cast<const float4*>(rec0 + (size_t)pp * part_stride + c8 + 4);
+                    acc[0] += v0.x * w; acc[1] += v0.y * w; acc[2] += v0.z * w; acc[3] += v0.w * w;
+                    acc[4] += v1.x * w; acc[5] += v1.y * w; acc[6] += v1.z * w; acc[7] += v1.w * w;
                 }
             }
         }
         if (p.n_outer == 1) {
             const float inv = 1.f / L;
-            uint2 pk = make_uint2(pack_bf16x2(acc.x * inv, acc.y * inv), pack_bf16x2(acc.z * inv, acc.w * inv));
+            const uint4 pk = make_uint4(pack_bf16x2(acc[0] * inv, acc[1] * inv), pack_bf16x2(acc[2] * inv, acc[3] * inv),
+                                        pack_bf16x2(acc[4] * inv, acc[5] * inv), pack_bf16x2(acc[6] * inv, acc[7] * inv));
             uint8_t* ob = reinterpret_cast<uint8_t*>(p.out);
-            const int col = lane * 4;
-            size_t off = p.out_npad > 0 ? packed_act_offset(grow, (h * HD + col) >> 3, p.out_npad) + (size_t)(col & 7) * 2
-                                        : (((size_t)grow * p.nh + h) * HD + col) * 2;
-            *reinterpret_cast<uint2*>(ob + off) = pk;
+            const size_t off = p.out_npad > 0 ? packed_act_offset(grow, (h * HD + c8) >> 3, p.out_npad)
+                                              : (((size_t)grow * p.nh + h) * HD + c8) * 2;
+            *reinterpret_cast<uint4*>(ob + off) = pk;
         } else {
             const size_t gbase = ((size_t)h * p.n_outer + outer) * Tpad + grow;
-            *reinterpret_cast<float4*>(p.part_o + gbase * HD + lane * 4) = acc;
-            if (lane == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
+            *reinterpret_cast<float4*>(p.part_o + gbase * HD + c8) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            *reinterpret_cast<float4*>(p.part_o + gbase * HD + c8 + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+            if (c8 == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
     // nobody leaves while a peer's copy may still be reading this CTA's deposit

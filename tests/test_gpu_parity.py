@@ -217,6 +217,11 @@ ATTN_CASES = [
     ("rand128_P896_h32", gen.tree_random(128, 9), 896, 32, 128), ("rand128_P897_h32", gen.tree_random(128, 9), 897, 32, 128),
     # 40 heads: clusters of three CTAs (row blocks of 44, 44 and 40 query rows), and a 17-node tree on them
     ("rand128_P2048_h40", gen.tree_random(128, 11), 2048, 40, 128), ("rand17_P700_h40", gen.tree_random(17, 12), 700, 40, 128),
+    # head_dim 64 with 32 heads (the mma.sync kernel): query tiles split over the CTAs of a head, one and two tiles per CTA
+    ("heap64_P256_h32_hd64", gen.tree_heap(64), 256, 32, 64), ("rand128_P500_h32_hd64", gen.tree_random(128, 13), 500, 32, 64),
+    # shares just below / above the one-block limit of the tcgen05 kernel (192 rows), and a streamed share with a ragged tail
+    ("rand33_P735_h32", gen.tree_random(33, 14), 735, 32, 128), ("rand33_P736_h32", gen.tree_random(33, 14), 736, 32, 128),
+    ("rand90_P5000_h32", gen.tree_random(90, 15), 5000, 32, 128),
 ]
 
 
