@@ -546,11 +546,14 @@ __device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     /
     return r != 0;
 }
 
+// CPT: the most columns of S one softmax thread holds (a block has at most 2 CPT rows); instances for the streamed
+// 64-row blocks and for one-block shares of up to 128, 160 and 192 rows.
+template <int CPT>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
                                                                 const __grid_constant__ CUtensorMap tm_k,
                                                                 const __grid_constant__ CUtensorMap tm_v) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
-    constexpr int HD = 128, REC = HD + 4, CPT = kTcOneShot / 2;    // CPT: most columns of S one thread holds
+    constexpr int HD = 128, REC = HD + 4;
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
     const int Tpad = p.n_mt * 16;
     uint8_t* q_s = sm;                                                           // [2][128][128 B]
@@ -1081,7 +1084,10 @@ static bool attn_tensor_map(const void* ptr, long long cols, long long rows, lon
 static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -1125,7 +1131,11 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     if (!attn_tensor_map(p.q, width, p.T, width, &tm_q) || !attn_tensor_map(p.k, width, p.prefix_len + d.Tk, p.kv_stride, &tm_k) ||
         !attn_tensor_map(p.v, width, p.prefix_len + d.Tk, p.kv_stride, &tm_v))
         return cudaErrorNotSupported;
-    cudaError_t e = launch_cluster(k_tree_attn_tc, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    cudaError_t e;
+    if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else e = launch_cluster(k_tree_attn_tc<96>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
