@@ -247,6 +247,34 @@ def test_tree_attention_matches_oracle(cats, name, parent, P, nh, hd):
     assert err <= TOL, err
 
 
+@pytest.mark.parametrize("T,P,nh,hd", [(40, 700, 8, 128), (16, 300, 8, 128), (70, 260, 4, 64)])
+def test_tree_attention_with_padded_cache_rows(cats, T, P, nh, hd):
+    """The cache rows may be wider than n_heads * head_dim (kv_row_stride_elems > n_heads * head_dim): heads are found at
+    h * head_dim inside a row, the pad is never read.  The pad is filled with NaN so that a wrong pitch shows."""
+    parent = gen.tree_random(T, 21)
+    S, D, stride = P + T, nh * hd, nh * hd + 72
+    q = gen.normal_bf16((T, nh, hd), 1.0, "cpu", "attn_pad", T, "q")
+    k = gen.normal_bf16((S, D), 1.0, "cpu", "attn_pad", T, "k")
+    v = gen.normal_bf16((S, D), 1.0, "cpu", "attn_pad", T, "v")
+    _, mask, _, _ = oracle.build_tree_mask(parent, P)
+    scale = 1.0 / np.sqrt(hd)
+    want = oracle.tree_attention(q.float().numpy().astype(np.float64), cache_to_f32(k), cache_to_f32(v), mask, P, nh, hd, scale)
+    kw = torch.full((S, stride), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vw = torch.full((S, stride), float("nan"), dtype=torch.bfloat16, device="cuda")
+    kw[:, :D] = k.cuda()
+    vw[:, :D] = v.cuda()
+    out = torch.zeros((T, nh, hd), dtype=torch.bfloat16, device="cuda")
+    cfg = cats.model_cfg(gen.ModelShape(hidden=D, n_heads=nh, head_dim=hd, ffn=64, vocab=128, n_layers=1), S)
+    ws = cats.new_workspace(cfg, T, P)
+    st = cats.new_status()
+    cats.cats_tree_attention(q.cuda(), kw, vw, dev(mask.view(np.int64)), T, P, nh, hd, stride, float(scale), out, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    g = out.float().cpu().numpy()
+    assert np.isfinite(g).all()
+    assert np.abs(g - want).max() <= TOL
+
+
 @pytest.mark.parametrize("P,name,parent", CONFIG5_FULL, ids=["P%d_%s" % (c[0], c[1]) for c in CONFIG5_FULL])
 def test_config5_attention_sweep_full_size(cats, P, name, parent):
     """Config 5 at its full sizes: 32 heads x 128, prefixes up to 16384, the three tree shapes, K/V ~ N(0,1).  The oracle is
