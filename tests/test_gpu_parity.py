@@ -222,6 +222,9 @@ ATTN_CASES = [
     # shares just below / above the one-block limit of the tcgen05 kernel (192 rows), and a streamed share with a ragged tail
     ("rand33_P735_h32", gen.tree_random(33, 14), 735, 32, 128), ("rand33_P736_h32", gen.tree_random(33, 14), 736, 32, 128),
     ("rand90_P5000_h32", gen.tree_random(90, 15), 5000, 32, 128),
+    # no prefix at all; and 140 cache rows over four CTAs of 48 rows each: the last CTA of every cluster has no rows
+    ("rand128_P0_h32", gen.tree_random(128, 17), 0, 32, 128), ("rand40_P0_h5", gen.tree_random(40, 18), 0, 5, 128),
+    ("rand40_P100_h32", gen.tree_random(40, 16), 100, 32, 128),
 ]
 
 
