@@ -563,8 +563,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));
     uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete
     uint64_t* bar_o = rbar + 3;           //      P(b) V(b) complete
-    uint64_t* bar_p = rbar + 4;           //      P(b) written (256 arrivals)
-    uint64_t* bar_kv = rbar + 5;          // [kTcMaxStages]  block landed (bytes counted)
+    uint64_t* bar_p = rbar + 4;           // [2]  P(b) written (256 arrivals), by block parity
+    uint64_t* bar_kv = rbar + 6;          // [kTcMaxStages]  block landed (bytes counted)
     uint64_t* bar_q = bar_kv + kTcMaxStages;     //      Q landed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 1);
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -609,6 +609,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             mbar_init(bar_s + 1, 1);
             mbar_init(bar_o, 1);
             mbar_init(bar_p, 256);
+            mbar_init(bar_p + 1, 256);
             for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 1);
             mbar_init(bar_q, 1);
             if (p.csize > 1) {
@@ -672,7 +673,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                     tc_fence_after_sync();
                     issue_qk(b + 1);
                 }
-                ok = mbar_wait(bar_p, (uint32_t)b & 1u, wait_expired);
+                ok = mbar_wait(bar_p + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
@@ -804,9 +805,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 tmem_wait_st();
             }
             tc_fence_before_sync();
-            // no second arrival before every thread has made its first: the hand-off barrier counts one per thread and block
-            if (b > 0 && ok) ok = mbar_wait(bar_p, (uint32_t)(b - 1) & 1u, wait_expired);
-            mbar_arrive(bar_p);
+            // Two hand-off barriers alternate by block, each counting one arrival per thread and block: no arrival for
+            // block b before every thread has arrived for block b - 2 (a thread can be at most one block ahead of the
+            // slowest, since S(b + 1) exists only after P(b - 1) V(b - 1) was issued).
+            if (b > 1 && ok) ok = mbar_wait(bar_p + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
+            mbar_arrive(bar_p + (b & 1));
         }
         // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
         if (nb > 0) {
