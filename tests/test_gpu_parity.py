@@ -278,6 +278,30 @@ def test_tree_attention_with_padded_cache_rows(cats, T, P, nh, hd):
     assert np.abs(g - want).max() <= TOL
 
 
+@pytest.mark.parametrize("T,P,nh,hd", [(64, 6000, 32, 128), (128, 3000, 32, 128), (40, 500, 32, 128), (16, 2000, 32, 128), (50, 900, 8, 64)])
+def test_tree_attention_is_deterministic(cats, T, P, nh, hd):
+    """Same inputs, bit-identical outputs (fixed reduction order), over many launches back to back: the blocks of a share
+    are handed between the load, MMA and softmax warps through barriers only, so a missing one would show up here."""
+    parent = gen.tree_random(T, 31)
+    S, D = P + T, nh * hd
+    q = gen.normal_bf16((T, nh, hd), 1.0, "cuda", "attn_det", T, "q")
+    k = gen.normal_bf16((S, D), 1.0, "cuda", "attn_det", T, "k")
+    v = gen.normal_bf16((S, D), 1.0, "cuda", "attn_det", T, "v")
+    _, mask, _, _ = oracle.build_tree_mask(parent, P)
+    d_mask = dev(mask.view(np.int64))
+    cfg = cats.model_cfg(gen.ModelShape(hidden=D, n_heads=nh, head_dim=hd, ffn=64, vocab=128, n_layers=1), S)
+    ws = cats.new_workspace(cfg, T, P)
+    st = cats.new_status()
+    outs = [torch.zeros((T, nh, hd), dtype=torch.bfloat16, device="cuda") for _ in range(40)]
+    for o in outs:
+        cats.cats_tree_attention(q, k, v, d_mask, T, P, nh, hd, D, float(1.0 / np.sqrt(hd)), o, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ref = outs[0].view(torch.int16)
+    assert all(torch.equal(o.view(torch.int16), ref) for o in outs[1:])
+    assert torch.isfinite(outs[0].float()).all()
+
+
 @pytest.mark.parametrize("P,name,parent", CONFIG5_FULL, ids=["P%d_%s" % (c[0], c[1]) for c in CONFIG5_FULL])
 def test_config5_attention_sweep_full_size(cats, P, name, parent):
     """Config 5 at its full sizes: 32 heads x 128, prefixes up to 16384, the three tree shapes, K/V ~ N(0,1).  The oracle is
