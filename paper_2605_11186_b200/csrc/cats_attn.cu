@@ -1,5 +1,8 @@
 // Tree-masked attention of the T draft-tree nodes against the KV prefix plus their own ancestors.
 //
+// Two kernels: k_tree_attn (bf16 mma.sync; head_dim 64 or 128), described first, and k_tree_attn_tc (tcgen05, tensor
+// memory and TMA; head_dim 128), further down, which takes every tree of more than 16 nodes at head_dim 128.
+//
 // Q [T_pad][hd] sits in shared memory; the cache rows stream through a double-buffered cp.async pipeline
 // (128-bit loads); S = Q K^T and O += P V run on bf16 tensor-core MMAs (fp32 accumulation, online softmax in
 // fp32 with warp-shuffle row reductions, the probabilities as a bf16 pair hi + lo).  Prefix rows need no mask;
@@ -487,10 +490,6 @@ constexpr int kTcStream = 64;         // cache rows per block when a share is st
 constexpr int kTcOneShot = 192;       // a share of at most this many rows is one block
 constexpr int kTcMaxStages = 4;
 
-// byte offset of 16-byte chunk ch (0..15) of row r in a [2 halves][rows][128 B] tile with the 128-byte swizzle
-__device__ __forceinline__ uint32_t tc_off(int r, int ch, int rows) {
-    return (uint32_t)((ch >> 3) * rows * 128 + r * 128 + (((ch & 7) ^ (r & 7)) << 4));
-}
 __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v) {
     uint32_t r[16];
     asm volatile(
