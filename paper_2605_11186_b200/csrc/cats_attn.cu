@@ -609,8 +609,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             mbar_init(bar_o, 1);
             mbar_init(bar_p, 256);
             mbar_init(bar_p + 1, 256);
-            for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 1);
-            mbar_init(bar_q, 1);
             if (p.csize > 1) {
                 const int rank_ = split % p.csize;
                 const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
@@ -622,18 +620,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             }
         }
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
     uint64_t ld_policy = 0;
     if (warp == 9 && lane == 0) {
-        // prefix rows do not depend on the previous kernel: request them for every stage of the ring now
+        // The loader sets up its own barriers and requests the prefix rows of every stage of the ring at once: they depend
+        // neither on the previous kernel nor on the rest of the set-up.
+        for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 1);
+        mbar_init(bar_q, 1);
+        mbar_fence_init();
         ld_policy = l2_policy_evict_first();
         for (int b = 0; b < NST && b < nb; ++b) {
             mbar_expect_tx(bar_kv + b, (uint32_t)stage_bytes);
             load_kv(b, b, 0, ld_policy);
         }
     }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
     // every receiving barrier is armed before anybody can send: arrive here, wait just before the pushes
     if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_wait();
