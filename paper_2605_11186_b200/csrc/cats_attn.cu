@@ -482,7 +482,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // cluster as in the kernel above (the receiving barrier is armed early, the cluster barrier completed just before
 // the pushes).  A share of at most 192 rows is one block: nothing is streamed then.
 // ---------------------------------------------------------------------------------------------------
-constexpr int kTcThreads = 320;       // warps 0-7: softmax; warp 8: MMA issue, tensor-memory allocation; warp 9: TMA loads
+constexpr int kTcThreads = 352;       // warps 0-7: softmax; 8: issue of Q K^T, tensor-memory allocation; 9: TMA loads; 10: issue of P V
+                                      // (streamed shares only: a one-block share is launched with 320 threads)
 constexpr int kTcBoxRows = 32;        // rows of one TMA box (64 head-dim elements wide)
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
@@ -547,7 +548,8 @@ __device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     /
 
 // CPT: the most columns of S one softmax thread holds (a block has at most 2 CPT rows); instances for the streamed
 // 64-row blocks and for one-block shares of up to 128, 160 and 192 rows.
-template <int CPT>
+// STREAM: the share is streamed in blocks (otherwise it is one block, and everything that hands blocks on is compiled out).
+template <int CPT, bool STREAM>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
                                                                 const __grid_constant__ CUtensorMap tm_k,
                                                                 const __grid_constant__ CUtensorMap tm_v) {
@@ -560,11 +562,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][2][128] row maxima (by block parity), [2][128] row sums
     float* recv = xch + 768;                                                     // [csize][rpr][REC]
     uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));
-    uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete
-    uint64_t* bar_o = rbar + 3;           //      P(b) V(b) complete
-    uint64_t* bar_p = rbar + 4;           // [2]  P(b) written (256 arrivals), by block parity
-    uint64_t* bar_kv = rbar + 6;          // [kTcMaxStages]  block landed (bytes counted)
-    uint64_t* bar_q = bar_kv + kTcMaxStages;     //      Q landed
+    // Every barrier that a thread may find more than one phase ahead of itself would give a wrong answer to a parity
+    // wait, so each one is either indexed by block parity (its next completion needs the waiter's own progress) or by
+    // ring stage (the classical full / empty pair).
+    uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete, by block parity
+    uint64_t* bar_o = rbar + 3;           // [2]  P(b) V(b) complete, by block parity
+    uint64_t* bar_p = rbar + 5;           // [2]  P(b) written (256 arrivals), by block parity
+    uint64_t* bar_kv = rbar + 7;          // [kTcMaxStages]  block landed in the stage (bytes counted)
+    uint64_t* bar_free = bar_kv + kTcMaxStages;  // [kTcMaxStages]  the P V product that read the stage has completed
+    uint64_t* bar_q = bar_free + kTcMaxStages;   //      Q landed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 1);
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -575,7 +581,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     const int c_end = min(S, c_begin + p.rows_per_split);
     const int NB = p.blk;                                  // rows per block, a multiple of 32
     const int NST = p.stages;                              // stages of the ring
-    const int nb = (c_end - c_begin + NB - 1) / NB;
+    const int nb = STREAM ? (c_end - c_begin + NB - 1) / NB : (c_end > c_begin ? 1 : 0);
     const uint32_t half = (uint32_t)NB * 128u;             // bytes between the two head-dim halves of a block
     const size_t stage_bytes = (size_t)NB * 512;           // K block, then V block
 
@@ -607,6 +613,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             mbar_init(bar_s, 1);
             mbar_init(bar_s + 1, 1);
             mbar_init(bar_o, 1);
+            mbar_init(bar_o + 1, 1);
             mbar_init(bar_p, 256);
             mbar_init(bar_p + 1, 256);
             if (p.csize > 1) {
@@ -624,7 +631,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     if (warp == 9 && lane == 0) {
         // The loader sets up its own barriers and requests the prefix rows of every stage of the ring at once: they depend
         // neither on the previous kernel nor on the rest of the set-up.
-        for (int i = 0; i < kTcMaxStages; ++i) mbar_init(bar_kv + i, 1);
+        for (int i = 0; i < kTcMaxStages; ++i) { mbar_init(bar_kv + i, 1); mbar_init(bar_free + i, 1); }
         mbar_init(bar_q, 1);
         mbar_fence_init();
         ld_policy = l2_policy_evict_first();
@@ -643,11 +650,38 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     const uint32_t tO = tbase + 384;
     const uint32_t q_u32 = smem_u32(q_s);
 
+    // O += P(b) V(b), issued as soon as the softmax warps have written P(b)
+    auto issue_pv = [&](int b) -> bool {
+        const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
+        if (!(mbar_wait(bar_kv + b % NST, (uint32_t)(b / NST) & 1u, wait_expired) &&      // V(b) (long since landed)
+              mbar_wait(bar_p + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired)))
+            return false;
+        tc_fence_after_sync();
+        const int r0 = c_begin + b * NB;
+        const int n16 = min(NB, (c_end - r0 + 15) & ~15);
+        const uint32_t vs_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes) + (uint32_t)NB * 256u;
+        const uint32_t tP = tbase + (uint32_t)(b & 1) * kTcSStride;
+        const uint64_t dv0 = umma_desc_sw128_mn(vs_u32, half);
+        const int nk = n16 / 16;
+        for (int kk = 0; kk < nk; ++kk)
+            umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, b > 0 || kk > 0);
+        for (int kk = 0; kk < nk; ++kk)
+            umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, true);
+        umma_commit(bar_o + (b & 1));
+        umma_commit(bar_free + b % NST);
+        return true;
+    };
     if (warp == 8) {
-        // ---- MMA issue: QK(0); then per block QK(b+1) ahead of PV(b) ----
+        // ---- issue of S(b) = Q K(b)^T: as soon as block b has landed and the product that read the S / P buffer of
+        //      block b - 2 has completed (issuing one tcgen05.mma costs its thread about a hundred cycles, so the two
+        //      kinds of products are issued by two threads) ----
         if (lane == 0 && nb > 0) {
-            const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
-            auto issue_qk = [&](int b) {
+            bool ok = mbar_wait(bar_q, 0, wait_expired);
+            for (int b = 0; b < nb && ok; ++b) {
+                ok = mbar_wait(bar_kv + b % NST, (uint32_t)(b / NST) & 1u, wait_expired);
+                if (ok && b >= 2) ok = mbar_wait(bar_o + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
+                if (!ok) break;
+                tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
                 const int n16 = min(NB, (c_end - r0 + 15) & ~15);
                 const uint32_t ks_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes);
@@ -661,35 +695,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                     umma_bf16(tS, da, db, idesc, ks > 0);
                 }
                 umma_commit(bar_s + (b & 1));
-            };
-            bool ok = mbar_wait(bar_q, 0, wait_expired) && mbar_wait(bar_kv, 0, wait_expired);         // Q and block 0
-            if (ok) {
-                tc_fence_after_sync();
-                issue_qk(0);
             }
-            for (int b = 0; b < nb && ok; ++b) {
-                if (b + 1 < nb) {
-                    ok = mbar_wait(bar_kv + (b + 1) % NST, (uint32_t)((b + 1) / NST) & 1u, wait_expired);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    issue_qk(b + 1);
-                }
-                ok = mbar_wait(bar_p + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const int r0 = c_begin + b * NB;
-                const int n16 = min(NB, (c_end - r0 + 15) & ~15);
-                const uint32_t vs_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes) + (uint32_t)NB * 256u;
-                const uint32_t tP = tbase + (uint32_t)(b & 1) * kTcSStride;
-                const uint64_t dv0 = umma_desc_sw128_mn(vs_u32, half);
-                const int nk = n16 / 16;
-                for (int kk = 0; kk < nk; ++kk)
-                    umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, b > 0 || kk > 0);
-                for (int kk = 0; kk < nk; ++kk)
-                    umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, true);
-                umma_commit(bar_o);
-            }
+            if (!STREAM && ok) issue_pv(0);      // one-block share: the same thread issues P V as well
         }
+    } else if (STREAM && warp == 10) {
+        // ---- issue of O += P(b) V(b) for streamed shares (a one-block share is launched without this warp) ----
+        if (lane == 0)
+            for (int b = 0; b < nb; ++b)
+                if (!issue_pv(b)) break;
     } else if (warp == 9) {
         // ---- loader: Q and the boxes that depend on the previous kernel, then a refill whenever a P V product frees a stage ----
         if (lane == 0) {
@@ -699,8 +712,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 tma_load_2d(q_s + 128 * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
             }
             for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 1, ld_policy);
-            for (int j = NST; j < nb; ++j) {
-                if (!mbar_wait(bar_o, (uint32_t)(j - NST) & 1u, wait_expired)) break;
+            for (int j = NST; STREAM && j < nb; ++j) {
+                if (!mbar_wait(bar_free + j % NST, (uint32_t)(j / NST - 1) & 1u, wait_expired)) break;
                 mbar_expect_tx(bar_kv + j % NST, (uint32_t)stage_bytes);
                 load_kv(j, j % NST, 2, ld_policy);
             }
@@ -765,9 +778,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                     ref = m_run;
                 }
             }
-            if (b > 0 && act && __any_sync(0xffffffffu, corr != 1.f)) {
+            if (STREAM && b > 0 && act && __any_sync(0xffffffffu, corr != 1.f)) {
                 // O follows the reference; P(b-1) V(b-1) must have completed first
-                if (ok) ok = mbar_wait(bar_o, (uint32_t)(b - 1) & 1u, wait_expired);
+                if (ok) ok = mbar_wait(bar_o + ((b - 1) & 1), (uint32_t)((b - 1) >> 1) & 1u, wait_expired);
                 tc_fence_after_sync();
                 {
 #pragma unroll
@@ -807,14 +820,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             }
             tc_fence_before_sync();
             // Two hand-off barriers alternate by block, each counting one arrival per thread and block: no arrival for
-            // block b before every thread has arrived for block b - 2 (a thread can be at most one block ahead of the
-            // slowest, since S(b + 1) exists only after P(b - 1) V(b - 1) was issued).
-            if (b > 1 && ok) ok = mbar_wait(bar_p + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
+            // block b before every thread has arrived for block b - 2 (which holds anyway: S(b) is issued only after
+            // P(b - 2) V(b - 2) has completed).
+            if (STREAM && b > 1 && ok) ok = mbar_wait(bar_p + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
             mbar_arrive(bar_p + (b & 1));
         }
         // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
         if (nb > 0) {
-            if (ok) ok = mbar_wait(bar_o, (uint32_t)(nb - 1) & 1u, wait_expired);
+            if (ok) ok = mbar_wait(bar_o + ((nb - 1) & 1), (uint32_t)((nb - 1) >> 1) & 1u, wait_expired);
             tc_fence_after_sync();
         }
         float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
@@ -1088,10 +1101,11 @@ static bool attn_tensor_map(const void* ptr, long long cols, long long rows, lon
 static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -1114,7 +1128,7 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
-    const size_t fixed = 1024 + 128 * 256 + 3072 + recv + 128;     // alignment slack, Q, pair exchange, received partials, barriers
+    const size_t fixed = 1024 + 128 * 256 + 3072 + recv + 192;     // alignment slack, Q, pair exchange, received partials, barriers
     // the ring: stages of 64 rows of K and V (32 KB each), as many as fit, at least three (which also hold a one-block share)
     int stages = (int)((227 * 1024 - fixed) / (kTcStream * 512));
     if (stages > kTcMaxStages) stages = kTcMaxStages;
@@ -1136,10 +1150,12 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
         !attn_tensor_map(p.v, width, p.prefix_len + d.Tk, p.kv_stride, &tm_v))
         return cudaErrorNotSupported;
     cudaError_t e;
-    if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else e = launch_cluster(k_tree_attn_tc<96>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    const dim3 one(kTcThreads - 32);      // the warp that issues P V on its own exists for streamed shares only
+    if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<32, true>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else e = launch_cluster(k_tree_attn_tc<96, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
