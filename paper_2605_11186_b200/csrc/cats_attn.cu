@@ -765,17 +765,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 // nothing is rescaled); any reference gives the same merged result.  The two warps of a quadrant vote in the
                 // barrier that also orders their loads of S before their stores of P; only if some row of the 32 wants
                 // a new reference are the maxima exchanged.
-                const bool want = !(m_run != -INFINITY && mx <= m_run + 8.f);
-                if (pair_barrier_or(quad, want)) {
-                    xch[((b & 1) * 2 + hf) * 128 + row] = mx;
+                if (!STREAM) {
+                    // the only block: its maximum is the reference (one exchange, whose barrier orders the loads and stores)
+                    xch[hf * 128 + row] = mx;
                     pair_barrier(quad);
-                    mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
-                    const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
-                    ref = (mn == -INFINITY) ? 0.f : mn;
-                    corr = exp2f(m_run - ref);
-                    m_run = mn;
+                    m_run = fmaxf(mx, xch[(hf ^ 1) * 128 + row]);
+                    ref = (m_run == -INFINITY) ? 0.f : m_run;
                 } else {
-                    ref = m_run;
+                    const bool want = !(m_run != -INFINITY && mx <= m_run + 8.f);
+                    if (pair_barrier_or(quad, want)) {
+                        xch[((b & 1) * 2 + hf) * 128 + row] = mx;
+                        pair_barrier(quad);
+                        mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
+                        const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
+                        ref = (mn == -INFINITY) ? 0.f : mn;
+                        corr = exp2f(m_run - ref);
+                        m_run = mn;
+                    } else {
+                        ref = m_run;
+                    }
                 }
             }
             if (STREAM && b > 0 && act && __any_sync(0xffffffffu, corr != 1.f)) {
@@ -815,7 +823,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                         tmem_st8(tS + lane_base + (uint32_t)(ncol + ((c0 + c) >> 1)), lo);
                     }
                 }
-                l_run = l_run * corr + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
+                l_run = (STREAM ? l_run * corr : 0.f) + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
                 tmem_wait_st();
             }
             tc_fence_before_sync();
