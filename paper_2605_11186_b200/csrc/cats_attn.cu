@@ -467,12 +467,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // ---------------------------------------------------------------------------------------------------
 // The same attention on the 5th-generation tensor cores (head_dim 128).
 //
-// One CTA per (head, share of the cache rows), ten warps.  Q (128 rows, zero beyond T) and a ring of K/V blocks
-// sit in shared memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of
+// One CTA per (head, share of the cache rows), ten or eleven warps.  Q (128 rows, zero beyond T) and a ring of K/V
+// blocks sit in shared memory in the layout tcgen05.mma reads: two halves of 64 head-dim elements, each a stack of
 // 128-byte rows with the 128-byte swizzle, written by TMA (one thread of warp 9 issues every copy; a refill goes into
 // the stage the last P V product released).  The SAME bytes serve as the K-major operand of S = Q K^T (row = cache
-// row) and as the MN-major operand of O += P V (row = K index).  Warp 8 issues the MMAs: S(b+1) = Q K(b+1)^T is
-// issued before P(b) V(b), so the tensor core works on the next block while warps 0-7 take the softmax of this one.
+// row) and as the MN-major operand of O += P V (row = K index).  One thread of warp 8 issues S(b) = Q K(b)^T as soon
+// as block b has landed (and the product that read the S / P buffer of block b - 2 has completed), one thread of
+// warp 10 issues P(b) V(b) as soon as P(b) is written: the tensor core works on the next block during the softmax of
+// this one, and neither kind of product waits for the ~100 cycles the other's issue costs per instruction.
 // S has two buffers in tensor memory, one query row per lane; warps w and w+4 share the 32 rows of lane quadrant
 // w and split the block's columns.  The reference of the exponentials moves only when a row's maximum outgrows it
 // by 2^8, which the two warps find out by a vote inside the barrier that orders their loads of S before their stores
@@ -480,7 +482,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // memory over the columns S occupied, as two bf16 operands hi + lo (the upper and the next 16 bits of the fp32
 // value), and enter P V as the A operand from tensor memory.  The CTA's partial (m, l, O) is then merged across the
 // cluster as in the kernel above (the receiving barrier is armed early, the cluster barrier completed just before
-// the pushes).  A share of at most 192 rows is one block: nothing is streamed then.
+// the pushes).  A share of at most 192 rows is one block: those instances are compiled without ring, vote, rescale
+// and second issuing warp (warp 8 issues both products).
 // ---------------------------------------------------------------------------------------------------
 constexpr int kTcThreads = 352;       // warps 0-7: softmax; 8: issue of Q K^T, tensor-memory allocation; 9: TMA loads; 10: issue of P V
                                       // (streamed shares only: a one-block share is launched with 320 threads)
