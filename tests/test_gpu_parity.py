@@ -278,6 +278,46 @@ def test_tree_attention_with_padded_cache_rows(cats, T, P, nh, hd):
     assert np.abs(g - want).max() <= TOL
 
 
+def _random_attention_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        T = int(rng.integers(1, 129))
+        P = int(rng.choice([0, int(rng.integers(1, 64)), int(rng.integers(64, 700)), int(rng.integers(700, 2600))]))
+        nh = int(rng.choice([1, 2, 3, 5, 8, 12, 20, 32, 40]))
+        hd = 128 if rng.random() < 0.8 else 64
+        out.append((i, T, P, nh, hd))
+    return out
+
+
+@pytest.mark.parametrize("i,T,P,nh,hd", _random_attention_shapes(48, 20260511), ids=lambda v: str(v))
+def test_tree_attention_random_shapes(cats, i, T, P, nh, hd):
+    """Seeded random shapes: every combination of tree size, prefix length and head count picks its own split of the
+    cache rows (cluster size, rows per CTA, one block or streamed, ragged last block); a sample of heads is compared."""
+    parent = gen.tree_random(T, 100 + i)
+    S, D = P + T, nh * hd
+    q = gen.normal_bf16((T, nh, hd), 1.0, "cuda", "attn_rand", i, "q")
+    k = gen.normal_bf16((S, D), 1.0, "cuda", "attn_rand", i, "k")
+    v = gen.normal_bf16((S, D), 1.0, "cuda", "attn_rand", i, "v")
+    _, mask, _, _ = oracle.build_tree_mask(parent, P)
+    scale = 1.0 / np.sqrt(hd)
+    out = torch.zeros((T, nh, hd), dtype=torch.bfloat16, device="cuda")
+    cfg = cats.model_cfg(gen.ModelShape(hidden=D, n_heads=nh, head_dim=hd, ffn=64, vocab=128, n_layers=1), S)
+    ws = cats.new_workspace(cfg, T, P)
+    st = cats.new_status()
+    cats.cats_tree_attention(q, k, v, dev(mask.view(np.int64)), T, P, nh, hd, D, float(scale), out, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    g = out.float().cpu().numpy()
+    assert np.isfinite(g).all()
+    heads = sorted(set([0, nh - 1, nh // 2]))
+    qf, kf, vf = q.float().cpu().numpy().astype(np.float64), k.float().cpu().numpy(), v.float().cpu().numpy()
+    for h in heads:
+        want = oracle.tree_attention(np.ascontiguousarray(qf[:, h:h + 1]), np.ascontiguousarray(kf[:, h * hd:(h + 1) * hd]),
+                                     np.ascontiguousarray(vf[:, h * hd:(h + 1) * hd]), mask, P, 1, hd, scale)
+        assert np.abs(g[:, h] - want[:, 0]).max() <= TOL, (h, float(np.abs(g[:, h] - want[:, 0]).max()))
+
+
 @pytest.mark.parametrize("T,P,nh,hd", [(64, 6000, 32, 128), (128, 3000, 32, 128), (40, 500, 32, 128), (16, 2000, 32, 128), (50, 900, 8, 64)])
 def test_tree_attention_is_deterministic(cats, T, P, nh, hd):
     """Same inputs, bit-identical outputs (fixed reduction order), over many launches back to back: the blocks of a share
