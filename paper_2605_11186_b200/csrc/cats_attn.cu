@@ -481,8 +481,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // of P; only then are maxima exchanged and O (in tensor memory) rescaled.  The probabilities go back to tensor
 // memory over the columns S occupied, as two bf16 operands hi + lo (the upper and the next 16 bits of the fp32
 // value), and enter P V as the A operand from tensor memory.  The CTA's partial (m, l, O) is then merged across the
-// cluster as in the kernel above (the receiving barrier is armed early, the cluster barrier completed just before
-// the pushes).  A share of at most 192 rows is one block: those instances are compiled without ring, vote, rescale
+// cluster: every softmax thread stores its half row straight into the shared memory of the CTA that merges that row
+// (distributed shared memory; one phase of the cluster barrier makes sure every CTA has started, the next publishes the
+// records), and the merge reads local memory only.  A share of at most 192 rows is one block: those instances are compiled without ring, vote, rescale
 // and second issuing warp (warp 8 issues both products).
 // ---------------------------------------------------------------------------------------------------
 constexpr int kTcThreads = 352;       // warps 0-7: softmax; 8: issue of Q K^T, tensor-memory allocation; 9: TMA loads; 10: issue of P V
@@ -619,15 +620,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             mbar_init(bar_o + 1, 1);
             mbar_init(bar_p, 256);
             mbar_init(bar_p + 1, 256);
-            if (p.csize > 1) {
-                const int rank_ = split % p.csize;
-                const int r0 = min(Tpad, rank_ * p.rpr), r1 = min(Tpad, r0 + p.rpr);
-                mbar_init(rbar, 1);
-                mbar_fence_init();
-                mbar_expect_tx(rbar, (uint32_t)(r1 - r0) * REC * 4u * (uint32_t)p.csize);
-            } else {
-                mbar_fence_init();
-            }
+            mbar_fence_init();
         }
     }
     uint64_t ld_policy = 0;
@@ -646,7 +639,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    // every receiving barrier is armed before anybody can send: arrive here, wait just before the pushes
+    // nobody stores into a peer's shared memory before that CTA has started: arrive here, wait just before the deposit
     if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_wait();
     const uint32_t tbase = *tmem_slot;
@@ -836,16 +829,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             if (STREAM && b > 1 && ok) ok = mbar_wait(bar_p + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
             mbar_arrive(bar_p + (b & 1));
         }
-        // ---- this thread's half of the row's O, and the row's (m, l), into the CTA's deposit ----
+        // ---- this thread's half of the row's O, and the row's (m, l), go straight into the shared memory of the CTA
+        //      that merges the row: stores through distributed shared memory, made visible by the cluster barrier ----
         if (nb > 0) {
             if (ok) ok = mbar_wait(bar_o + ((nb - 1) & 1), (uint32_t)((nb - 1) >> 1) & 1u, wait_expired);
             tc_fence_after_sync();
         }
-        float* loc = reinterpret_cast<float*>(kv_s);            // [Tpad][REC], aliases the ring
+        if (p.csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA of the cluster has started
         if (act) {
             float* xl = xch + 512;                              // [2][128]
             xl[hf * 128 + row] = l_run;
-            float* wo = loc + (size_t)row * REC + hf * (HD / 2);
+            // the record of (part = this CTA, row): in the merging CTA's recv area, or, for a lone CTA, over the idle ring
+            const int dest = p.csize > 1 ? min(row / p.rpr, p.csize - 1) : 0;
+            const float* rec = p.csize > 1 ? recv + ((size_t)(split % p.csize) * p.rpr + (row - dest * p.rpr)) * REC
+                                           : reinterpret_cast<const float*>(kv_s) + (size_t)row * REC;
+            const uint32_t ra = cluster_map(smem_u32(rec), dest);
 #pragma unroll
             for (int c = 0; c < HD / 2; c += 16) {
                 float o[16];
@@ -857,11 +855,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 }
                 if (row < Tpad) {
 #pragma unroll
-                    for (int e = 0; e < 16; e += 4) *reinterpret_cast<float4*>(wo + c + e) = make_float4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+                    for (int e = 0; e < 16; e += 4)
+                        asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(ra + (uint32_t)(hf * (HD / 2) + c + e) * 4u), "f"(o[e]), "f"(o[e + 1]), "f"(o[e + 2]), "f"(o[e + 3]) : "memory");
                 }
             }
             pair_barrier(quad);
-            if (hf == 0 && row < Tpad) *reinterpret_cast<float2*>(loc + (size_t)row * REC + HD) = make_float2(m_run, l_run + xl[128 + row]);
+            if (hf == 0 && row < Tpad)
+                asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra + (uint32_t)HD * 4u), "f"(m_run), "f"(l_run + xl[128 + row]) : "memory");
         }
     }
     tc_fence_before_sync();
@@ -869,39 +870,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     const int rank = split % csize, outer = split / csize;
     const int n_parts = csize;
     const float* src_parts = reinterpret_cast<const float*>(kv_s);
-    const float* loc_c = src_parts;
     int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
     if (csize > 1) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the deposit is read by bulk copies
-        __syncthreads();
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // the peers' receiving barriers exist
-        if (warp == 8) {
-            tc_fence_after_sync();
-            tmem_dealloc(tbase, kTcCols);
-        } else if (lane == 0 && warp < n_parts) {       // one sender per destination, spread over the warps
-            const int dest = warp;
-            const int r0 = min(Tpad, dest * rpr), r1 = min(Tpad, r0 + rpr);
-            if (r1 > r0) {
-                const uint32_t bytes = (uint32_t)(r1 - r0) * REC * 4;
-                const uint32_t src = smem_u32(loc_c + (size_t)r0 * REC);
-                const uint32_t dst_local = smem_u32(recv + ((size_t)rank * rpr) * REC);
-                const uint32_t dst = cluster_map(dst_local, dest), bar = cluster_map(smem_u32(rbar), dest);
-                asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(dst), "r"(src), "r"(bytes), "r"(bar) : "memory");
-            }
-        }
+        // warps 0-7 have passed the first phase of the cluster barrier above; the second one publishes the records
+        if (warp >= 8) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         row0 = min(Tpad, rank * rpr);
         n_my = min(Tpad, row0 + rpr) - row0;
-        if (n_my > 0) mbar_wait(rbar, 0, wait_expired);
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // this CTA holds everything it needs
         src_parts = recv;
         part_stride = rpr * REC;
     } else {
         __syncthreads();
-        if (warp == 8) {
-            tc_fence_after_sync();
-            tmem_dealloc(tbase, kTcCols);
-        }
+    }
+    if (warp == 8) {
+        tc_fence_after_sync();
+        tmem_dealloc(tbase, kTcCols);
     }
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
     // One thread per (query row, 8 output columns): all rows of the CTA are merged at once, every load of a thread is
@@ -952,8 +936,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             if (c8 == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
-    // nobody leaves while a peer's copy may still be reading this CTA's deposit
-    if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
