@@ -1,7 +1,7 @@
 // Tree-masked attention of the T draft-tree nodes against the KV prefix plus their own ancestors.
 //
 // Two kernels: k_tree_attn (bf16 mma.sync; head_dim 64 or 128), described first, and k_tree_attn_tc (tcgen05, tensor
-// memory and TMA; head_dim 128), further down, which takes every tree of more than 16 nodes at head_dim 128.
+// memory and TMA), further down, which takes every head_dim-128 problem.
 //
 // Q [T_pad][hd] sits in shared memory; the cache rows stream through a double-buffered cp.async pipeline
 // (128-bit loads); S = Q K^T and O += P V run on bf16 tensor-core MMAs (fp32 accumulation, online softmax in
@@ -993,11 +993,10 @@ size_t attn_plan(AttnProblem& p) {
     // split each block of rows, and it finishes its own query rows alone: no exchange between CTAs at all.
     p.qsplit = 0;
     p.mt_per_cta = 0;
-    // The tcgen05 kernel (head_dim 128, positive scale) is ahead except for a single query tile over a cache of a few
-    // thousand rows, where seven eighths of its 128 MMA rows are padding (measured in the 7B forward at prefix 512: 3.13
-    // vs 3.12 ms at T = 16, 3.16 vs 3.22 at 32, 3.40 vs 3.48 at 64, 3.98 vs 4.14 at 128; alone at T = 16: 16.4 vs 14.9 us
-    // over 1024 rows, 27.4 vs 27.4 over 3900, 74 vs 81 over 16384; at T = 128 over 16384 rows: 85 vs 253 us).
-    p.use_tc = (p.hd == 128 && p.scale > 0.f && (tpad > 16 || S > 4096)) ? 1 : 0;
+    // The tcgen05 kernel takes every head_dim-128 problem with a positive scale (measured in the 7B forward at prefix 512
+    // against the mma.sync kernel: 3.07 vs 3.07 ms at T = 1, 3.09 vs 3.10 at 8, 3.11 vs 3.13 at 16, 3.15 vs 3.22 at 32,
+    // 3.40 vs 3.48 at 64, 3.96 vs 4.14 at 128; alone over 16384 rows: 74 vs 81 us at T = 16, 85 vs 253 us at T = 128).
+    p.use_tc = (p.hd == 128 && p.scale > 0.f) ? 1 : 0;
     if (attn_tc_override() >= 0) p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_override() == 1) ? 1 : 0;
     const int n_mt = tpad / 16;
     if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
