@@ -565,7 +565,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     uint8_t* kv_s = q_s + 128 * 256;                                             // ring of K and V blocks
     float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][2][128] row maxima (by block parity), [2][128] row sums
     float* recv = xch + 768;                                                     // [csize][rpr][REC]
-    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));
+    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // base of the mbarriers; slot 0 unused
     // Every barrier that a thread may find more than one phase ahead of itself would give a wrong answer to a parity
     // wait, so each one is either indexed by block parity (its next completion needs the waiter's own progress) or by
     // ring stage (the classical full / empty pair).
