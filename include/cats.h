@@ -13,8 +13,13 @@
  *
  * Conventions shared by every entry point
  *   - Pointers named d_* are DEVICE pointers; the caller owns every buffer.
- *     The library allocates no device memory and keeps no state besides
- *     function attributes set once per process.
+ *     The library allocates no device memory.  The state it keeps is host-side
+ *     and derived from arguments only: kernel attributes set once per process,
+ *     a cache of up to 256 encoded tensor maps keyed by (pointer, shape) for
+ *     the attention kernel, the per-device address of the scratch array of
+ *     cats_tree_attention_static, and the switches of include/cats_debug.h
+ *     (all at their defaults unless a test or a benchmark sets them).  No
+ *     environment variable is read.
  *   - `stream` is a cudaStream_t passed as void*.  Calls are asynchronous,
  *     never synchronise and never copy to the host (except the *_host entry
  *     point, which says so).
@@ -75,8 +80,8 @@ typedef struct {
 } cats_layer_weights;
 
 /* Weight packing.  The projections are bound by reading every weight once per
- * forward ("every generation step loads the model weights"; Eq. 3-4 count
- * exactly those bytes), so the library keeps each matrix as a sequence of
+ * forward (Section 1: decoding is bound by weight movement; the byte model of
+ * Eq. 3-4 counts exactly those bytes), so the library keeps each matrix as a sequence of
  * 16 KB chunks -- (128-row tile, 64-column block), already in the layout the
  * tensor cores read from shared memory -- that one SM can stream with plain
  * contiguous bulk copies.
@@ -92,9 +97,9 @@ size_t cats_packed_weight_bytes(int32_t n_src, int32_t layout, int32_t rows, int
 int cats_pack_weights(const void *const *d_src, int32_t n_src, int32_t layout, int32_t rows, int32_t cols,
                       void *d_dst, void *stream);
 
-/* Ancestor mask, depth and position ids of the draft tree ("tree-based
- * attention mask encoding the main draft sequence and SV correction branches",
- * Fig. 4; Algorithm 1, mask = T.tree_mask).
+/* Ancestor mask, depth and position ids of the draft tree (the tree attention
+ * mask of Fig. 4, which covers the main draft chain and the correction branches;
+ * Algorithm 1, Stage 3, mask = T.tree_mask).
  *   d_parent [T] int32 in.  d_mask [T][2] uint64 out: bit j of row i (word
  *   j>>6, bit j&63) is set iff j == i or j is an ancestor of i.  d_pos [T]
  *   int32 out = prefix_len + depth.  d_depth [T] int32 out, may be NULL.
@@ -116,8 +121,8 @@ int cats_embed_tokens(const void *d_embed, const int32_t *d_tokens, int32_t T, i
 size_t cats_workspace_bytes(const cats_model_cfg *cfg, int32_t T, int32_t max_prefix);
 
 /* One decoder layer over the T tree nodes under the tree mask (Algorithm 1,
- * Stage 3: H_tgt <- M_{L_SV+1:L_total}(T.hidden_states, mask, KV_M); "a single
- * batched forward pass under the corresponding tree attention mask").
+ * Stage 3: H_tgt <- M_{L_SV+1:L_total}(T.hidden_states, mask, KV_M); Section
+ * 3.2, final verification: all tree nodes go through the layers in one batch).
  *   d_resid [T][hidden] fp32, in/out: the residual stream.
  *   d_kcache/d_vcache: THIS layer's caches, bf16 [max_seq][n_heads*head_dim];
  *     rows [0,prefix_len) are read, rows prefix_len+i are written (k rotated).
@@ -128,8 +133,8 @@ int cats_verify_layer(const cats_model_cfg *cfg, const cats_layer_weights *w, fl
                       int32_t prefix_len, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
 
 /* The same layer over a SUBSET of the tree (Algorithm 1, Stage 2: the
- * correction tokens are re-forwarded through layers 1..L_SV "under tree-masked
- * attention" while the main-chain nodes already have their K/V in those
+ * correction tokens are re-forwarded through layers 1..L_SV with the tree mask
+ * applied, while the main-chain nodes already have their K/V in those
  * layers).
  *   d_nodes [m] int32, device: tree node indices, strictly ascending, in [0,T).
  *   d_resid [m][hidden] fp32 in/out: hidden states of those nodes only.
@@ -193,8 +198,8 @@ int cats_lm_head_argmax(const cats_model_cfg *cfg, const void *d_final_norm, con
                         const float *d_resid, int32_t T, float *d_logits, int32_t *d_argmax, void *d_ws,
                         size_t ws_bytes, int32_t *d_status, void *stream);
 
-/* Greedy longest-accepted-path walk and bonus token (Algorithm 1, "Walk the
- * tree to find the longest accepted prefix"; y_out and the bonus token).
+/* Greedy longest-accepted-path walk and bonus token (Algorithm 1, the walk
+ * step of Stage 3: y_out and the bonus token).
  * A child is accepted iff its token equals d_argmax at its parent; among equal
  * sibling tokens the lowest node index wins.
  *   d_path [T] out: accepted node indices, d_path[0] = 0; *d_path_len >= 1.
@@ -204,8 +209,8 @@ int cats_accept_path(const int32_t *d_parent, const int32_t *d_tokens, const int
                      int32_t *d_path, int32_t *d_path_len, int32_t *d_out_tokens, int32_t *d_n_out,
                      int32_t *d_status, void *stream);
 
-/* Typical (relaxed) acceptance, the second criterion Acc of Algorithm 1
- * ("greedy or typical"; the tables' relaxed setting at temperature 0.7), as the
+/* Typical (relaxed) acceptance, the second criterion Acc that Algorithm 1
+ * allows (the tables' relaxed setting at temperature 0.7), as the
  * cited Medusa work defines it: with p = softmax(logits / t) at the parent, a
  * child token x is acceptable iff  p(x) > min(eps, delta * exp(-H(p))).
  *
@@ -238,8 +243,8 @@ int cats_accept_path_typical(const int32_t *d_parent, const int32_t *d_tokens, c
                              int32_t *d_path_len, int32_t *d_out_tokens, int32_t *d_n_out,
                              int32_t *d_status, void *stream);
 
-/* KV roll-back along the accepted path (Algorithm 1, "Roll back KV_M ... to
- * length s along the accepted path"): for every layer, K and V, row
+/* KV roll-back along the accepted path (Algorithm 1, last step of the cycle):
+ * for every layer, K and V, row
  * prefix_len + d_path[k] moves to row prefix_len + k, in place;
  * *d_new_len = prefix_len + *d_path_len.  Caches are 16-bit elements laid out
  * [n_layers][layer_stride_elems]; a row has row_elems elements (multiple of 8).

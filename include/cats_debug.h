@@ -1,0 +1,57 @@
+/*
+ * cats_debug.h -- measurement and fault-injection hooks of libcats.
+ *
+ * These are not part of the product interface (include/cats.h): the benchmark
+ * uses them to time parts of a forward, the tests use them to reach code that
+ * normal operation never runs (the fallback attention kernel, the expiry of a
+ * bounded device-side wait).  All state is process-wide, host-side except the
+ * wait limit, and starts at the documented default.  None of them has a
+ * counterpart in the paper.
+ */
+#ifndef CATS_DEBUG_H_
+#define CATS_DEBUG_H_
+
+#include "cats.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Bit i of mask enables stage i of every decoder layer launched afterwards
+ * (0 norm1, 1 qkv, 2 attention, 3 o-proj, 4 norm2, 5 gate/up, 6 down).
+ * Default 0x7f: everything runs.  With stages disabled the results are
+ * meaningless; only the timing of what still runs is of interest. */
+void cats_debug_stage_mask(unsigned mask);
+
+/* Byte offsets of the intermediate buffers inside the workspace
+ * cats_workspace_bytes sizes: out[0..4] = xn, q, o, act (packed activation
+ * layout, except q: [T][n_heads*head_dim] bf16) and part (fp32 split-K partial
+ * sums [pieces][T][hidden]); out[5] = fp32 elements between two partial sums;
+ * out[6], out[7] = pieces written by the O and the down projection.
+ * out: HOST array of 8 size_t. */
+int cats_debug_workspace_layout(const cats_model_cfg *cfg, int32_t T, size_t *out);
+
+/* Attention kernel used for head_dim 128: -1 (default) chosen by shape, 0 the
+ * mma.sync kernel (the fallback when the driver offers no tensor maps), 1 the
+ * tcgen05 kernel. */
+void cats_debug_attention_kernel(int which);
+
+/* Limit of every bounded device-side wait, in nanoseconds, on the CURRENT
+ * device (0 restores the default of 1 s).  Synchronises the device. */
+int cats_debug_wait_limit_ns(unsigned long long ns);
+
+/* Fault injection, host-made: launches issued afterwards withhold one signal
+ * so that a bounded wait runs out (the kernel then reports CATS_ERR_TIMEOUT
+ * through *d_status and returns; nothing traps, nothing waits without limit).
+ *   0 none (default);
+ *   1 projection kernel: CTAs that contribute a partial tile to a tile another
+ *     CTA owns do not raise their ready flag;
+ *   2 tcgen05 attention kernel: the loader announces the query tile on its
+ *     barrier but never copies it.
+ * Set a short wait limit first, or each expiry takes a second. */
+void cats_debug_inject_fault(int which);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CATS_DEBUG_H_ */

@@ -26,7 +26,8 @@
  * deviation between contract mode and pure mode is "parity unpinned": the
  * paper states no tolerance for 16-bit inference.
  *
- * Build: gcc -O2 -fopenmp -shared -fPIC cats_ref.c -o libcats_ref.so -lm
+ * Build: gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC cats_ref.c -o libcats_ref.so -lm
+ * (no fused multiply-add: products and sums are rounded separately on every host)
  * OpenMP is used over independent output rows only.
  */
 #include <math.h>
@@ -200,8 +201,8 @@ int cats_ref_tree_attention(const double *q, const float *kc, const float *vc, c
 
 /* The same attention for nq query rows that need not be all T tree nodes: query
  * i carries its own 128-bit visibility row mask[i] over the T tree rows P..P+T-1
- * (Stage 2 of Algorithm 1 re-forwards only the correction nodes "under
- * tree-masked attention"; the other tree rows are already in the cache).
+ * (Stage 2 of Algorithm 1 re-forwards only the correction nodes, with the
+ * tree mask applied; the other tree rows are already in the cache).
  * q, out [nq][nh][hd]; probs (optional) [nh][nq][P+T]. */
 int cats_ref_tree_attention_rows(const double *q, const float *kc, const float *vc, const uint64_t *mask,
                                  int32_t nq, int32_t T, int32_t P, int32_t nh, int32_t hd,
@@ -253,8 +254,8 @@ int cats_ref_tree_attention_rows(const double *q, const float *kc, const float *
 static double silu(double x) { return x / (1.0 + exp(-x)); }
 
 /* ---- O3: one decoder layer over the T tree nodes (Algorithm 1, Stage 3:
- * "H_tgt <- M(T.hidden_states, mask=T.tree_mask, KV_M)"; "single batched
- * forward pass under the corresponding tree attention mask").
+ * H_tgt <- M(T.hidden_states, mask=T.tree_mask, KV_M); Section 3.2, final
+ * verification: all tree nodes in one batch under the tree mask).
  * resid [T][H] fp32 in/out.  kc, vc: this layer's caches, float
  * [max_seq][nh*hd]; rows [0,P) are the committed prefix, rows P+i are written
  * here.  q_out (optional) [T][nh*hd] fp64 receives the rotated, rounded q. */
@@ -307,8 +308,8 @@ int cats_ref_verify_layer(const cats_ref_cfg *cfg, const cats_ref_layer_weights 
 }
 
 /* ---- O3 over a subset of the tree (Algorithm 1, Stage 2: the correction
- * tokens are "re-forwarded from layer 1 through L_SV under tree-masked
- * attention"; the main-chain nodes already have their K/V in these layers).
+ * tokens go through layers 1..L_SV again with the tree mask applied; the
+ * main-chain nodes already have their K/V in these layers).
  * nodes[0..m) are tree node indices, strictly ascending; resid [m][H] holds the
  * hidden states of those nodes only.  The K/V of node nodes[j] is written to
  * cache row P + nodes[j]; every other cache row is read-only.  Node nodes[j]
@@ -399,8 +400,8 @@ int cats_ref_lm_head_argmax(const cats_ref_cfg *cfg, const uint16_t *final_norm,
     return 0;
 }
 
-/* ---- O5: greedy longest-accepted-path walk (Algorithm 1, "Walk the tree to
- * find the longest accepted prefix" and the bonus token).  A child is accepted
+/* ---- O5: greedy longest-accepted-path walk (Algorithm 1, the walk step
+ * of Stage 3, and the bonus token).  A child is accepted
  * iff its token equals the target's argmax at its parent; among equal sibling
  * tokens the lowest node index wins.  path[0] = 0 (root); out_tokens holds the
  * accepted draft tokens followed by the bonus token; n_out == path_len. */
@@ -553,8 +554,8 @@ int cats_ref_accept_path_typical(const int32_t *parent, const int32_t *tokens, c
     return walk_with_verdicts(parent, tokens, argmax, ok, T, path, path_len, out_tokens, n_out);
 }
 
-/* ---- O6: KV rollback along the accepted path (Algorithm 1, "Roll back KV_M
- * ... to length s along the accepted path").  For every layer, K and V: row
+/* ---- O6: KV rollback along the accepted path (Algorithm 1, last step of
+ * the cycle).  For every layer, K and V: row
  * P+path[k] moves to row P+k, k ascending, in place.  src/dst (optional)
  * receive the row index lists.  The cache element type is opaque: elem_bytes
  * bytes per element. */

@@ -182,6 +182,22 @@ def stage_mask(mask: int) -> None:
     lib.cats_debug_stage_mask(C.c_uint(mask))
 
 
+def attention_kernel(which: int) -> None:
+    """cats_debug_attention_kernel: -1 by shape (default), 0 the mma.sync kernel, 1 the tcgen05 kernel."""
+    lib.cats_debug_attention_kernel(C.c_int(which))
+
+
+def wait_limit_ns(ns: int) -> None:
+    """cats_debug_wait_limit_ns: limit of the bounded device-side waits on the current device (0: the default, 1 s)."""
+    _check(lib.cats_debug_wait_limit_ns(C.c_ulonglong(ns)), "cats_debug_wait_limit_ns")
+
+
+def inject_fault(which: int) -> None:
+    """cats_debug_inject_fault: 0 none, 1 a projection's contributors keep their ready flags, 2 the attention loader
+    never copies Q."""
+    lib.cats_debug_inject_fault(C.c_int(which))
+
+
 def workspace_layout(cfg: ModelCfg, T: int) -> dict:
     """Byte offsets of the intermediate buffers inside the workspace (for tests that inspect them)."""
     out = (C.c_size_t * 8)()

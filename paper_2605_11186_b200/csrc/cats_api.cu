@@ -8,6 +8,8 @@ namespace cats {
 
 thread_local int g_launch_count = 0;
 thread_local bool g_call_boundary = true;
+int g_debug_attn_kernel = -1;
+int g_debug_fault = 0;
 
 namespace {
 
@@ -210,12 +212,16 @@ const char* cats_status_string(int s) {
 
 int cats_last_launch_count(void) { return g_launch_count; }
 
-/* Bring-up / measurement hooks, not part of the public header.  cats_debug_stage_mask: bit i enables
- * stage i of every decoder layer (0 norm1, 1 qkv, 2 attention, 3 o-proj, 4 norm2, 5 gate/up, 6 down);
- * 0x7f restores normal operation.  cats_debug_workspace_layout: byte offsets of the intermediate
- * buffers inside the workspace: xn, q, o, act, part (fp32 split-K partial sums), and in out[5] the
- * number of fp32 elements between two partial sums. */
+/* Measurement and fault-injection hooks, declared in include/cats_debug.h. */
 void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
+void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which ? 1 : 0); }
+void cats_debug_inject_fault(int which) { g_debug_fault = (which == 1 || which == 2) ? which : 0; }
+int cats_debug_wait_limit_ns(unsigned long long ns) {
+    if (ns == 0) ns = kWaitLimitNs;
+    if (set_wait_limit_gemm(ns) != cudaSuccess || set_wait_limit_attn(ns) != cudaSuccess || set_wait_limit_small(ns) != cudaSuccess)
+        return CATS_ERR_CUDA;
+    return CATS_OK;
+}
 int cats_debug_workspace_layout(const cats_model_cfg* cfg, int32_t T, size_t* out) {
     if (check_cfg(cfg) != CATS_OK || T < 1 || T > CATS_MAX_TREE || !out) return CATS_ERR_INVALID_ARG;
     Workspace w = carve(cfg, T, nullptr);
@@ -422,7 +428,7 @@ int cats_accept_path(const int32_t* d_parent, const int32_t* d_tokens, const int
     if (!d_parent || !d_tokens || !d_argmax || !d_path || !d_path_len || !d_out_tokens || !d_n_out || !d_status)
         return CATS_ERR_INVALID_ARG;
     if (T < 1 || T > CATS_MAX_TREE) return CATS_ERR_INVALID_ARG;
-    CATS_CUDA(launch_walk(d_parent, d_tokens, d_argmax, T, d_path, d_path_len, d_out_tokens, d_n_out, (cudaStream_t)stream));
+    CATS_CUDA(launch_walk(d_parent, d_tokens, d_argmax, T, d_path, d_path_len, d_out_tokens, d_n_out, d_status, (cudaStream_t)stream));
     return CATS_OK;
 }
 
@@ -486,7 +492,7 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
         CATS_CUDA(launch_walk_typical(d_parent, d_tokens, a->d_argmax, ty.cand, ty.lse, ty.entropy, T, a->inv_temperature,
                                       a->log_eps, a->log_delta, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
     else
-        CATS_CUDA(launch_walk(d_parent, d_tokens, a->d_argmax, T, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, st));
+        CATS_CUDA(launch_walk(d_parent, d_tokens, a->d_argmax, T, a->d_path, a->d_scalars + 0, a->d_out_tokens, a->d_scalars + 1, a->d_status, st));
     if (a->compact)
         CATS_CUDA(launch_compact(a->d_kcache, a->d_vcache, c->n_layers, (long long)lstride, (long long)c->n_heads * c->head_dim, P,
                                  a->d_path, a->d_scalars + 0, a->d_scalars + 2, nullptr, nullptr, a->d_status, st));

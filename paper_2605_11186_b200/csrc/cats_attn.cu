@@ -67,6 +67,7 @@ struct AttnDev {
     uint16_t* out;
     float* part_o;       // n_outer > 1: [nh][n_outer][T_pad][hd] fp32
     float* part_ml;      //              [nh][n_outer][T_pad][2]
+    int dbg_skip_q;      // fault injection (tcgen05 kernel): the loader announces Q but never copies it
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -703,7 +704,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         // ---- loader: Q and the boxes that depend on the previous kernel, then a refill whenever a P V product frees a stage ----
         if (lane == 0) {
             if (nb > 0) mbar_expect_tx(bar_q, 128u * 256u);
-            for (int rb = 0; rb < 128 && nb > 0; rb += kTcBoxRows) {
+            for (int rb = 0; rb < 128 && nb > 0 && !p.dbg_skip_q; rb += kTcBoxRows) {
                 tma_load_2d(q_s + (size_t)rb * 128, &tm_q, h * HD, rb, bar_q, ld_policy);
                 tma_load_2d(q_s + 128 * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
             }
@@ -966,11 +967,10 @@ __global__ void __launch_bounds__(128) k_attn_combine(const float* __restrict__ 
 
 // Chooses the cluster size (CTAs per head that share one merge through distributed shared memory) and, for long
 // prefixes with few heads, the number of clusters per head.  Returns the bytes of workspace the outer merge needs.
-// CATS_ATTN_TC=0 / 1 forces the mma.sync / the tcgen05 kernel (for measurements); unset: chosen by shape.
-static int attn_tc_override() {
-    static const int v = [] { const char* e = getenv("CATS_ATTN_TC"); return e == nullptr ? -1 : (e[0] == '1' ? 1 : 0); }();
-    return v;
-}
+// cats_debug_attention_kernel(0 / 1) forces the mma.sync / the tcgen05 kernel (for measurements and for testing the
+// fallback); -1, the default: chosen by shape.
+static int attn_tc_override() { return g_debug_attn_kernel; }
+cudaError_t set_wait_limit_attn(unsigned long long ns) { return cudaMemcpyToSymbol(g_wait_limit_ns, &ns, sizeof(ns)); }
 
 size_t attn_plan(AttnProblem& p) {
     const int S = p.prefix_len + (p.T_tree > 0 ? p.T_tree : p.T);
@@ -1118,6 +1118,7 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     d.out_npad = p.out_packed_npad;
     d.part_o = p.part_o; d.part_ml = p.part_ml;
     d.d_status = p.d_status;
+    d.dbg_skip_q = g_debug_fault == 2 ? 1 : 0;
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
@@ -1287,9 +1288,11 @@ extern "C" int cats_tree_attention_static(const void* d_q, const void* d_k, cons
     a.kv_stride = kv_row_stride_elems; a.scale = scale; a.out = d_out; a.d_status = d_status;
     const size_t need = attn_plan(a);
     if (need > kStaticScratchBytes) return CATS_ERR_WORKSPACE;   // the problem needs more scratch than the library carries
+    // Looked up on every call that passes the checks, whether or not this problem needs scratch, so that the FIRST
+    // accepted call on a device always does the per-device set-up (a small warm-up call is enough).
+    void* base = nullptr;
+    if (static_scratch_address(&base) != cudaSuccess) return CATS_ERR_CUDA;
     if (need > 0) {
-        void* base = nullptr;
-        if (static_scratch_address(&base) != cudaSuccess) return CATS_ERR_CUDA;
         const int tpad = (T + 15) / 16 * 16;
         a.part_o = static_cast<float*>(base);
         a.part_ml = a.part_o + (size_t)n_heads * a.n_splits * tpad * head_dim;

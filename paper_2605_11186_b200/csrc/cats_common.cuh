@@ -12,6 +12,9 @@ namespace cats {
 
 constexpr int kMaxTree = CATS_MAX_TREE;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;  // every device-side wait gives up after 1 s
+// The limit the waits of this translation unit actually use (one copy per .cu file, each with a host-side setter that
+// the fault-injection hook cats_debug_wait_limit_ns calls); read on the slow path of a wait only.
+static __device__ unsigned long long g_wait_limit_ns = kWaitLimitNs;
 
 __device__ __forceinline__ void report(int32_t* d_status, int code) {
     if (d_status) atomicMin(d_status, code);
@@ -83,7 +86,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (globaltimer_ns() - t0 > g_wait_limit_ns) {
                 *abort_flag = 1;
                 return false;
             }

@@ -69,6 +69,7 @@ struct GemmDev {
     int warm_chunks;             // 16 KB chunks to pull through a landing buffer (warms L2)
     int warm_upc, warm_n_ku, warm_n_kb;
     long long warm_total_chunks;
+    int dbg_skip_publish;        // fault injection: contributors of shared tiles keep their flags to themselves
 };
 
 struct GemmCtrl {
@@ -339,7 +340,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                     unsigned long long t0 = globaltimer_ns();
                     for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
                         while (ld_acquire(p.fix_flags + c2) == 0) {
-                            if (*abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+                            if (*abort_flag || globaltimer_ns() - t0 > g_wait_limit_ns) { *abort_flag = 1; break; }
                         }
                     }
                 }
@@ -384,7 +385,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
                 store_tile_transposed(taddr, p.n_pad, p.n_pad, acc_s, f, et, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
                 __threadfence();
                 epi_barrier();
-                if (et == 0) st_release(p.fix_flags + my_slot, 1);
+                if (et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
             } else {
                 // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
 #pragma unroll
@@ -639,6 +640,8 @@ cudaError_t launch_pack_weights(const void* const* src, int n_src, int layout, i
 // ---------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------
+cudaError_t set_wait_limit_gemm(unsigned long long ns) { return cudaMemcpyToSymbol(g_wait_limit_ns, &ns, sizeof(ns)); }
+
 int gemm_num_tiles(const GemmProblem& p) {
     if (p.epi == EPI_SWIGLU) return (p.n_out + 63) / 64;
     return p.n_mats * ((p.n_out + 127) / 128);
@@ -776,6 +779,7 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.tree_tokens = p.tree_tokens;
     d.cand = p.cand;
     d.d_status = p.d_status;
+    d.dbg_skip_publish = g_debug_fault == 1 ? 1 : 0;
     d.warm_ptr = nullptr;
     d.warm_chunks = 0;
     if (p.warm_next != nullptr && p.warm_next->W[0] != nullptr) {

@@ -14,6 +14,13 @@ extern thread_local int g_launch_count;
 // prefetch) can overlap work issued by earlier calls.
 extern thread_local bool g_call_boundary;
 
+// Measurement / fault-injection state set through the cats_debug_* hooks (include/cats_debug.h); process-wide.
+extern int g_debug_attn_kernel;   // -1: attention kernel chosen by shape; 0: mma.sync kernel; 1: tcgen05 kernel
+extern int g_debug_fault;         // 0: none; 1: a helper CTA of a projection never publishes; 2: the attention loader drops Q
+cudaError_t set_wait_limit_gemm(unsigned long long ns);
+cudaError_t set_wait_limit_attn(unsigned long long ns);
+cudaError_t set_wait_limit_small(unsigned long long ns);
+
 // Launch with programmatic stream serialization: the kernel may start while its predecessor in the
 // stream is still draining; every kernel calls griddepcontrol.wait before touching dependent data.
 template <typename... KArgs, typename... Args>
@@ -56,7 +63,7 @@ cudaError_t launch_walk_typical(const int32_t* parent, const int32_t* tokens, co
                                 float log_delta, int32_t* path, int32_t* path_len, int32_t* out_tokens, int32_t* n_out,
                                 cudaStream_t st);
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
-                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, cudaStream_t st);
+                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_stride, long long row_elems, int prefix_len,
                            const int32_t* path, const int32_t* path_len, int32_t* new_len, int32_t* src_rows,
                            int32_t* dst_rows, int32_t* d_status, cudaStream_t st);

@@ -260,20 +260,25 @@ __global__ void __launch_bounds__(128) k_head_reduce(const float* __restrict__ p
 __global__ void __launch_bounds__(32) k_walk(const int32_t* __restrict__ parent, const int32_t* __restrict__ tokens,
                                              const int32_t* __restrict__ amax, int T, int32_t* __restrict__ path,
                                              int32_t* __restrict__ path_len, int32_t* __restrict__ out_tokens,
-                                             int32_t* __restrict__ n_out) {
+                                             int32_t* __restrict__ n_out, int32_t* d_status) {
     pdl_launch_dependents();
     pdl_wait();
     int lane = threadIdx.x;
     int par[4], tok[4];
+    bool bad = false;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         int j = q * 32 + lane;
         par[q] = j < T ? parent[j] : -2;
         tok[q] = j < T ? tokens[j] : -1;
+        // Only an edge parent[j] < j can be followed, so the path is strictly increasing and never
+        // longer than T whatever the array holds; a malformed entry is reported and leads nowhere.
+        if (j < T && (j == 0 ? par[q] != -1 : (par[q] < 0 || par[q] >= j))) { bad = true; par[q] = -2; }
     }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) report(d_status, CATS_ERR_BAD_TREE);
     int cur = 0, len = 1, no = 0;
     if (lane == 0) path[0] = 0;
-    for (int step = 0; step < T; ++step) {   // a path has at most T nodes
+    for (int step = 0; step + 1 < T; ++step) {   // a path has at most T nodes
         int want = amax[cur];
         int next = -1;
 #pragma unroll
@@ -408,6 +413,8 @@ __global__ void __launch_bounds__(256) k_compact(uint16_t* __restrict__ kc, uint
 // ---------------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------------
+cudaError_t set_wait_limit_small(unsigned long long ns) { return cudaMemcpyToSymbol(g_wait_limit_ns, &ns, sizeof(ns)); }
+
 // The same operation with the row held in registers and no dynamic shared memory, one row per CLUSTER of cs CTAs
 // (cs = 1, 2 or 4): CTA `rank` owns columns [rank, rank + 1) * H / cs, NC float4 per thread, so that all loads of a
 // thread are in flight at once; the sums of squares meet through distributed shared memory, added in rank order.
@@ -638,8 +645,8 @@ cudaError_t launch_walk_typical(const int32_t* parent, const int32_t* tokens, co
 }
 
 cudaError_t launch_walk(const int32_t* parent, const int32_t* tokens, const int32_t* amax, int T, int32_t* path,
-                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, cudaStream_t st) {
-    return launch_pdl(k_walk, dim3(1), dim3(32), 0, st, parent, tokens, amax, T, path, path_len, out_tokens, n_out);
+                        int32_t* path_len, int32_t* out_tokens, int32_t* n_out, int32_t* d_status, cudaStream_t st) {
+    return launch_pdl(k_walk, dim3(1), dim3(32), 0, st, parent, tokens, amax, T, path, path_len, out_tokens, n_out, d_status);
 }
 
 cudaError_t launch_compact(void* kc, void* vc, int n_layers, long long layer_stride, long long row_elems, int prefix_len,

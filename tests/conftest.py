@@ -12,6 +12,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_sessionstart(session):
+    # A child run of the suite may ask for one attention kernel (tests/test_gpu_attention_fallback.py).
+    which = os.environ.get("CATS_TEST_ATTENTION_KERNEL")
+    if which is not None:
+        import torch
+        if torch.cuda.is_available():
+            from paper_2605_11186_b200 import binding
+            binding.attention_kernel(int(which))
+
+
 def pytest_collection_modifyitems(config, items):
     import torch
     if torch.cuda.is_available():

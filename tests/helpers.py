@@ -86,3 +86,29 @@ def planted_tree(cfg, nm, T, k, root_token, P, kc, vc, seed_key, p_keep=0.7):
             for r, c in enumerate(kids):
                 tokens[c] = order[start + r]
     return parent_full, tokens
+
+
+def assert_bf16_output_close(name, got, want, tol, frac_limit=0.02):
+    """A bf16 output against the oracle's values: the stated absolute tolerance, and -- the bound that still bites
+    when the values themselves are small, as attention outputs over long prefixes are -- every element within one
+    bf16 ulp (at the larger magnitude) plus 1e-3 of the largest expected value, and only a small fraction of the
+    elements differing at all.  Returns (max-abs-err, max |want|) for the caller's report."""
+    g = np.asarray(got, np.float64)
+    w = np.asarray(want, np.float64)
+    wmax = float(np.abs(w).max())
+    d = np.abs(g - w)
+    err = float(d.max())
+    assert err <= tol, "%s: max-abs-err %g > %g (max |want| %g)" % (name, err, tol, wmax)
+    wb = w.astype(np.float32).astype(np.float64)
+    mag = np.maximum(np.abs(g), np.abs(wb))
+    ulp = 2.0 ** (np.floor(np.log2(np.maximum(mag, 1e-30))) - 7)
+    bad = d > ulp * 1.001 + 1e-3 * wmax
+    assert not bad.any(), "%s: %d elements off by more than one bf16 ulp, max-abs-err %g, max |want| %g" % (
+        name, int(bad.sum()), err, wmax)
+    # elements that differ from the oracle's value rounded to bf16
+    import torch
+    w16 = torch.from_numpy(w.astype(np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
+    frac = float((g != w16).mean())
+    assert frac < frac_limit, "%s: %.2f %% of the elements differ from the rounded oracle value" % (name, 100 * frac)
+    print("%s: max-abs-err %.3g, max |want| %.3g, %.2f %% of elements differ" % (name, err, wmax, 100 * frac))
+    return err, wmax

@@ -8,9 +8,14 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "cats.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(cats_[a-z_0-9]+)\s*\(", text)))
+    """Every function declared in include/*.h (the product header and the debug-hook header)."""
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in sorted(os.listdir(inc)):
+        if f.endswith(".h"):
+            text = re.sub(r"/\*.*?\*/", "", open(os.path.join(inc, f)).read(), flags=re.S)
+            names |= set(re.findall(r"\b(cats_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def _lib():
@@ -18,7 +23,7 @@ def _lib():
     return C.CDLL(build.build())
 
 
-def test_header_declares_the_five_north_star_calls():
+def test_header_declares_the_five_core_calls():
     names = _declared_functions()
     for n in ("cats_build_tree_mask", "cats_verify_layer", "cats_tree_attention", "cats_accept_path", "cats_compact_kv"):
         assert n in names

@@ -135,6 +135,46 @@ def test_linear_matches_torch_matmul():
     assert np.abs(oracle.linear(Wsq, xs) - (torch.from_numpy(xs) @ wf).numpy()).max() > 1e-3
 
 
+def test_linear_fp32_accumulation_mode_is_a_sequential_float32_sum():
+    """The oracle's fp32-accumulation mode (set_accum32) sets the noise floor that the deep-stack GPU tests report
+    beside their errors, so it is pinned like any other function: every output must equal, bit for bit, a float32
+    running sum over ascending k of separately rounded float32 products (written here with numpy scalars); and it must
+    sit at the distance from the fp64 sum that float32 rounding of ~K terms predicts, not at zero and not far away."""
+    rng = np.random.default_rng(33)
+    n_out, K, T = 11, 300, 5
+    W = oracle.to_bf16(rng.standard_normal((n_out, K)).astype(np.float32))
+    x = rng.standard_normal((T, K))
+    want64 = oracle.linear(W, x)
+    oracle.set_accum32(True)
+    try:
+        got = oracle.linear(W, x)
+    finally:
+        oracle.set_accum32(False)
+    Wf = oracle.from_bf16(W)
+    xf = x.astype(np.float32)
+    want = np.zeros((T, n_out), np.float32)
+    for t in range(T):
+        for o in range(n_out):
+            acc = np.float32(0.0)
+            for k in range(K):
+                acc = np.float32(acc + np.float32(Wf[o, k] * xf[t, k]))
+            want[t, o] = acc
+    assert np.array_equal(got.astype(np.float32), want) and np.array_equal(got, want.astype(np.float64))
+    # a descending-k or pairwise sum would differ in the last bits of most outputs
+    rev = np.zeros((T, n_out), np.float32)
+    for t in range(T):
+        for o in range(n_out):
+            acc = np.float32(0.0)
+            for k in range(K - 1, -1, -1):
+                acc = np.float32(acc + np.float32(Wf[o, k] * xf[t, k]))
+            rev[t, o] = acc
+    assert not np.array_equal(rev, want)
+    # distance from the fp64 sum: inputs rounded to float32 plus ~K float32 additions of terms of size ~1
+    d = np.abs(got - want64).max()
+    assert 1e-7 < d < 2e-4, d
+    assert np.array_equal(oracle.linear(W, x), want64)      # the switch is off again
+
+
 def test_rope_closed_forms():
     rng = np.random.default_rng(4)
     hd = 64
