@@ -32,7 +32,11 @@ METRIC = "verified tree tokens/sec per forward (7B-shape)"
 UNIT = "tree tokens/s"
 PREFIX = 512
 SWEEP = (16, 32, 64, 128)
-NCU_TRAFFIC_PER_LAUNCH = (32 * (113.7e6 + 42.5e6 + 195.5e6 + 95.6e6) + 272e6) / 129
+# dram__bytes_read + dram__bytes_write of the four projection launches of a layer at T=64, from the ncu capture of a
+# 2-layer stack summarised under profiles/ (QKV 109.7+3.8, O 42.5+0.0, gate/up 189.2+4.8, down 91.6+3.3 MB), scaled to the
+# 128 layer launches of a forward; the LM head (not captured) is counted at its packed size.
+NCU_TRAFFIC_PER_LAUNCH = (32 * (113.5e6 + 42.5e6 + 194.0e6 + 94.9e6) + 262.1e6) / 129
+TARGET_FORWARD_FRAC_OF_8TBS = 0.70
 
 
 # --------------------------------------------------------------------------------------------------
@@ -304,7 +308,9 @@ def run_ours(args, rank, world, local_rank):
                 r, _, _, _ = measure(T_, max(5, args.steps // 2), 3, with_breakdown=False)
             b = roofline.forward_bytes(shape, PREFIX, T_)
             sweep[str(T_)] = {"tok_s": T_ / r["sec_per_step"], "ms": r["sec_per_step"] * 1e3,
-                              "gbs": b / r["sec_per_step"] / 1e9, "accepted": r["accepted"]}
+                              "gbs": b / r["sec_per_step"] / 1e9, "accepted": r["accepted"],
+                              "forward_frac_of_measured": b / r["sec_per_step"] / 1e9 / measured_peaks()[0],
+                              "forward_frac_of_8TBs": b / r["sec_per_step"] / 8e12}
 
     # the rows built after the greedy path: the same forward under typical acceptance (softmax statistics in the LM-head
     # epilogue, relaxed walk), and the draft-stage shape (a one-token pass, the other weight-streaming loop of a cycle)
@@ -351,12 +357,13 @@ def run_ours(args, rank, world, local_rank):
         "roofline": {"bound": "hbm", "kernel": "k_gemm_sk (all %d projection launches of a forward)" % n_gemm,
                      "achieved": wb / n_gemm / (gemm_sec / n_gemm) / 1e9, "peak": peak, "unit": "GB/s",
                      "frac": wb / gemm_sec / 1e9 / peak, "peak_kind": peak_kind,
-                     # dram__bytes_read + write per launch from the ncu capture of a 2-layer stack (profiles/k_gemm_sk_7b_T64.md),
-                     # scaled to the 129 launches of a forward: 32 x (113.7 + 42.5 + 195.5 + 95.6) MB + LM head
                      "traffic": NCU_TRAFFIC_PER_LAUNCH if T == 64 else None,
                      "bytes_per_launch": wb / n_gemm, "us_per_launch": gemm_sec / n_gemm * 1e6,
                      "forward_achieved": fb / sec_step / 1e9, "forward_frac": fb / sec_step / 1e9 / peak,
-                     "forward_frac_of_8TBs": fb / sec_step / 8e12},
+                     "forward_frac_of_8TBs": fb / sec_step / 8e12,
+                     # the stated goal is on the WHOLE forward against the nominal 8 TB/s, not on the projections alone
+                     "target_forward_frac_of_8TBs": TARGET_FORWARD_FRAC_OF_8TBS,
+                     "target_met": bool(fb / sec_step / 8e12 >= TARGET_FORWARD_FRAC_OF_8TBS)},
         "breakdown_ms": {k: v * 1e3 for k, v in main["breakdown"].items()},
         "sweep": sweep,
         "widening": widening,
@@ -369,58 +376,85 @@ def run_ours(args, rank, world, local_rank):
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------------
 
-def oracle_sample(T, n_layers_sample, repeats=1):
-    """Times the oracle, as it stands, on a bounded sample of the workload: the first n_layers_sample layers plus the
-    LM head; the layer time is scaled to 32 layers.  Returns (seconds per full forward, cores, description)."""
+_ORACLE_INPUTS = {}
+
+
+def oracle_sample(T, n_layers_sample):
+    """Times the oracle, as it stands, on the first n_layers_sample decoder layers plus the LM head, the walk and the
+    compaction of the benchmark's workload (weights of one layer at a time, generated outside the timed parts).
+    Returns (seconds of the sampled work, seconds per full forward -- the layer time scaled to 32 layers when fewer
+    were run --, cores, description)."""
     import oracle
     shape = gen.LLAMA_7B
-    m = shape.replace(n_layers=n_layers_sample)
-    model = gen.make_model(m, ("bench", 0), device="cpu")
+    n = n_layers_sample
     max_seq = PREFIX + 128
-    kc, vc = gen.make_kv_prefix(m, n_layers_sample, max_seq, PREFIX, ("bench", 0))
     parent, _ = gen.tree_topk_shape(T, gen.topk_k_for(T))
-    tokens = gen.uniform_tokens(T, m.vocab, "bench_tokens", T)
-    layers = [{k: gen.bf16_bits(v) for k, v in w.items()} for w in model["layers"]]
-    cfg = oracle.RefCfg(m.hidden, m.n_heads, m.head_dim, m.ffn, m.vocab, n_layers_sample, max_seq, m.rms_eps, m.rope_base)
-    cfg0 = oracle.RefCfg(m.hidden, m.n_heads, m.head_dim, m.ffn, m.vocab, 0, max_seq, m.rms_eps, m.rope_base)
-    emb, fn, wl = gen.bf16_bits(model["embed"]), gen.bf16_bits(model["final_norm"]), gen.bf16_bits(model["w_lm"])
-    r_k, r_v = kc.float().numpy(), vc.float().numpy()
-    best_full, best_head = None, None
-    for _ in range(repeats):
+    tokens = gen.uniform_tokens(T, shape.vocab, "bench_tokens", T)
+    cfg = oracle.RefCfg(shape.hidden, shape.n_heads, shape.head_dim, shape.ffn, shape.vocab, n, max_seq, shape.rms_eps, shape.rope_base)
+    if "head" not in _ORACLE_INPUTS:          # generated once per process, outside every timed part
+        head = gen.make_model(shape.replace(n_layers=0), ("bench", 0), device="cpu")
+        _ORACLE_INPUTS["head"] = (gen.bf16_bits(head["embed"]), gen.bf16_bits(head["final_norm"]), gen.bf16_bits(head["w_lm"]))
+    emb, fn, wl = _ORACLE_INPUTS["head"]
+    if ("kv", n) not in _ORACLE_INPUTS:
+        kc, vc = gen.make_kv_prefix(shape, n, max_seq, PREFIX, ("bench", 0))
+        _ORACLE_INPUTS[("kv", n)] = (kc.float().numpy(), vc.float().numpy())
+    r_k, r_v = (a.copy() for a in _ORACLE_INPUTS[("kv", n)])
+    t_layers = 0.0
+    t0 = time.perf_counter()
+    _, mask, pos, _ = oracle.build_tree_mask(parent, PREFIX)
+    resid = oracle.embed(emb, tokens)
+    t_rest = time.perf_counter() - t0
+    for l in range(n):
+        if n <= 2 and ("layer", l) in _ORACLE_INPUTS:
+            w = _ORACLE_INPUTS[("layer", l)]
+        else:
+            w = {k: gen.bf16_bits(v) for k, v in gen.make_layer(shape, ("bench", 0), l).items()}
+            if n <= 2:
+                _ORACLE_INPUTS[("layer", l)] = w
         t0 = time.perf_counter()
-        _, amax, _, _ = oracle.verify_forward(cfg, layers, emb, fn, wl, parent, tokens, PREFIX, r_k, r_v, want_logits=False)
-        path, _ = oracle.accept_path(parent, tokens, amax)
-        oracle.compact_kv(r_k.copy(), r_v.copy(), PREFIX, path)
-        t_full = time.perf_counter() - t0
-        t0 = time.perf_counter()
-        oracle.verify_forward(cfg0, [], emb, fn, wl, parent, tokens, PREFIX, r_k[:0], r_v[:0], want_logits=False)
-        t_head = time.perf_counter() - t0
-        best_full = t_full if best_full is None else min(best_full, t_full)
-        best_head = t_head if best_head is None else min(best_head, t_head)
-    t_layers = max(best_full - best_head, 1e-9)
-    sec = t_layers * (shape.n_layers / n_layers_sample) + best_head
-    desc = ("oracle timed on %d of 32 layers + LM head + walk + compaction at T=%d, layer time scaled x%d"
-            % (n_layers_sample, T, shape.n_layers // n_layers_sample))
-    return sec, oracle.n_threads(), desc
+        oracle.verify_layer(cfg, w, resid, r_k[l], r_v[l], mask, pos, PREFIX)
+        t_layers += time.perf_counter() - t0
+        del w
+    t0 = time.perf_counter()
+    _, amax, _ = oracle.lm_head_argmax(cfg, fn, wl, resid, want_logits=False)
+    path, _ = oracle.accept_path(parent, tokens, amax)
+    oracle.compact_kv(r_k, r_v, PREFIX, path)
+    t_rest += time.perf_counter() - t0
+    sampled = t_layers + t_rest
+    full = t_layers * (shape.n_layers / n) + t_rest
+    if n == shape.n_layers:
+        desc = "one full pass of the oracle: 32 layers + LM head + walk + compaction at T=%d" % T
+    else:
+        desc = ("oracle timed on %d of 32 layers + LM head + walk + compaction at T=%d; layer time scaled x%g to a full forward"
+                % (n, T, shape.n_layers / n))
+    return sampled, full, oracle.n_threads(), desc
 
 
 def run_reference(args):
+    """The oracle as the reference arm.  A step is a bounded sample of the workload (2 of the 32 layers + the LM head +
+    walk + compaction): ms_per_step is the time that sample really took, value the throughput of a full forward with the
+    layer time scaled to 32 layers (stated in cpu_baseline.kind)."""
     T = args.tree_size
-    secs = []
+    n_sample = 2
+    sampled, fulls = [], []
     cores, desc = None, None
     for i in range(args.warmup + args.steps):
-        sec, cores, desc = oracle_sample(T, 1)
+        s_, f_, cores, desc = oracle_sample(T, n_sample)
         if i >= args.warmup:
-            secs.append(sec)
-    sec = float(np.mean(secs))
+            sampled.append(s_)
+            fulls.append(f_)
+    sec = float(np.mean(fulls))
     val = T / sec
     return {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "warmup": args.warmup, "ms_per_step": float(np.mean(sampled)) * 1e3, "extrapolated_ms_per_forward": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
             "config": {"workload": "cfg3: 32-layer 7B-shaped verification forward + LM head (vocab 32000), prefix 512, "
                                    "top-k draft tree of T=%d nodes, greedy walk + KV compaction" % T, "tree_nodes": T,
                        "prefix_len": PREFIX},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores,
+                             "kind": "oracle (extrapolated: %d of 32 layers timed per step, layer time scaled x%d)" % (n_sample, 32 // n_sample),
+                             "sample": desc},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
 
@@ -456,7 +490,7 @@ def main():
     out = run_ours(args, rank, world, local_rank)
     if rank == 0:
         if not args.no_cpu_baseline:
-            sec, cores, desc = oracle_sample(args.tree_size, 2)
+            _, sec, cores, desc = oracle_sample(args.tree_size, gen.LLAMA_7B.n_layers)       # one full pass, about half a minute
             out["cpu_baseline"] = {"value": args.tree_size / sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
         print(json.dumps(out), flush=True)
     if world > 1:

@@ -24,7 +24,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + ".tmp.%d" % os.getpid()
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        [os.path.join(CSRC, f) for f in SOURCES] + ["-o", tmp]
+        [os.path.join(CSRC, f) for f in SOURCES] + ["-ldl", "-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

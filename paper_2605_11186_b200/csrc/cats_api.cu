@@ -2,6 +2,8 @@
 // tree-verification forward.  See include/cats.h for the contract of every entry point.
 #include <cstring>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "cats_kernels.cuh"
 
 namespace cats {
@@ -10,6 +12,7 @@ thread_local int g_launch_count = 0;
 thread_local bool g_call_boundary = true;
 int g_debug_attn_kernel = -1;
 int g_debug_fault = 0;
+int g_debug_chain = 0;
 
 namespace {
 
@@ -18,6 +21,12 @@ namespace {
 // 3 o-proj, 4 norm2, 5 gate/up, 6 down).  All stages run by default.
 unsigned g_stage_mask = 0x7f;
 inline bool stage_on(int i) { return (g_stage_mask >> i) & 1u; }
+
+// One NVTX range per public call (visible in a timeline tool; a no-op when none is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -64,7 +73,7 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     w.psum = (float*)take((size_t)vt * 128 * 4);
     w.ps1 = (float*)take((size_t)vt * 128 * 4);
     w.fix_part = (float*)take((size_t)kFixSlots * tpad * 128 * 4);
-    w.fix_flags = (int*)take((size_t)kFixSlots * sizeof(int));
+    w.fix_flags = (int*)take((size_t)(kFixSlots + kChainSyncInts) * sizeof(int));   // the chained launch's counters follow the flags
     w.scratch = (float*)take((size_t)T * c->hidden * 4);
     w.nodes = (int32_t*)take((size_t)CATS_MAX_TREE * sizeof(int32_t));
     w.bytes = off;
@@ -101,7 +110,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
+                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots + kChainSyncInts, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -120,35 +129,37 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     attn_plan(a);
     if (stage_on(2)) CATS_CUDA(launch_tree_attention(a, st));
 
-    g = GemmProblem{};
-    g.epi = EPI_PARTIAL; g.T = T; g.K = D; g.n_out = H; g.n_mats = 1; g.W[0] = w->wo; g.X = ws.o;
-    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    int pieces_o = gemm_plan(g).max_pieces;
-    nxt = GemmProblem{};
-    nxt.epi = EPI_SWIGLU; nxt.T = T; nxt.K = H; nxt.n_out = F; nxt.n_mats = 2; nxt.W[0] = w->w_gate_up;
-    g.warm_next = &nxt;
-    if (stage_on(3)) CATS_CUDA(launch_gemm(g, st));
+    GemmProblem go = {};
+    go.epi = EPI_PARTIAL; go.T = T; go.K = D; go.n_out = H; go.n_mats = 1; go.W[0] = w->wo; go.X = ws.o;
+    go.fix_part = ws.fix_part; go.fix_flags = ws.fix_flags; go.part = ws.part; go.part_stride = ws.part_stride; go.d_status = d_status;
+    const int pieces_o = gemm_plan(go).max_pieces;
+    GemmProblem ggu = {};
+    ggu.epi = EPI_SWIGLU; ggu.T = T; ggu.K = H; ggu.n_out = F; ggu.n_mats = 2; ggu.W[0] = w->w_gate_up; ggu.X = ws.xn;
+    ggu.fix_part = ws.fix_part; ggu.fix_flags = ws.fix_flags; ggu.act_out = ws.act; ggu.d_status = d_status;
+    GemmProblem gd = {};
+    gd.epi = EPI_PARTIAL; gd.T = T; gd.K = F; gd.n_out = H; gd.n_mats = 1; gd.W[0] = w->w_down; gd.X = ws.act;
+    gd.fix_part = ws.fix_part; gd.fix_flags = ws.fix_flags; gd.part = ws.part; gd.part_stride = ws.part_stride; gd.d_status = d_status;
+    const int pieces_d = gemm_plan(gd).max_pieces;
+    GemmProblem nxt_after = {};
+    if (next_is_head) { nxt_after.epi = EPI_LMHEAD; nxt_after.T = T; nxt_after.K = H; nxt_after.n_out = c->vocab; nxt_after.n_mats = 1; nxt_after.W[0] = next_w; }
+    else { nxt_after.epi = EPI_QKV; nxt_after.T = T; nxt_after.K = H; nxt_after.n_out = D; nxt_after.n_mats = 3; nxt_after.W[0] = next_w; }
+    gd.warm_next = next_w ? &nxt_after : nullptr;
+
+    const bool tail_on = stage_on(3) && stage_on(4) && stage_on(5) && stage_on(6);
+    if (tail_on && g_debug_chain && gemm_chain_supported() && H % 4 == 0) {
+        // the second half of the layer as ONE launch: the weight ring lives on across the three projections
+        NormProblem nm = {resid, ws.part, pieces_o, ws.part_stride, w->mlp_norm, ws.xn, T, H, c->rms_eps};
+        CATS_CUDA(launch_layer_tail(go, nm, ggu, gd, ws.fix_flags + kFixSlots, st));
+        return pieces_d;
+    }
+    go.warm_next = &ggu;
+    if (stage_on(3)) CATS_CUDA(launch_gemm(go, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
                                  nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st, d_status));
-
-    g = GemmProblem{};
-    g.epi = EPI_SWIGLU; g.T = T; g.K = H; g.n_out = F; g.n_mats = 2; g.W[0] = w->w_gate_up; g.X = ws.xn;
-    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.act_out = ws.act; g.d_status = d_status;
-    nxt = GemmProblem{};
-    nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = F; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->w_down;
-    g.warm_next = &nxt;
-    if (stage_on(5)) CATS_CUDA(launch_gemm(g, st));
-
-    g = GemmProblem{};
-    g.epi = EPI_PARTIAL; g.T = T; g.K = F; g.n_out = H; g.n_mats = 1; g.W[0] = w->w_down; g.X = ws.act;
-    g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags; g.part = ws.part; g.part_stride = ws.part_stride; g.d_status = d_status;
-    int pieces_d = gemm_plan(g).max_pieces;
-    nxt = GemmProblem{};
-    if (next_is_head) { nxt.epi = EPI_LMHEAD; nxt.T = T; nxt.K = H; nxt.n_out = c->vocab; nxt.n_mats = 1; nxt.W[0] = next_w; }
-    else { nxt.epi = EPI_QKV; nxt.T = T; nxt.K = H; nxt.n_out = D; nxt.n_mats = 3; nxt.W[0] = next_w; }
-    g.warm_next = next_w ? &nxt : nullptr;
-    if (stage_on(6)) CATS_CUDA(launch_gemm(g, st));
+    ggu.warm_next = &gd;
+    if (stage_on(5)) CATS_CUDA(launch_gemm(ggu, st));
+    if (stage_on(6)) CATS_CUDA(launch_gemm(gd, st));
     return pieces_d;
 }
 
@@ -164,7 +175,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               const TypicalOut* ty = nullptr) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
+                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots + kChainSyncInts, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -215,6 +226,7 @@ int cats_last_launch_count(void) { return g_launch_count; }
 /* Measurement and fault-injection hooks, declared in include/cats_debug.h. */
 void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
 void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which ? 1 : 0); }
+void cats_debug_chained_launch(int on) { g_debug_chain = on ? 1 : 0; }
 void cats_debug_inject_fault(int which) { g_debug_fault = (which == 1 || which == 2) ? which : 0; }
 int cats_debug_wait_limit_ns(unsigned long long ns) {
     if (ns == 0) ns = kWaitLimitNs;
@@ -253,6 +265,7 @@ size_t cats_packed_weight_bytes(int32_t n_src, int32_t layout, int32_t rows, int
 int cats_pack_weights(const void* const* d_src, int32_t n_src, int32_t layout, int32_t rows, int32_t cols, void* d_dst,
                       void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_pack_weights");
     g_call_boundary = true;
     if (!d_src || !d_dst || cats_packed_weight_bytes(n_src, layout, rows, cols) == 0) return CATS_ERR_INVALID_ARG;
     for (int i = 0; i < n_src; ++i)
@@ -266,6 +279,7 @@ int cats_pack_weights(const void* const* d_src, int32_t n_src, int32_t layout, i
 int cats_build_tree_mask(const int32_t* d_parent, int32_t T, int32_t prefix_len, uint64_t* d_mask, int32_t* d_pos,
                          int32_t* d_depth, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_build_tree_mask");
     g_call_boundary = true;
     if (!d_parent || !d_mask || !d_pos || !d_status) return CATS_ERR_INVALID_ARG;
     int rc = check_tree_args(T, prefix_len);
@@ -277,6 +291,7 @@ int cats_build_tree_mask(const int32_t* d_parent, int32_t T, int32_t prefix_len,
 int cats_embed_tokens(const void* d_embed, const int32_t* d_tokens, int32_t T, int32_t hidden, int32_t vocab, float* d_resid,
                       int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_embed_tokens");
     g_call_boundary = true;
     if (!d_embed || !d_tokens || !d_resid || !d_status) return CATS_ERR_INVALID_ARG;
     if (T < 1 || T > CATS_MAX_TREE || hidden < 8 || hidden % 8 || vocab < 1) return CATS_ERR_INVALID_ARG;
@@ -289,6 +304,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
                       const uint64_t* d_mask, const int32_t* d_pos, int32_t T, int32_t prefix_len, void* d_ws, size_t ws_bytes,
                       int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_verify_layer");
     g_call_boundary = true;
     int rc = check_cfg(cfg);
     if (rc) return rc;
@@ -317,6 +333,7 @@ int cats_verify_layer_nodes(const cats_model_cfg* cfg, const cats_layer_weights*
                             void* d_vcache, const uint64_t* d_mask, const int32_t* d_pos, const int32_t* d_nodes, int32_t m,
                             int32_t T, int32_t prefix_len, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_verify_layer_nodes");
     g_call_boundary = true;
     int rc = check_cfg(cfg);
     if (rc) return rc;
@@ -345,6 +362,7 @@ int cats_tree_attention(const void* d_q, const void* d_k, const void* d_v, const
                         int32_t n_heads, int32_t head_dim, int64_t kv_row_stride_elems, float scale, void* d_out, void* d_ws,
                         size_t ws_bytes, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_tree_attention");
     g_call_boundary = true;
     if (!d_q || !d_k || !d_v || !d_mask || !d_out || !d_status) return CATS_ERR_INVALID_ARG;
     int rc = check_tree_args(T, prefix_len);
@@ -370,6 +388,7 @@ int cats_tree_attention(const void* d_q, const void* d_k, const void* d_v, const
 int cats_lm_head_argmax(const cats_model_cfg* cfg, const void* d_final_norm, const void* d_w_lm, const float* d_resid, int32_t T,
                         float* d_logits, int32_t* d_argmax, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_lm_head_argmax");
     g_call_boundary = true;
     int rc = check_cfg(cfg);
     if (rc) return rc;
@@ -388,6 +407,7 @@ int cats_lm_head_typical(const cats_model_cfg* cfg, const void* d_final_norm, co
                          int32_t* d_argmax, float* d_lse, float* d_entropy, float* d_cand_logit, void* d_ws, size_t ws_bytes,
                          int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_lm_head_typical");
     g_call_boundary = true;
     int rc = check_cfg(cfg);
     if (rc) return rc;
@@ -411,6 +431,7 @@ int cats_accept_path_typical(const int32_t* d_parent, const int32_t* d_tokens, c
                              float log_delta, int32_t* d_path, int32_t* d_path_len, int32_t* d_out_tokens, int32_t* d_n_out,
                              int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_accept_path_typical");
     g_call_boundary = true;
     if (!d_parent || !d_tokens || !d_argmax || !d_cand_logit || !d_lse || !d_entropy || !d_path || !d_path_len || !d_out_tokens ||
         !d_n_out || !d_status)
@@ -424,6 +445,7 @@ int cats_accept_path_typical(const int32_t* d_parent, const int32_t* d_tokens, c
 int cats_accept_path(const int32_t* d_parent, const int32_t* d_tokens, const int32_t* d_argmax, int32_t T, int32_t* d_path,
                      int32_t* d_path_len, int32_t* d_out_tokens, int32_t* d_n_out, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_accept_path");
     g_call_boundary = true;
     if (!d_parent || !d_tokens || !d_argmax || !d_path || !d_path_len || !d_out_tokens || !d_n_out || !d_status)
         return CATS_ERR_INVALID_ARG;
@@ -436,6 +458,7 @@ int cats_compact_kv(void* d_kcache, void* d_vcache, int32_t n_layers, int64_t la
                     int32_t prefix_len, const int32_t* d_path, const int32_t* d_path_len, int32_t* d_new_len, int32_t* d_src_rows,
                     int32_t* d_dst_rows, int32_t* d_status, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_compact_kv");
     g_call_boundary = true;
     if (!d_kcache || !d_vcache || !d_path || !d_path_len || !d_status) return CATS_ERR_INVALID_ARG;
     if (n_layers < 1 || row_elems < 8 || row_elems % 8 || layer_stride_elems % 8 || prefix_len < 0) return CATS_ERR_INVALID_ARG;
@@ -447,6 +470,7 @@ int cats_compact_kv(void* d_kcache, void* d_vcache, int32_t n_layers, int64_t la
 
 int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, const int32_t* d_tokens, void* stream) {
     g_launch_count = 0;
+    NvtxRange nvtx_range("cats_verify_forward");
     g_call_boundary = true;
     if (!a || !d_parent || !d_tokens) return CATS_ERR_INVALID_ARG;
     const cats_model_cfg* c = a->cfg;

@@ -129,64 +129,439 @@ __device__ __forceinline__ void st_release(int* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-// Register and shared-memory footprint are chosen so that one CTA of the RMSNorm kernel (256 threads, <= 80 registers,
-// no dynamic shared memory) fits on the SM beside a resident CTA of this kernel: 224 x 192 + 256 x 80 registers <= 64 K,
-// and 224.5 KB + 2 x 1 KB reserved + the norm's static 32 B <= 228 KB.  With programmatic dependent launch the CTAs of
-// the projection that FOLLOWS a norm then take the SMs as soon as the previous projection leaves them and fill their
-// weight ring while the norm is still running.
-#ifndef CATS_GEMM_MAXREG
-#define CATS_GEMM_MAXREG 192
-#endif
-template <int EPI>
-__global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    uint8_t* stages = smem_raw;                                                             // 1024-byte aligned (checked)
-    float* acc_s = reinterpret_cast<float*>(stages + (size_t)p.n_stages * p.stage_bytes);   // [32][128] fp32
-    uint8_t* landing = reinterpret_cast<uint8_t*>(acc_s) + (size_t)kStagingCols * 128 * 4;  // 16 KB, contents never read
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(landing + kWChunk);
-    volatile int* abort_flag = &ctrl->abort_flag;
-    if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled operand tiles need this alignment; never seen violated
-        if (threadIdx.x == 0) report(p.d_status, CATS_ERR_UNSUPPORTED);
-        return;
-    }
+// ---------------------------------------------------------------------------------------------------
+// The kernel is written as four roles (W producer, X producer, MMA issuer, epilogue warps), each a function over ONE
+// projection ("phase") that carries its pipeline counters in and out.  k_gemm_sk runs one phase; k_gemm_chain runs
+// several projections of a decoder layer back to back in one launch, so that the weight ring never drains between
+// them: the W producer runs ahead into the next projection's weights while the epilogues of this one finish and the
+// grid-wide dependency (all CTAs done, the RMSNorm in between) resolves.
+// ---------------------------------------------------------------------------------------------------
+struct CtaRange {
+    long long u0, u1;     // this CTA's units in the phase's unit space (see below)
+    int vlen, koff;       // every tile owns vlen consecutive units, unit v of a tile being its K unit koff + v
+    bool helper;
+};
 
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const int cta = blockIdx.x;
-    const int S = p.n_stages;
-    // The CTA's work is a range [u0, u1) of a unit space in which every tile owns vlen consecutive units, unit v of a
-    // tile being its K unit koff + v.
-    //   split_s == 0, head_units == 0: all (tile, K) units, even contiguous shares ("stream-K"); vlen = n_ku.
-    //   split_s > 0: every tile cut into split_s aligned pieces.
-    //   head_units > 0: CTA t < n_tiles owns tile t and runs its first head_units K units; the CTAs after them
-    //     ("helpers") share the remaining units of all tiles evenly and only contribute partial tiles.
-    long long u0, u1;
-    int vlen = p.n_ku, koff = 0;
-    bool helper = false;
+// The CTA's work is a range [u0, u1) of a unit space in which every tile owns vlen consecutive units.
+//   split_s == 0, head_units == 0: all (tile, K) units, even contiguous shares ("stream-K"); vlen = n_ku.
+//   split_s > 0: every tile cut into split_s aligned pieces.
+//   head_units > 0: CTA t < n_tiles owns tile t and runs its first head_units K units; the CTAs after them
+//     ("helpers") share the remaining units of all tiles evenly and only contribute partial tiles.
+__device__ __forceinline__ CtaRange cta_range(const GemmDev& p, int cta) {
+    CtaRange r;
+    r.vlen = p.n_ku;
+    r.koff = 0;
+    r.helper = false;
     if (p.head_units > 0) {
         if (cta < p.n_tiles) {
-            vlen = p.head_units;
-            u0 = (long long)cta * vlen;
-            u1 = u0 + vlen;
+            r.vlen = p.head_units;
+            r.u0 = (long long)cta * r.vlen;
+            r.u1 = r.u0 + r.vlen;
         } else {
-            helper = true;
-            vlen = p.n_ku - p.head_units;
-            koff = p.head_units;
-            u0 = min((long long)p.total_rem, (long long)(cta - p.n_tiles) * p.help_upc);
-            u1 = min((long long)p.total_rem, u0 + p.help_upc);
+            r.helper = true;
+            r.vlen = p.n_ku - p.head_units;
+            r.koff = p.head_units;
+            r.u0 = min((long long)p.total_rem, (long long)(cta - p.n_tiles) * p.help_upc);
+            r.u1 = min((long long)p.total_rem, r.u0 + p.help_upc);
         }
     } else if (p.split_s > 0) {
         const long long t0 = (long long)(cta / p.split_s) * p.n_ku;
-        u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
-        u1 = min(t0 + p.n_ku, u0 + (long long)p.units_per_cta);
+        r.u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
+        r.u1 = min(t0 + p.n_ku, r.u0 + (long long)p.units_per_cta);
+        if (cta >= p.n_tiles * p.split_s) r.u0 = r.u1 = 0;       // a CTA beyond this phase's grid (chained launches)
     } else {
-        u0 = (long long)cta * p.units_per_cta;
-        u1 = min(p.total_units, u0 + (long long)p.units_per_cta);
+        r.u0 = min(p.total_units, (long long)cta * p.units_per_cta);
+        r.u1 = min(p.total_units, r.u0 + (long long)p.units_per_cta);
     }
-    const int n_units = (int)max(0ll, u1 - u0);
+    if (r.u1 < r.u0) r.u1 = r.u0;
+    return r;
+}
 
+struct Pipe {               // the CTA's pipeline resources, the same for every phase of a launch
+    uint8_t* stages;        // ring of S stages
+    float* acc_s;           // [32][128] fp32 epilogue staging tile
+    uint8_t* landing;       // 16 KB, contents never read
+    GemmCtrl* ctrl;
+    volatile int* abort_flag;
+    uint32_t tmem_acc;
+    int S;
+};
+
+// One copy producer (a single thread): is_w streams W, else X.  A stage holds kUnitKb K blocks fetched by ONE copy of W
+// (contiguous in the packed matrix) and ONE copy of X: a bulk copy costs its issuing thread a fixed ~0.45 us whatever
+// its size (measured), so the two kinds of copies come from different threads.  i: units issued so far by this CTA
+// over all phases (ring position).  Returns false after an abort.
+__device__ __forceinline__ bool produce_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, bool is_w, uint64_t pol, int& i) {
+    const int S = pp.S;
+    const int n_units = (int)(r.u1 - r.u0);
+    for (int k = 0; k < n_units; ++k, ++i) {
+        if (i >= S && !mbar_wait(&pp.ctrl->empty[i % S], ((i / S) - 1) & 1, pp.abort_flag)) return false;
+        const int s = i % S;
+        const long long u = r.u0 + k;
+        const int tile = (int)(u / r.vlen);
+        const int kb = (r.koff + (int)(u - (long long)tile * r.vlen)) * kUnitKb;
+        const int nk = min(kUnitKb, p.n_kb - kb);
+        uint8_t* stage = pp.stages + (size_t)s * p.stage_bytes;
+        if (is_w) {
+            const uint32_t bytes = (uint32_t)nk * kWChunk;
+            mbar_expect_tx(&pp.ctrl->full[s], bytes);
+            bulk_load(stage, p.Wp + ((size_t)tile * p.n_kb + kb) * kWChunk, bytes, &pp.ctrl->full[s], pol);
+        } else {
+            const uint32_t bytes = (uint32_t)nk * p.x_chunk_bytes;
+            mbar_expect_tx(&pp.ctrl->full[s], bytes);
+            bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &pp.ctrl->full[s], pol);
+        }
+    }
+    return true;
+}
+
+// Real copies of the first chunks the same CTA of the NEXT launch's projection will read, into a landing buffer nobody
+// reads: they leave those lines in L2 while this kernel drains and runs its last epilogue.
+__device__ __forceinline__ void warm_next_projection(const GemmDev& p, const Pipe& pp, int cta) {
+    if (p.warm_ptr == nullptr || p.warm_chunks <= 0) return;
+    // first chunk of this CTA's range in the next matrix: unit cta * upc -> (tile, K block)
+    const long long wu = (long long)cta * p.warm_upc;
+    const long long wt = wu / p.warm_n_ku;
+    long long first = wt * p.warm_n_kb + (wu - wt * p.warm_n_ku) * kUnitKb;
+    long long n = min((long long)p.warm_chunks, p.warm_total_chunks - first);
+    if (n < 0) n = 0;
+    mbar_expect_tx(&pp.ctrl->warm, (uint32_t)n * kWChunk);
+    for (long long j = 0; j < n; ++j)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(pp.landing)), "l"(p.warm_ptr + (size_t)(first + j) * kWChunk), "r"(kWChunk), "r"(smem_u32(&pp.ctrl->warm))
+                     : "memory");
+    volatile int ignore = 0;
+    mbar_wait(&pp.ctrl->warm, 0, &ignore);   // the landing buffer must stay alive until the copies have landed
+}
+
+// After an abort: let the copies in flight land (bounded) before the CTA goes away.  i: units issued by this producer.
+__device__ __forceinline__ void drain_after_abort(const Pipe& pp, int i) {
+    volatile int ignore = 0;
+    for (int j = max(0, i - pp.S); j < i; ++j) mbar_wait(&pp.ctrl->full[j % pp.S], (j / pp.S) & 1, &ignore);
+}
+
+// The MMA issuer (a single thread).  i: ring position, seg: accumulator segments so far (both over all phases).
+__device__ __forceinline__ bool mma_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, int& i, int& seg) {
+    const int S = pp.S;
+    const uint32_t idesc = umma_idesc_bf16_m128(p.n_pad);
+    bool ok = true;
+    for (long long u = r.u0; u < r.u1 && ok; ++seg) {
+        const long long tile_end = (u / r.vlen + 1) * r.vlen;
+        const long long seg_end = min(r.u1, tile_end);
+        const int b = seg & 1;
+        if (seg >= 2) ok = mbar_wait(&pp.ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, pp.abort_flag);
+        tc_fence_after_sync();
+        const uint32_t d_addr = pp.tmem_acc + (uint32_t)(b * p.n_pad);
+        bool first = true;
+        for (; u < seg_end && ok; ++u, ++i) {
+            const int s = i % S;
+            ok = mbar_wait(&pp.ctrl->full[s], (i / S) & 1, pp.abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int kb = (r.koff + (int)(u % r.vlen)) * kUnitKb;
+            const int nk = min(kUnitKb, p.n_kb - kb);
+            const uint32_t a_addr = smem_u32(pp.stages + (size_t)s * p.stage_bytes);
+            const uint32_t b_addr = a_addr + kUnitKb * kWChunk;
+            for (int j = 0; j < nk; ++j) {
+                const uint64_t da = umma_desc_sw128(a_addr + j * kWChunk);
+                const uint64_t db = umma_desc_sw128(b_addr + j * p.x_chunk_bytes);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_bf16(d_addr, da + 2 * k, db + 2 * k, idesc, !(first && k == 0));
+                first = false;
+            }
+            umma_commit(&pp.ctrl->empty[s]);
+        }
+        umma_commit(&pp.ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
+    }
+    return ok;
+}
+
+// The four epilogue warps (128 threads) over one phase.  seg: accumulator segments so far over all phases.
+template <int EPI>
+__device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, int cta, int warp, int lane,
+                                               int& seg, bool& ok) {
+    const int q4 = warp & 3;               // TMEM lane quadrant this warp may read
+    const int f = q4 * 32 + lane;          // accumulator row = weight row inside the tile
+    const int et = (warp - 2) * 32 + lane; // 0..127 among the epilogue threads
+    for (long long u = r.u0; u < r.u1; ++seg) {
+        const int tile = (int)(u / r.vlen);
+        const long long tile_begin = (long long)tile * r.vlen;
+        const long long tile_end = tile_begin + r.vlen;
+        const long long seg_end = min(r.u1, tile_end);
+        const bool tail = (seg_end == tile_end);
+        const bool head = !r.helper && (u == tile_begin);
+        u = seg_end;
+        const int b = seg & 1;
+        int head_cta = 0, last_cta = 0;         // stream-K: the CTAs that share this tile
+        int g_first = 0, g_n = 0, my_slot = cta;   // contributors' slots this (owning) piece adds; slot a contributor writes
+        if (p.head_units > 0) {
+            // the tile's remaining units [tile * R, (tile + 1) * R) are spread over at most two helpers
+            const int R = p.n_ku - p.head_units;
+            const int j0 = (int)(((long long)tile * R) / p.help_upc), j1 = (int)(((long long)(tile + 1) * R - 1) / p.help_upc);
+            g_first = 2 * tile;
+            g_n = j1 - j0 + 1;
+            if (r.helper) my_slot = 2 * tile + ((cta - p.n_tiles) - j0);
+        } else {
+            head_cta = (int)(tile_begin / p.units_per_cta);
+            last_cta = (int)((tile_end - 1) / p.units_per_cta);
+            g_first = cta + 1;
+            g_n = (head && !tail) ? last_cta - cta : 0;
+        }
+        // A tile this CTA owns but shares with other CTAs: their partial tiles are usually published long before
+        // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
+        const bool gather = head && g_n > 0 && EPI != EPI_PARTIAL;
+        float pre[64];
+        if (ok && gather) {
+            if (et == 0) {
+                unsigned long long t0 = globaltimer_ns();
+                for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
+                    while (ld_acquire(p.fix_flags + c2) == 0) {
+                        if (*pp.abort_flag || globaltimer_ns() - t0 > g_wait_limit_ns) { *pp.abort_flag = 1; break; }
+                    }
+                }
+            }
+            epi_barrier();
+            ok = !*pp.abort_flag;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) pre[cc * 16 + i] = 0.f;
+                if (ok && cc * 16 < p.n_pad) {
+                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
+                        const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(cc * 16) * 128 + f;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pre[cc * 16 + i] += __ldcg(src + (size_t)i * 128);
+                    }
+                }
+            }
+        }
+        if (ok) ok = mbar_wait(&pp.ctrl->acc_full[b], (seg >> 1) & 1, pp.abort_flag);
+        ok = ok && !*pp.abort_flag;
+        tc_fence_after_sync();
+        const uint32_t taddr = pp.tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * p.n_pad);
+        int mat = 0, row0;
+        if (EPI == EPI_SWIGLU) row0 = tile * 64;
+        else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
+
+        if (!ok) {
+            // nothing: fall through to the arrive below so that nobody waits on this accumulator
+        } else if (EPI == EPI_PARTIAL) {
+            const int feat = row0 + f;
+            const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
+            store_tile_transposed(taddr, p.n_pad, p.T, pp.acc_s, f, et, p.part + (size_t)piece * p.part_stride + row0,
+                                  (size_t)p.n_out, p.n_out - row0);
+            if (head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
+                for (int sl = last_cta - head_cta + 1; sl < p.max_pieces; ++sl) {
+                    float* z = p.part + (size_t)sl * p.part_stride + feat;
+                    for (int n = 0; n < p.T; ++n) z[(size_t)n * p.n_out] = 0.f;
+                }
+            }
+        } else if (!head) {
+            // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
+            store_tile_transposed(taddr, p.n_pad, p.n_pad, pp.acc_s, f, et, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
+            __threadfence();
+            epi_barrier();
+            if (et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
+        } else {
+            // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
+#pragma unroll
+            for (int qc = 0; qc < CATS_MAX_TREE / kStagingCols; ++qc) {
+                const int c0 = qc * kStagingCols;
+                if (c0 >= p.T || !ok) break;
+#pragma unroll
+                for (int hc = 0; hc < kStagingCols / 16; ++hc) {
+                    const int c = hc * 16;
+                    if (c0 + c >= p.n_pad) break;
+                    float v[16];
+                    tmem_ld16(taddr + c0 + c, v);
+                    if (gather) {
+                        if (qc * (kStagingCols / 16) + hc < 4) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) v[i] += pre[((qc * (kStagingCols / 16) + hc) & 3) * 16 + i];
+                        } else {
+                            for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
+                                const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) v[i] += __ldcg(src + (size_t)i * 128);
+                            }
+                        }
+                    }
+                    if (EPI == EPI_LMHEAD && p.logits != nullptr && row0 + f < p.n_out) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            int n = c0 + c + i;
+                            if (n < p.T) p.logits[(size_t)n * p.n_out + row0 + f] = v[i];
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pp.acc_s[(c + i) * 128 + f] = v[i];
+                }
+                epi_barrier();
+                const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
+                if (EPI == EPI_QKV) {
+                    // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
+                    // the thread are issued before the first store, so their latencies overlap.
+                    const int j8 = (et & 15) * 8;
+                    const int feat = row0 + j8;
+                    const int hd = p.head_dim, half = hd >> 1;
+                    const int in_head = feat % hd;
+                    const bool first_half = in_head < half;
+                    const int partner = first_half ? j8 + half : j8 - half;
+                    const int ri = in_head % half;
+                    const float sgn = first_half ? -1.f : 1.f;
+                    constexpr int NI = kStagingCols / 8;
+                    if (feat < p.n_out) {
+                        uint4 packed[NI];
+                        if (mat < 2) {
+                            float4 cs[NI][4];     // (cos, sin) of the 8 feature pairs
+#pragma unroll
+                            for (int it = 0; it < NI; ++it) {
+                                const int nl = (et >> 4) + 8 * it;
+                                const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * half + ri);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) cs[it][q] = nl < n_hi ? __ldg(src + q) : make_float4(1.f, 0.f, 1.f, 0.f);
+                            }
+#pragma unroll
+                            for (int it = 0; it < NI; ++it) {
+                                const int nl = (et >> 4) + 8 * it;
+                                const float4 x0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
+                                const float4 x1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
+                                const float4 y0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + partner);
+                                const float4 y1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + partner + 4);
+                                packed[it].x = pack_bf16x2(x0.x * cs[it][0].x + sgn * y0.x * cs[it][0].y, x0.y * cs[it][0].z + sgn * y0.y * cs[it][0].w);
+                                packed[it].y = pack_bf16x2(x0.z * cs[it][1].x + sgn * y0.z * cs[it][1].y, x0.w * cs[it][1].z + sgn * y0.w * cs[it][1].w);
+                                packed[it].z = pack_bf16x2(x1.x * cs[it][2].x + sgn * y1.x * cs[it][2].y, x1.y * cs[it][2].z + sgn * y1.y * cs[it][2].w);
+                                packed[it].w = pack_bf16x2(x1.z * cs[it][3].x + sgn * y1.z * cs[it][3].y, x1.w * cs[it][3].z + sgn * y1.w * cs[it][3].w);
+                            }
+                        } else {
+#pragma unroll
+                            for (int it = 0; it < NI; ++it) {
+                                const int nl = (et >> 4) + 8 * it;
+                                const float4 x0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
+                                const float4 x1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
+                                packed[it] = make_uint4(pack_bf16x2(x0.x, x0.y), pack_bf16x2(x0.z, x0.w), pack_bf16x2(x1.x, x1.y),
+                                                        pack_bf16x2(x1.z, x1.w));
+                            }
+                        }
+                        if (mat == 0 || p.kv_rows == nullptr) {
+                            uint16_t* base = mat == 0 ? p.q_out + (size_t)c0 * p.n_out
+                                                      : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
+#pragma unroll
+                            for (int it = 0; it < NI; ++it) {
+                                const int nl = (et >> 4) + 8 * it;
+                                if (nl < n_hi) *reinterpret_cast<uint4*>(base + (size_t)nl * p.n_out + feat) = packed[it];
+                            }
+                        } else {
+                            // a subset of the tree: row t of the batch is tree node kv_rows[t]
+                            uint16_t* base = (mat == 1 ? p.kcache : p.vcache) + (size_t)p.prefix_len * p.n_out;
+#pragma unroll
+                            for (int it = 0; it < NI; ++it) {
+                                const int nl = (et >> 4) + 8 * it;
+                                if (nl < n_hi)
+                                    *reinterpret_cast<uint4*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
+                            }
+                        }
+                    }
+                } else if (EPI == EPI_SWIGLU) {
+                    // features beyond n_out come out as silu(0)*0 = 0 (zero-padded weights): they are stored too,
+                    // so that the padded K block of the down projection's input reads as zeros.
+                    // thread -> 8 consecutive features = one 16-byte group of the packed layout, every 16th node
+                    const int j8 = (et & 7) * 8;
+                    const int feat = row0 + j8;
+                    constexpr int NI = kStagingCols / 16;
+#pragma unroll
+                    for (int it = 0; it < NI; ++it) {
+                        const int nl = (et >> 3) + 16 * it;
+                        const float4 g0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
+                        const float4 g1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
+                        const float4 u0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + 64 + j8);
+                        const float4 u1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + 64 + j8 + 4);
+                        uint4 o;
+                        o.x = pack_bf16x2(__fdividef(g0.x, 1.f + __expf(-g0.x)) * u0.x, __fdividef(g0.y, 1.f + __expf(-g0.y)) * u0.y);
+                        o.y = pack_bf16x2(__fdividef(g0.z, 1.f + __expf(-g0.z)) * u0.z, __fdividef(g0.w, 1.f + __expf(-g0.w)) * u0.w);
+                        o.z = pack_bf16x2(__fdividef(g1.x, 1.f + __expf(-g1.x)) * u1.x, __fdividef(g1.y, 1.f + __expf(-g1.y)) * u1.y);
+                        o.w = pack_bf16x2(__fdividef(g1.z, 1.f + __expf(-g1.z)) * u1.z, __fdividef(g1.w, 1.f + __expf(-g1.w)) * u1.w);
+                        if (nl < n_hi) *reinterpret_cast<uint4*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad)) = o;
+                    }
+                } else if (EPI == EPI_LMHEAD) {
+                    for (int nl = warp - 2; nl < n_hi; nl += 4) {
+                        float best = -INFINITY;
+                        int bi = 0x7fffffff;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            int ff = lane + 32 * i;
+                            float v = pp.acc_s[nl * 128 + ff];
+                            if (row0 + ff < p.n_out && v > best) { best = v; bi = row0 + ff; }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                            int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+                        }
+                        if (lane == 0) {
+                            p.pmax[(size_t)tile * 128 + c0 + nl] = best;
+                            p.pidx[(size_t)tile * 128 + c0 + nl] = bi;
+                        }
+                        if (p.psum != nullptr) {
+                            // softmax statistics of this vocabulary tile at the given temperature, relative to the
+                            // tile's own maximum: Z = sum e, S1 = sum e * (logit - max), e = exp((logit - max) / t)
+                            float z = 0.f, s1 = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                int ff = lane + 32 * i;
+                                if (row0 + ff < p.n_out) {
+                                    float d = pp.acc_s[nl * 128 + ff] - best;
+                                    float e = exp2f(d * p.inv_temp_log2e);
+                                    z += e;
+                                    s1 = fmaf(e, d, s1);
+                                }
+                            }
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) {
+                                z += __shfl_xor_sync(0xffffffffu, z, o);
+                                s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+                            }
+                            if (lane == 0) {
+                                p.psum[(size_t)tile * 128 + c0 + nl] = z;
+                                p.ps1[(size_t)tile * 128 + c0 + nl] = s1;
+                            }
+                        }
+                    }
+                    if (p.cand != nullptr && et > 0 && et < p.T) {
+                        // logit of tree node et's own token under its parent's distribution, if this tile holds it
+                        const int pa = __ldg(p.tree_parent + et), tk = __ldg(p.tree_tokens + et);
+                        if (pa >= c0 && pa < c0 + n_hi && tk >= row0 && tk < row0 + 128 && tk < p.n_out)
+                            p.cand[et] = pp.acc_s[(pa - c0) * 128 + (tk - row0)];
+                    }
+                }
+                epi_barrier();
+            }
+            if (gather && et == 0)
+                for (int c2 = g_first; c2 < g_first + g_n; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&pp.ctrl->acc_empty[b]);
+    }
+}
+
+// Carves the dynamic shared memory, initialises the barriers and allocates tensor memory.  Every thread calls it.
+// Returns false (after reporting) if the shared-memory window is not 1024-byte aligned; never seen violated.
+__device__ __forceinline__ bool pipe_setup(Pipe& pp, uint8_t* smem_raw, int n_stages, uint32_t stage_bytes, uint32_t tmem_cols,
+                                           int32_t* d_status) {
+    pp.stages = smem_raw;                                                                   // 1024-byte aligned (checked)
+    pp.acc_s = reinterpret_cast<float*>(pp.stages + (size_t)n_stages * stage_bytes);        // [32][128] fp32
+    pp.landing = reinterpret_cast<uint8_t*>(pp.acc_s) + (size_t)kStagingCols * 128 * 4;     // 16 KB, contents never read
+    pp.ctrl = reinterpret_cast<GemmCtrl*>(pp.landing + kWChunk);
+    pp.abort_flag = &pp.ctrl->abort_flag;
+    pp.S = n_stages;
+    if ((smem_u32(smem_raw) & 1023u) != 0) {   // the swizzled operand tiles need this alignment
+        if (threadIdx.x == 0) report(d_status, CATS_ERR_UNSUPPORTED);
+        return false;
+    }
+    GemmCtrl* ctrl = pp.ctrl;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(&ctrl->full[s], 2);      // one arrive.expect_tx from each copy producer
             mbar_init(&ctrl->empty[s], 1);
         }
@@ -198,384 +573,296 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
         ctrl->abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == 1) {
-        tmem_alloc(&ctrl->tmem_base, p.tmem_cols);
+    if ((threadIdx.x >> 5) == 1) {
+        tmem_alloc(&ctrl->tmem_base, tmem_cols);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pp.tmem_acc = ctrl->tmem_base;
+    return true;
+}
+
+__device__ __forceinline__ void pipe_teardown(const Pipe& pp, uint32_t tmem_cols, int32_t* d_status) {
+    tc_fence_before_sync();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(pp.tmem_acc, tmem_cols);
+    }
+    if (threadIdx.x == 0 && pp.ctrl->abort_flag) report(d_status, CATS_ERR_TIMEOUT);
+}
+
+// Register and shared-memory footprint are chosen so that one CTA of the RMSNorm kernel (256 threads, <= 80 registers,
+// no dynamic shared memory) fits on the SM beside a resident CTA of this kernel: 224 x 192 + 256 x 80 registers <= 64 K,
+// and 224.5 KB + 2 x 1 KB reserved + the norm's static 32 B <= 228 KB.  With programmatic dependent launch the CTAs of
+// the projection that FOLLOWS a norm then take the SMs as soon as the previous projection leaves them and fill their
+// weight ring while the norm is still running.
+#ifndef CATS_GEMM_MAXREG
+#define CATS_GEMM_MAXREG 192
+#endif
+template <int EPI>
+__global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Pipe pp;
+    if (!pipe_setup(pp, smem_raw, p.n_stages, p.stage_bytes, p.tmem_cols, p.d_status)) return;
     pdl_launch_dependents();
-    const uint32_t tmem_acc = ctrl->tmem_base;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+    const CtaRange r = cta_range(p, cta);
 
     if (warp == 0 || warp == 6) {
         // ---------------- copy producers: warp 0 streams W, warp 6 streams X ----------------
-        // One bulk copy costs its issuing thread a fixed ~0.45 us whatever its size (measured), so a stage holds
-        // kUnitKb K blocks fetched by ONE copy of W (contiguous in the packed matrix) and ONE copy of X, and the two
-        // kinds of copies come from different threads.
         if (lane == 0) {
             const bool is_w = (warp == 0);
             const uint64_t pol = is_w ? l2_policy_evict_first() : l2_policy_evict_last();
-            auto issue = [&](int i) {
-                const int s = i % S;
-                const long long u = u0 + i;
-                const int tile = (int)(u / vlen);
-                const int kb = (koff + (int)(u - (long long)tile * vlen)) * kUnitKb;
-                const int nk = min(kUnitKb, p.n_kb - kb);
-                uint8_t* stage = stages + (size_t)s * p.stage_bytes;
-                if (is_w) {
-                    const uint32_t bytes = (uint32_t)nk * kWChunk;
-                    mbar_expect_tx(&ctrl->full[s], bytes);
-                    bulk_load(stage, p.Wp + ((size_t)tile * p.n_kb + kb) * kWChunk, bytes, &ctrl->full[s], pol);
-                } else {
-                    const uint32_t bytes = (uint32_t)nk * p.x_chunk_bytes;
-                    mbar_expect_tx(&ctrl->full[s], bytes);
-                    bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &ctrl->full[s], pol);
-                }
-            };
             if (!is_w) pdl_wait();    // activations come from the previous kernel; weights never do
-            int issued = 0;
-            for (int i = 0; i < n_units; ++i) {
-                if (i >= S && !mbar_wait(&ctrl->empty[i % S], ((i / S) - 1) & 1, abort_flag)) break;
-                issue(i);
-                issued = i + 1;
-            }
-            if (is_w) {
-                // Real copies of the first chunks the same CTA of the next projection will read, into a landing buffer
-                // nobody reads: they leave those lines in L2 while this kernel drains and runs its last epilogue.
-                if (p.warm_ptr != nullptr && p.warm_chunks > 0) {
-                    // first chunk of this CTA's range in the next matrix: unit cta * upc -> (tile, K block)
-                    const long long wu = (long long)cta * p.warm_upc;
-                    const long long wt = wu / p.warm_n_ku;
-                    long long first = wt * p.warm_n_kb + (wu - wt * p.warm_n_ku) * kUnitKb;
-                    long long n = min((long long)p.warm_chunks, p.warm_total_chunks - first);
-                    if (n < 0) n = 0;
-                    mbar_expect_tx(&ctrl->warm, (uint32_t)n * kWChunk);
-                    for (long long j = 0; j < n; ++j)
-                        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                     ::"r"(smem_u32(landing)), "l"(p.warm_ptr + (size_t)(first + j) * kWChunk), "r"(kWChunk), "r"(smem_u32(&ctrl->warm))
-                                     : "memory");
-                    volatile int ignore = 0;
-                    mbar_wait(&ctrl->warm, 0, &ignore);   // the landing buffer must stay alive until the copies have landed
-                }
-            }
-            if (*abort_flag) {   // let the copies in flight land (bounded) before the CTA goes away
-                volatile int ignore = 0;
-                for (int i = max(0, issued - S); i < issued; ++i) mbar_wait(&ctrl->full[i % S], (i / S) & 1, &ignore);
-            }
+            int i = 0;
+            produce_units(p, r, pp, is_w, pol, i);
+            if (is_w) warm_next_projection(p, pp, cta);
+            if (*pp.abort_flag) drain_after_abort(pp, i);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16_m128(p.n_pad);
             int i = 0, seg = 0;
-            bool ok = true;
-            for (long long u = u0; u < u1 && ok; ++seg) {
-                const long long tile_end = (u / vlen + 1) * vlen;
-                const long long seg_end = min(u1, tile_end);
-                const int b = seg & 1;
-                if (seg >= 2) ok = mbar_wait(&ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, abort_flag);
-                tc_fence_after_sync();
-                const uint32_t d_addr = tmem_acc + (uint32_t)(b * p.n_pad);
-                bool first = true;
-                for (; u < seg_end && ok; ++u, ++i) {
-                    int s = i % S;
-                    ok = mbar_wait(&ctrl->full[s], (i / S) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const int kb = (koff + (int)(u % vlen)) * kUnitKb;
-                    const int nk = min(kUnitKb, p.n_kb - kb);
-                    const uint32_t a_addr = smem_u32(stages + (size_t)s * p.stage_bytes);
-                    const uint32_t b_addr = a_addr + kUnitKb * kWChunk;
-                    for (int j = 0; j < nk; ++j) {
-                        const uint64_t da = umma_desc_sw128(a_addr + j * kWChunk);
-                        const uint64_t db = umma_desc_sw128(b_addr + j * p.x_chunk_bytes);
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) umma_bf16(d_addr, da + 2 * k, db + 2 * k, idesc, !(first && k == 0));
-                        first = false;
-                    }
-                    umma_commit(&ctrl->empty[s]);
-                }
-                umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
-            }
+            mma_units(p, r, pp, i, seg);
         }
     } else if (warp < 6) {
         // ---------------- epilogue warps ----------------
-        const int q4 = warp & 3;               // TMEM lane quadrant this warp may read
-        const int f = q4 * 32 + lane;          // accumulator row = weight row inside the tile
-        const int et = (warp - 2) * 32 + lane; // 0..127 among the epilogue threads
         pdl_wait();
         int seg = 0;
         bool ok = true;
-        for (long long u = u0; u < u1; ++seg) {
-            const int tile = (int)(u / vlen);
-            const long long tile_begin = (long long)tile * vlen;
-            const long long tile_end = tile_begin + vlen;
-            const long long seg_end = min(u1, tile_end);
-            const bool tail = (seg_end == tile_end);
-            const bool head = !helper && (u == tile_begin);
-            u = seg_end;
-            const int b = seg & 1;
-            int head_cta = 0, last_cta = 0;         // stream-K: the CTAs that share this tile
-            int g_first = 0, g_n = 0, my_slot = cta;   // contributors' slots this (owning) piece adds; slot a contributor writes
-            if (p.head_units > 0) {
-                // the tile's remaining units [tile * R, (tile + 1) * R) are spread over at most two helpers
-                const int R = p.n_ku - p.head_units;
-                const int j0 = (int)(((long long)tile * R) / p.help_upc), j1 = (int)(((long long)(tile + 1) * R - 1) / p.help_upc);
-                g_first = 2 * tile;
-                g_n = j1 - j0 + 1;
-                if (helper) my_slot = 2 * tile + ((cta - p.n_tiles) - j0);
-            } else {
-                head_cta = (int)(tile_begin / p.units_per_cta);
-                last_cta = (int)((tile_end - 1) / p.units_per_cta);
-                g_first = cta + 1;
-                g_n = (head && !tail) ? last_cta - cta : 0;
-            }
-            // A tile this CTA owns but shares with other CTAs: their partial tiles are usually published long before
-            // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
-            const bool gather = head && g_n > 0 && EPI != EPI_PARTIAL;
-            float pre[64];
-            if (ok && gather) {
-                if (et == 0) {
-                    unsigned long long t0 = globaltimer_ns();
-                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
-                        while (ld_acquire(p.fix_flags + c2) == 0) {
-                            if (*abort_flag || globaltimer_ns() - t0 > g_wait_limit_ns) { *abort_flag = 1; break; }
-                        }
-                    }
-                }
-                epi_barrier();
-                ok = !*abort_flag;
-#pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) pre[cc * 16 + i] = 0.f;
-                    if (ok && cc * 16 < p.n_pad) {
-                        for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
-                            const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(cc * 16) * 128 + f;
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) pre[cc * 16 + i] += __ldcg(src + (size_t)i * 128);
-                        }
-                    }
-                }
-            }
-            if (ok) ok = mbar_wait(&ctrl->acc_full[b], (seg >> 1) & 1, abort_flag);
-            ok = ok && !*abort_flag;
-            tc_fence_after_sync();
-            const uint32_t taddr = tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * p.n_pad);
-            int mat = 0, row0;
-            if (EPI == EPI_SWIGLU) row0 = tile * 64;
-            else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
+        epilogue_units<EPI>(p, r, pp, cta, warp, lane, seg, ok);
+    }
+    pipe_teardown(pp, p.tmem_cols, p.d_status);
+}
 
-            if (!ok) {
-                // nothing: fall through to the arrive below so that nobody waits on this accumulator
-            } else if (EPI == EPI_PARTIAL) {
-                const int feat = row0 + f;
-                const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
-                store_tile_transposed(taddr, p.n_pad, p.T, acc_s, f, et, p.part + (size_t)piece * p.part_stride + row0,
-                                      (size_t)p.n_out, p.n_out - row0);
-                if (head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
-                    for (int sl = last_cta - head_cta + 1; sl < p.max_pieces; ++sl) {
-                        float* z = p.part + (size_t)sl * p.part_stride + feat;
-                        for (int n = 0; n < p.T; ++n) z[(size_t)n * p.n_out] = 0.f;
-                    }
-                }
-            } else if (!head) {
-                // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
-                store_tile_transposed(taddr, p.n_pad, p.n_pad, acc_s, f, et, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
-                __threadfence();
-                epi_barrier();
-                if (et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
-            } else {
-                // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
-#pragma unroll
-                for (int qc = 0; qc < CATS_MAX_TREE / kStagingCols; ++qc) {
-                    const int c0 = qc * kStagingCols;
-                    if (c0 >= p.T || !ok) break;
-#pragma unroll
-                    for (int hc = 0; hc < kStagingCols / 16; ++hc) {
-                        const int c = hc * 16;
-                        if (c0 + c >= p.n_pad) break;
-                        float v[16];
-                        tmem_ld16(taddr + c0 + c, v);
-                        if (gather) {
-                            if (qc * (kStagingCols / 16) + hc < 4) {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) v[i] += pre[((qc * (kStagingCols / 16) + hc) & 3) * 16 + i];
-                            } else {
-                                for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
-                                    const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
-#pragma unroll
-                                    for (int i = 0; i < 16; ++i) v[i] += __ldcg(src + (size_t)i * 128);
-                                }
-                            }
-                        }
-                        if (EPI == EPI_LMHEAD && p.logits != nullptr && row0 + f < p.n_out) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                int n = c0 + c + i;
-                                if (n < p.T) p.logits[(size_t)n * p.n_out + row0 + f] = v[i];
-                            }
-                        }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) acc_s[(c + i) * 128 + f] = v[i];
-                    }
-                    epi_barrier();
-                    const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
-                    if (EPI == EPI_QKV) {
-                        // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
-                        // the thread are issued before the first store, so their latencies overlap.
-                        const int j8 = (et & 15) * 8;
-                        const int feat = row0 + j8;
-                        const int hd = p.head_dim, half = hd >> 1;
-                        const int in_head = feat % hd;
-                        const bool first_half = in_head < half;
-                        const int partner = first_half ? j8 + half : j8 - half;
-                        const int ri = in_head % half;
-                        const float sgn = first_half ? -1.f : 1.f;
-                        constexpr int NI = kStagingCols / 8;
-                        if (feat < p.n_out) {
-                            uint4 packed[NI];
-                            if (mat < 2) {
-                                float4 cs[NI][4];     // (cos, sin) of the 8 feature pairs
-#pragma unroll
-                                for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 4) + 8 * it;
-                                    const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * half + ri);
-#pragma unroll
-                                    for (int q = 0; q < 4; ++q) cs[it][q] = nl < n_hi ? __ldg(src + q) : make_float4(1.f, 0.f, 1.f, 0.f);
-                                }
-#pragma unroll
-                                for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 4) + 8 * it;
-                                    const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
-                                    const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
-                                    const float4 y0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner);
-                                    const float4 y1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner + 4);
-                                    packed[it].x = pack_bf16x2(x0.x * cs[it][0].x + sgn * y0.x * cs[it][0].y, x0.y * cs[it][0].z + sgn * y0.y * cs[it][0].w);
-                                    packed[it].y = pack_bf16x2(x0.z * cs[it][1].x + sgn * y0.z * cs[it][1].y, x0.w * cs[it][1].z + sgn * y0.w * cs[it][1].w);
-                                    packed[it].z = pack_bf16x2(x1.x * cs[it][2].x + sgn * y1.x * cs[it][2].y, x1.y * cs[it][2].z + sgn * y1.y * cs[it][2].w);
-                                    packed[it].w = pack_bf16x2(x1.z * cs[it][3].x + sgn * y1.z * cs[it][3].y, x1.w * cs[it][3].z + sgn * y1.w * cs[it][3].w);
-                                }
-                            } else {
-#pragma unroll
-                                for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 4) + 8 * it;
-                                    const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
-                                    const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
-                                    packed[it] = make_uint4(pack_bf16x2(x0.x, x0.y), pack_bf16x2(x0.z, x0.w), pack_bf16x2(x1.x, x1.y),
-                                                            pack_bf16x2(x1.z, x1.w));
-                                }
-                            }
-                            if (mat == 0 || p.kv_rows == nullptr) {
-                                uint16_t* base = mat == 0 ? p.q_out + (size_t)c0 * p.n_out
-                                                          : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
-#pragma unroll
-                                for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 4) + 8 * it;
-                                    if (nl < n_hi) *reinterpret_cast<uint4*>(base + (size_t)nl * p.n_out + feat) = packed[it];
-                                }
-                            } else {
-                                // a subset of the tree: row t of the batch is tree node kv_rows[t]
-                                uint16_t* base = (mat == 1 ? p.kcache : p.vcache) + (size_t)p.prefix_len * p.n_out;
-#pragma unroll
-                                for (int it = 0; it < NI; ++it) {
-                                    const int nl = (et >> 4) + 8 * it;
-                                    if (nl < n_hi)
-                                        *reinterpret_cast<uint4*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
-                                }
-                            }
-                        }
-                    } else if (EPI == EPI_SWIGLU) {
-                        // features beyond n_out come out as silu(0)*0 = 0 (zero-padded weights): they are stored too,
-                        // so that the padded K block of the down projection's input reads as zeros.
-                        // thread -> 8 consecutive features = one 16-byte group of the packed layout, every 16th node
-                        const int j8 = (et & 7) * 8;
-                        const int feat = row0 + j8;
-                        constexpr int NI = kStagingCols / 16;
-#pragma unroll
-                        for (int it = 0; it < NI; ++it) {
-                            const int nl = (et >> 3) + 16 * it;
-                            const float4 g0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
-                            const float4 g1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
-                            const float4 u0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8);
-                            const float4 u1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8 + 4);
-                            uint4 o;
-                            o.x = pack_bf16x2(__fdividef(g0.x, 1.f + __expf(-g0.x)) * u0.x, __fdividef(g0.y, 1.f + __expf(-g0.y)) * u0.y);
-                            o.y = pack_bf16x2(__fdividef(g0.z, 1.f + __expf(-g0.z)) * u0.z, __fdividef(g0.w, 1.f + __expf(-g0.w)) * u0.w);
-                            o.z = pack_bf16x2(__fdividef(g1.x, 1.f + __expf(-g1.x)) * u1.x, __fdividef(g1.y, 1.f + __expf(-g1.y)) * u1.y);
-                            o.w = pack_bf16x2(__fdividef(g1.z, 1.f + __expf(-g1.z)) * u1.z, __fdividef(g1.w, 1.f + __expf(-g1.w)) * u1.w);
-                            if (nl < n_hi) *reinterpret_cast<uint4*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad)) = o;
-                        }
-                    } else if (EPI == EPI_LMHEAD) {
-                        for (int nl = warp - 2; nl < n_hi; nl += 4) {
-                            float best = -INFINITY;
-                            int bi = 0x7fffffff;
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                int ff = lane + 32 * i;
-                                float v = acc_s[nl * 128 + ff];
-                                if (row0 + ff < p.n_out && v > best) { best = v; bi = row0 + ff; }
-                            }
-#pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) {
-                                float ov = __shfl_xor_sync(0xffffffffu, best, o);
-                                int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                                if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-                            }
-                            if (lane == 0) {
-                                p.pmax[(size_t)tile * 128 + c0 + nl] = best;
-                                p.pidx[(size_t)tile * 128 + c0 + nl] = bi;
-                            }
-                            if (p.psum != nullptr) {
-                                // softmax statistics of this vocabulary tile at the given temperature, relative to the
-                                // tile's own maximum: Z = sum e, S1 = sum e * (logit - max), e = exp((logit - max) / t)
-                                float z = 0.f, s1 = 0.f;
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) {
-                                    int ff = lane + 32 * i;
-                                    if (row0 + ff < p.n_out) {
-                                        float d = acc_s[nl * 128 + ff] - best;
-                                        float e = exp2f(d * p.inv_temp_log2e);
-                                        z += e;
-                                        s1 = fmaf(e, d, s1);
-                                    }
-                                }
-#pragma unroll
-                                for (int o = 16; o > 0; o >>= 1) {
-                                    z += __shfl_xor_sync(0xffffffffu, z, o);
-                                    s1 += __shfl_xor_sync(0xffffffffu, s1, o);
-                                }
-                                if (lane == 0) {
-                                    p.psum[(size_t)tile * 128 + c0 + nl] = z;
-                                    p.ps1[(size_t)tile * 128 + c0 + nl] = s1;
-                                }
-                            }
-                        }
-                        if (p.cand != nullptr && et > 0 && et < p.T) {
-                            // logit of tree node et's own token under its parent's distribution, if this tile holds it
-                            const int pa = __ldg(p.tree_parent + et), tk = __ldg(p.tree_tokens + et);
-                            if (pa >= c0 && pa < c0 + n_hi && tk >= row0 && tk < row0 + 128 && tk < p.n_out)
-                                p.cand[et] = acc_s[(pa - c0) * 128 + (tk - row0)];
-                        }
-                    }
-                    epi_barrier();
-                }
-                if (gather && et == 0)
-                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
+// ---------------------------------------------------------------------------------------------------
+// Several projections of a decoder layer in ONE launch (O projection -> RMSNorm -> gate/up + SwiGLU -> down projection).
+// The ring, the accumulators and the role assignment are those of k_gemm_sk; what changes is that they live on across
+// the projections:
+//   * the W producer walks through the weights of all phases without ever waiting for anything but a free stage, so
+//     while the last epilogues of a phase run and the dependency below resolves, the ring fills with the next
+//     phase's weights;
+//   * the X producer of phase n + 1 waits until every CTA has finished phase n (a counter in global memory that each
+//     CTA's epilogue warps bump with release semantics once their stores are fenced) -- or, where an RMSNorm sits
+//     between the two phases, until the norm's rows are done: row t is normalised by the epilogue warps of CTA t, which
+//     wait for the same counter, fold the phase's split-K partial sums into the residual stream and write the packed
+//     bf16 activations;
+//   * data another CTA wrote with ordinary stores is read here by bulk copies (async proxy): writers and the reader
+//     both issue fence.proxy.async around the release / acquire pair.
+// Every wait is bounded (g_wait_limit_ns); on expiry the CTA raises its abort flag and leaves as k_gemm_sk does.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kMaxPhases = 3;
+#ifdef CATS_TRACE
+#define CHAIN_TR(slot) do { if (c.trace) c.trace[(size_t)blockIdx.x * 32 + (slot)] = globaltimer_ns(); } while (0)
+#else
+#define CHAIN_TR(slot) do { } while (0)
+#endif
+
+struct NormDev {
+    float* resid;              // [T][H] fp32 in/out: += the partial sums of the phase before the norm
+    const float* part;         // [n_part][T][H]
+    int n_part;
+    size_t part_stride;
+    const uint16_t* gain;      // [H] bf16
+    uint8_t* xn;               // packed activations out
+    int H, T, n_pad;
+    float eps;
+};
+
+struct ChainDev {
+    int n_phases;
+    int norm_after;            // the RMSNorm runs between phase norm_after and the next one (-1: no norm)
+    GemmDev ph[kMaxPhases];
+    NormDev norm;
+    int* sync;                 // [2 * kMaxPhases] counters, zero at launch: phase done, norm rows done
+#ifdef CATS_TRACE
+    unsigned long long* trace;
+#endif
+};
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Bounded wait until *ctr >= target (one thread).
+__device__ __forceinline__ bool grid_wait(const int* ctr, int target, volatile int* abort_flag) {
+    if (ld_acquire(ctr) >= target) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (ld_acquire(ctr) >= target) return true;
+        if ((it & 15u) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > g_wait_limit_ns) {
+                *abort_flag = 1;
+                return false;
             }
-            tc_fence_before_sync();
-            mbar_arrive(&ctrl->acc_empty[b]);
         }
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_acc, p.tmem_cols);
+}
+
+// RMSNorm of row t by 128 threads: resid[t] += sum of the partial sums (slot order), xn[t] = bf16(gain * resid * rsqrt(mean
+// square + eps)).  Rows of up to 4096 columns stay in registers between the two passes; longer ones are read back.
+__device__ __forceinline__ void chain_norm_row(const NormDev& n, int t, int et, float* red) {
+    const int n4 = n.H >> 2;                     // float4 columns
+    float4* r4 = reinterpret_cast<float4*>(n.resid + (size_t)t * n.H);
+    const bool single = n4 <= 1024;
+    float4 a[8];
+    float ss = 0.f;
+    for (int base = 0; base < n4; base += 1024) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int cl = base + et + 128 * j;
+            a[j] = cl < n4 ? __ldcg(r4 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int s = 0; s < n.n_part; s += 2) {
+            const float4* p0 = reinterpret_cast<const float4*>(n.part + (size_t)s * n.part_stride + (size_t)t * n.H);
+            const float4* p1 = reinterpret_cast<const float4*>(n.part + (size_t)(s + 1) * n.part_stride + (size_t)t * n.H);
+            const bool two = s + 1 < n.n_part;
+            float4 q0[8], q1[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int cl = base + et + 128 * j;
+                q0[j] = cl < n4 ? __ldcg(p0 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+                q1[j] = (two && cl < n4) ? __ldcg(p1 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                a[j].x += q0[j].x; a[j].y += q0[j].y; a[j].z += q0[j].z; a[j].w += q0[j].w;
+                if (two) { a[j].x += q1[j].x; a[j].y += q1[j].y; a[j].z += q1[j].z; a[j].w += q1[j].w; }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int cl = base + et + 128 * j;
+            if (cl < n4) {
+                ss += a[j].x * a[j].x + a[j].y * a[j].y + a[j].z * a[j].z + a[j].w * a[j].w;
+                if (n.n_part > 0) r4[cl] = a[j];
+            }
+        }
     }
-    if (threadIdx.x == 0 && ctrl->abort_flag) report(p.d_status, CATS_ERR_TIMEOUT);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((et & 31) == 0) red[et >> 5] = ss;
+    epi_barrier();
+    const float tot = (red[0] + red[1]) + (red[2] + red[3]);
+    const float rs = rsqrtf(tot / (float)n.H + n.eps);
+    for (int base = 0; base < n4; base += 1024) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int cl = base + et + 128 * j;
+            if (cl < n4) {
+                const float4 x = single ? a[j] : r4[cl];
+                const uint2 g = __ldg(reinterpret_cast<const uint2*>(n.gain) + cl);
+                uint2 o;
+                o.x = pack_bf16x2(__uint_as_float(g.x << 16) * (x.x * rs), __uint_as_float(g.x & 0xFFFF0000u) * (x.y * rs));
+                o.y = pack_bf16x2(__uint_as_float(g.y << 16) * (x.z * rs), __uint_as_float(g.y & 0xFFFF0000u) * (x.w * rs));
+                *reinterpret_cast<uint2*>(n.xn + packed_act_offset(t, cl >> 1, n.n_pad) + (size_t)(cl & 1) * 8) = o;
+            }
+        }
+    }
+    epi_barrier();      // red[] may be reused
+}
+
+template <int E0, int E1, int E2>
+__global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_chain(const __grid_constant__ ChainDev c) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    Pipe pp;
+    if (!pipe_setup(pp, smem_raw, c.ph[0].n_stages, c.ph[0].stage_bytes, c.ph[0].tmem_cols, c.ph[0].d_status)) return;
+    pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+    const int G = (int)gridDim.x;
+    int* const done = c.sync;                   // done[ph]: CTAs whose outputs of phase ph are written and fenced
+    int* const normed = c.sync + kMaxPhases;    // normed[ph]: rows the norm after phase ph has finished
+
+    if (warp == 0) {
+        // ---------------- W producer: all phases, never waits for anything but a free stage ----------------
+        if (lane == 0) {
+            const uint64_t pol = l2_policy_evict_first();
+            int i = 0;
+            bool ok = true;
+            CHAIN_TR(0);
+            for (int ph = 0; ph < c.n_phases && ok; ++ph) { ok = produce_units(c.ph[ph], cta_range(c.ph[ph], cta), pp, true, pol, i); CHAIN_TR(1 + ph); }
+            if (ok) warm_next_projection(c.ph[c.n_phases - 1], pp, cta);
+            if (*pp.abort_flag) drain_after_abort(pp, i);
+        }
+    } else if (warp == 6) {
+        // ---------------- X producer: phase 0 depends on the previous kernel, the others on the phase before ----------------
+        if (lane == 0) {
+            const uint64_t pol = l2_policy_evict_last();
+            pdl_wait();
+            CHAIN_TR(4);
+            int i = 0;
+            bool ok = true;
+            for (int ph = 0; ph < c.n_phases && ok; ++ph) {
+                if (ph > 0) {
+                    ok = (c.norm_after == ph - 1) ? grid_wait(normed + ph - 1, c.norm.T, pp.abort_flag)
+                                                  : grid_wait(done + ph - 1, G, pp.abort_flag);
+                    fence_proxy_async();
+                    CHAIN_TR(4 + ph);
+                }
+                if (ok) ok = produce_units(c.ph[ph], cta_range(c.ph[ph], cta), pp, false, pol, i);
+            }
+            if (*pp.abort_flag) drain_after_abort(pp, i);
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            int i = 0, seg = 0;
+            bool ok = true;
+            for (int ph = 0; ph < c.n_phases && ok; ++ph) {
+#ifdef CATS_TRACE
+                if (cta_range(c.ph[ph], cta).u1 > cta_range(c.ph[ph], cta).u0) { mbar_wait(&pp.ctrl->full[i % pp.S], (i / pp.S) & 1, pp.abort_flag); CHAIN_TR(7 + ph); }
+#endif
+                ok = mma_units(c.ph[ph], cta_range(c.ph[ph], cta), pp, i, seg);
+                CHAIN_TR(10 + ph);
+            }
+        }
+    } else if (warp < 6) {
+        // ---------------- epilogue warps; between phases: publish, and the RMSNorm rows ----------------
+        const int et = (warp - 2) * 32 + lane;
+        pdl_wait();
+        int seg = 0;
+        bool ok = true;
+#pragma unroll
+        for (int ph = 0; ph < kMaxPhases; ++ph) {
+            if (ph < c.n_phases) {
+                const GemmDev& p = c.ph[ph];
+                const CtaRange r = cta_range(p, cta);
+                if (ph == 0) epilogue_units<E0>(p, r, pp, cta, warp, lane, seg, ok);
+                else if (ph == 1) epilogue_units<E1>(p, r, pp, cta, warp, lane, seg, ok);
+                else epilogue_units<E2>(p, r, pp, cta, warp, lane, seg, ok);
+                if (et == 0) CHAIN_TR(13 + ph);
+                if (ph + 1 < c.n_phases) {
+                    // this CTA's outputs of the phase are complete: make them visible, then count the CTA in
+                    fence_proxy_async();
+                    __threadfence();
+                    epi_barrier();
+                    if (et == 0 && ok) atomicAdd(done + ph, 1);
+                    if (c.norm_after == ph && cta < c.norm.T) {
+                        if (et == 0 && ok) grid_wait(done + ph, G, pp.abort_flag);
+                        epi_barrier();
+                        if (et == 0) CHAIN_TR(16);
+                        ok = ok && !*pp.abort_flag;
+                        if (ok) {
+                            chain_norm_row(c.norm, cta, et, pp.acc_s);
+                            if (et == 0) CHAIN_TR(17);
+                            fence_proxy_async();
+                            __threadfence();
+                            epi_barrier();
+                            if (et == 0) { atomicAdd(normed + ph, 1); CHAIN_TR(18); }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    pipe_teardown(pp, c.ph[0].tmem_cols, c.ph[0].d_status);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -715,19 +1002,14 @@ GemmPlan gemm_plan(const GemmProblem& p) {
     return pl;
 }
 
-cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
-    static bool attr_set = false;
-    const int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_sk<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_LMHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    GemmPlan pl = gemm_plan(p);
-    GemmDev d = {};
+namespace {
+constexpr int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
+constexpr size_t kStagingBytes = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
+
+// Device-side description of one projection.  max_stages: upper bound on the ring depth (a single launch needs no more
+// stages than a CTA has units).  Returns the dynamic shared memory the kernel needs.
+size_t make_gemm_dev(const GemmProblem& p, const GemmPlan& pl, int max_stages, GemmDev& d) {
+    d = GemmDev{};
     d.epi = p.epi;
     d.T = p.T;
     d.n_pad = ((p.T + 15) / 16) * 16;
@@ -745,13 +1027,11 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     d.total_rem = pl.head_units > 0 ? d.n_tiles * (d.n_ku - pl.head_units) : 0;
     d.x_chunk_bytes = (uint32_t)d.n_pad * 128;
     d.stage_bytes = kUnitKb * kWChunk + ((kUnitKb * d.x_chunk_bytes + 1023) / 1024) * 1024;
-    size_t staging = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
-    int stages = (int)((kMaxSmem - kCtrlBytes - staging) / d.stage_bytes);
+    int stages = (int)((kMaxSmem - kCtrlBytes - kStagingBytes) / d.stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
-    if (stages > pl.units_per_cta) stages = pl.units_per_cta;
+    if (stages > max_stages) stages = max_stages;
     if (stages < 1) stages = 1;
     d.n_stages = stages;
-    size_t smem = (size_t)stages * d.stage_bytes + staging + kCtrlBytes;
     uint32_t cols = 32;
     while ((int)cols < 2 * d.n_pad) cols <<= 1;
     d.tmem_cols = cols;
@@ -793,6 +1073,23 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         d.warm_n_kb = (p.warm_next->K + 63) / 64;
         d.warm_total_chunks = (long long)gemm_num_tiles(*p.warm_next) * d.warm_n_kb;
     }
+    return (size_t)stages * d.stage_bytes + kStagingBytes + kCtrlBytes;
+}
+}  // namespace
+
+cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_sk<EPI_PARTIAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_QKV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_gemm_sk<EPI_LMHEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const GemmPlan pl = gemm_plan(p);
+    GemmDev d;
+    const size_t smem = make_gemm_dev(p, pl, pl.units_per_cta, d);
     switch (p.epi) {
         case EPI_PARTIAL: return launch_pdl(k_gemm_sk<EPI_PARTIAL>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
         case EPI_QKV: return launch_pdl(k_gemm_sk<EPI_QKV>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
@@ -800,6 +1097,62 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         case EPI_LMHEAD: return launch_pdl(k_gemm_sk<EPI_LMHEAD>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
         default: return cudaErrorInvalidValue;
     }
+}
+
+// True when the chained launch can be used on the current device: all its CTAs wait on one another, so every one of
+// them must be resident at the same time (one per SM).
+#ifdef CATS_TRACE
+unsigned long long* g_chain_trace = nullptr;
+extern "C" void cats_trace_chain(void* d_buf) { g_chain_trace = (unsigned long long*)d_buf; }
+#endif
+
+bool gemm_chain_supported() {
+    static const int ok = [] {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        return sms >= kGemmCtas ? 1 : 0;
+    }();
+    return ok != 0;
+}
+
+// O projection -> RMSNorm -> gate/up + SwiGLU -> down projection as one launch (k_gemm_chain).
+cudaError_t launch_layer_tail(const GemmProblem& o_proj, const NormProblem& norm, const GemmProblem& gate_up, const GemmProblem& down,
+                              int* sync, cudaStream_t st) {
+    auto kern = k_gemm_chain<EPI_PARTIAL, EPI_SWIGLU, EPI_PARTIAL>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    if (o_proj.epi != EPI_PARTIAL || gate_up.epi != EPI_SWIGLU || down.epi != EPI_PARTIAL) return cudaErrorInvalidValue;
+    ChainDev c = {};
+    c.n_phases = 3;
+    c.norm_after = 0;
+    const GemmProblem* probs[3] = {&o_proj, &gate_up, &down};
+    size_t smem = 0;
+    for (int i = 0; i < 3; ++i) {
+        const GemmPlan pl = gemm_plan(*probs[i]);
+        if (pl.n_ctas > kGemmCtas) return cudaErrorInvalidValue;
+        smem = make_gemm_dev(*probs[i], pl, kMaxStages, c.ph[i]);
+        if (i < 2) { c.ph[i].warm_ptr = nullptr; c.ph[i].warm_chunks = 0; }
+    }
+    c.norm.resid = norm.resid;
+    c.norm.part = norm.part;
+    c.norm.n_part = norm.n_part;
+    c.norm.part_stride = norm.part_stride;
+    c.norm.gain = (const uint16_t*)norm.gain;
+    c.norm.xn = (uint8_t*)norm.xn_packed;
+    c.norm.H = norm.H;
+    c.norm.T = norm.T;
+    c.norm.n_pad = (norm.T + 15) / 16 * 16;
+    c.norm.eps = norm.eps;
+    c.sync = sync;
+#ifdef CATS_TRACE
+    c.trace = g_chain_trace;
+#endif
+    return launch_pdl(kern, dim3(kGemmCtas), dim3(kGemmThreads), smem, st, c);
 }
 
 }  // namespace cats
