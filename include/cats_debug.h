@@ -36,12 +36,6 @@ int cats_debug_workspace_layout(const cats_model_cfg *cfg, int32_t T, size_t *ou
  * tcgen05 kernel. */
 void cats_debug_attention_kernel(int which);
 
-/* 1: O projection, RMSNorm, gate/up and down projection of a decoder layer run
- * as one chained launch (k_gemm_chain) where the device allows it; 0 (default):
- * one launch per stage (what a partial stage mask selects anyway).  For A/B
- * measurements and for testing both paths. */
-void cats_debug_chained_launch(int on);
-
 /* Limit of every bounded device-side wait, in nanoseconds, on the CURRENT
  * device (0 restores the default of 1 s).  Synchronises the device. */
 int cats_debug_wait_limit_ns(unsigned long long ns);

@@ -187,11 +187,6 @@ def attention_kernel(which: int) -> None:
     lib.cats_debug_attention_kernel(C.c_int(which))
 
 
-def chained_launch(on: bool) -> None:
-    """cats_debug_chained_launch: the second half of a decoder layer as one launch (default) or one launch per stage."""
-    lib.cats_debug_chained_launch(C.c_int(1 if on else 0))
-
-
 def wait_limit_ns(ns: int) -> None:
     """cats_debug_wait_limit_ns: limit of the bounded device-side waits on the current device (0: the default, 1 s)."""
     _check(lib.cats_debug_wait_limit_ns(C.c_ulonglong(ns)), "cats_debug_wait_limit_ns")

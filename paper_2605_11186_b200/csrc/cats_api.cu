@@ -12,7 +12,6 @@ thread_local int g_launch_count = 0;
 thread_local bool g_call_boundary = true;
 int g_debug_attn_kernel = -1;
 int g_debug_fault = 0;
-int g_debug_chain = 0;
 
 namespace {
 
@@ -73,7 +72,7 @@ Workspace carve(const cats_model_cfg* c, int T, void* base) {
     w.psum = (float*)take((size_t)vt * 128 * 4);
     w.ps1 = (float*)take((size_t)vt * 128 * 4);
     w.fix_part = (float*)take((size_t)kFixSlots * tpad * 128 * 4);
-    w.fix_flags = (int*)take((size_t)(kFixSlots + kChainSyncInts) * sizeof(int));   // the chained launch's counters follow the flags
+    w.fix_flags = (int*)take((size_t)kFixSlots * sizeof(int));
     w.scratch = (float*)take((size_t)T * c->hidden * 4);
     w.nodes = (int32_t*)take((size_t)CATS_MAX_TREE * sizeof(int32_t));
     w.bytes = off;
@@ -110,7 +109,7 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots + kChainSyncInts, st, d_status));
+                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -145,13 +144,6 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     else { nxt_after.epi = EPI_QKV; nxt_after.T = T; nxt_after.K = H; nxt_after.n_out = D; nxt_after.n_mats = 3; nxt_after.W[0] = next_w; }
     gd.warm_next = next_w ? &nxt_after : nullptr;
 
-    const bool tail_on = stage_on(3) && stage_on(4) && stage_on(5) && stage_on(6);
-    if (tail_on && g_debug_chain && gemm_chain_supported() && H % 4 == 0) {
-        // the second half of the layer as ONE launch: the weight ring lives on across the three projections
-        NormProblem nm = {resid, ws.part, pieces_o, ws.part_stride, w->mlp_norm, ws.xn, T, H, c->rms_eps};
-        CATS_CUDA(launch_layer_tail(go, nm, ggu, gd, ws.fix_flags + kFixSlots, st));
-        return pieces_d;
-    }
     go.warm_next = &ggu;
     if (stage_on(3)) CATS_CUDA(launch_gemm(go, st));
     if (stage_on(4))
@@ -175,7 +167,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
               const TypicalOut* ty = nullptr) {
     const int H = c->hidden, V = c->vocab;
     CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
-                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots + kChainSyncInts, st, d_status));
+                             nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
     g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -226,7 +218,6 @@ int cats_last_launch_count(void) { return g_launch_count; }
 /* Measurement and fault-injection hooks, declared in include/cats_debug.h. */
 void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
 void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which ? 1 : 0); }
-void cats_debug_chained_launch(int on) { g_debug_chain = on ? 1 : 0; }
 void cats_debug_inject_fault(int which) { g_debug_fault = (which == 1 || which == 2) ? which : 0; }
 int cats_debug_wait_limit_ns(unsigned long long ns) {
     if (ns == 0) ns = kWaitLimitNs;

@@ -28,9 +28,6 @@
 // Weight chunks of the first stages are requested before griddepcontrol.wait (weights never depend on
 // an earlier kernel).  Every wait (mbarrier or flag) is bounded; on expiry the CTA reports
 // CATS_ERR_TIMEOUT, lets its copies land, frees its TMEM and returns.
-#include <cstdio>
-#include <cstdlib>
-
 #include "cats_kernels.cuh"
 
 namespace cats {
@@ -77,9 +74,6 @@ struct GemmDev {
     int warm_upc, warm_n_ku, warm_n_kb;
     long long warm_total_chunks;
     int dbg_skip_publish;        // fault injection: contributors of shared tiles keep their flags to themselves
-#ifdef CATS_TRACE
-    int dbg_mma;                 // timing experiment: 1 = issue only the first MMA of every unit
-#endif
 };
 
 struct GemmCtrl {
@@ -152,11 +146,8 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The kernel is written as four roles (W producer, X producer, MMA issuer, epilogue warps), each a function over ONE
-// projection ("phase") that carries its pipeline counters in and out.  k_gemm_sk runs one phase; k_gemm_chain runs
-// several projections of a decoder layer back to back in one launch, so that the weight ring never drains between
-// them: the W producer runs ahead into the next projection's weights while the epilogues of this one finish and the
-// grid-wide dependency (all CTAs done, the RMSNorm in between) resolves.
+// The kernel is written as its roles (W producer, X producer, two MMA issuers, epilogue warps), each a function over the
+// CTA's share of one projection that carries its pipeline counters in and out.
 // ---------------------------------------------------------------------------------------------------
 struct CtaRange {
     long long u0, u1;     // this CTA's units in the phase's unit space (see below)
@@ -190,7 +181,6 @@ __device__ __forceinline__ CtaRange cta_range(const GemmDev& p, int cta) {
         const long long t0 = (long long)(cta / p.split_s) * p.n_ku;
         r.u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
         r.u1 = min(t0 + p.n_ku, r.u0 + (long long)p.units_per_cta);
-        if (cta >= p.n_tiles * p.split_s) r.u0 = r.u1 = 0;       // a CTA beyond this phase's grid (chained launches)
     } else {
         r.u0 = min(p.total_units, (long long)cta * p.units_per_cta);
         r.u1 = min(p.total_units, r.u0 + (long long)p.units_per_cta);
@@ -675,456 +665,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Several projections of a decoder layer in ONE launch (O projection -> RMSNorm -> gate/up + SwiGLU -> down projection),
-// with a weight buffer deep enough to keep HBM busy across the dependency gaps between them.
-//
-// Between two projections nothing can be multiplied for several microseconds: the last epilogues of the first, the
-// grid-wide hand-over (every CTA's outputs written and visible), the RMSNorm where there is one, the activations'
-// trip from L2.  A kernel boundary costs the same gap.  What a single launch can do about it is keep FETCHING: the W
-// producer never waits for anything but buffer space, so the gap is lost only once the buffer is full.  The shared-memory
-// ring alone (4 stages, 128 KB) is full after 3 us; here the weights go one step further, into the tensor memory the
-// accumulators leave free (384 of the 512 columns at T <= 64):
-//   TMA bulk copy -> shared-memory W stage -> tcgen05.cp (one thread, asynchronous) -> tensor-memory slot -> tcgen05.mma
-//   with the A operand read from tensor memory, the activations (B operand) from their own small shared-memory ring.
-// At T = 64 shared memory holds 5 W stages + 3 X stages and tensor memory 4 more units beside the accumulators: 288 KB of
-// weights per SM, more than 7 us of stream.  Issuing an MMA whose A operand sits in tensor memory costs its thread more
-// than 100 ns, which alone would cap the stream below the HBM rate: two threads issue, each half of every K block into
-// its own accumulator half, and the epilogue adds the halves (fixed order, deterministic).
-//   * the W producer and the copier walk through the weights of all phases without waiting for any dependency;
-//   * the X producer of phase n + 1 waits until every CTA has finished phase n (a counter in global memory that each
-//     CTA bumps once its epilogue warps have passed a barrier and one of them has fenced) -- or, where an RMSNorm sits
-//     between the two phases, until the norm's rows are done: row t is normalised by the epilogue warps of CTA t, which
-//     wait for the same counter, fold the phase's split-K partial sums into the residual stream and write the packed
-//     bf16 activations;
-//   * data another CTA wrote with ordinary stores is read here by bulk copies (async proxy): the reader issues
-//     fence.proxy.async after its acquire.
-// Every wait is bounded (g_wait_limit_ns); on expiry the CTA raises its abort flag and leaves as k_gemm_sk does.
-// ---------------------------------------------------------------------------------------------------
-constexpr int kMaxPhases = 3;
-constexpr int kChainThreads = 288;        // warps: 0 W producer, 1 and 8 MMA issuers, 2-5 epilogue, 6 X producer, 7 copier
-constexpr int kMaxXStages = 4;
-constexpr int kMaxTSlots = 8;
-constexpr int kSlotCols = 32 * kUnitKb;   // tensor-memory columns of one unit of W (kUnitKb chunks of 128 x 64 bf16)
-#ifdef CATS_TRACE
-#define CHAIN_TR(slot) do { if (c.trace) c.trace[(size_t)blockIdx.x * 32 + (slot)] = globaltimer_ns(); } while (0)
-#else
-#define CHAIN_TR(slot) do { } while (0)
-#endif
-
-struct NormDev {
-    float* resid;              // [T][H] fp32 in/out: += the partial sums of the phase before the norm
-    const float* part;         // [n_part][T][H]
-    int n_part;
-    size_t part_stride;
-    const uint16_t* gain;      // [H] bf16
-    uint8_t* xn;               // packed activations out
-    int H, T, n_pad;
-    float eps;
-};
-
-struct ChainDev {
-    int n_phases;
-    int norm_after;            // the RMSNorm runs between phase norm_after and the next one (-1: no norm)
-    int sw, sx, nt;            // W stages, X stages (shared memory), W slots (tensor memory)
-    int dual;                  // 1: two MMA issuers, each with its own accumulator halves (trees of up to 96 nodes)
-    uint32_t x_stage_bytes;
-    GemmDev ph[kMaxPhases];
-    NormDev norm;
-    int* sync;                 // [2 * kMaxPhases] counters, zero at launch: phase done, norm rows done
-#ifdef CATS_TRACE
-    unsigned long long* trace;
-    int dbg;
-#endif
-};
-
-struct DeepCtrl {              // barriers of the deep pipeline, behind GemmCtrl in the control block
-    uint64_t x_full[kMaxXStages], x_empty[kMaxXStages];
-    uint64_t t_full[kMaxTSlots], t_empty[kMaxTSlots];
-};
-static_assert(sizeof(GemmCtrl) + sizeof(DeepCtrl) <= kCtrlBytes, "control block too large");
-
-struct DeepPipe {
-    Pipe pp;                   // pp.stages: W stages of kUnitKb * kWChunk bytes; ctrl->full / empty are theirs
-    uint8_t* xs;               // X stages
-    DeepCtrl* dc;
-    int SW, SX, NT;
-    uint32_t x_stage_bytes;
-    uint32_t tmem_slots;       // tensor-memory address of W slot 0
-};
-
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
-
-// 128 rows x 32 bytes (one K = 16 slice of a K-major operand tile, described like an MMA operand) from shared memory to
-// 8 columns of tensor memory, row r to lane r.  Asynchronous; tcgen05.commit tracks its completion.
-__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t sdesc) {
-    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-
-// Bounded wait until *ctr >= target (one thread).
-__device__ __forceinline__ bool grid_wait(const int* ctr, int target, volatile int* abort_flag) {
-    if (ld_acquire(ctr) >= target) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (ld_acquire(ctr) >= target) return true;
-        if ((it & 15u) == 0) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > g_wait_limit_ns) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void unit_coords(const GemmDev& p, const CtaRange& r, int k, int& tile, int& kb, int& nk) {
-    const long long u = r.u0 + k;
-    tile = (int)(u / r.vlen);
-    kb = (r.koff + (int)(u - (long long)tile * r.vlen)) * kUnitKb;
-    nk = min(kUnitKb, p.n_kb - kb);
-}
-
-// W producer (one thread): bulk copies into the shared-memory W stages.  i: units issued so far over all phases.
-__device__ __forceinline__ bool deep_produce_w(const GemmDev& p, const CtaRange& r, const DeepPipe& dp, uint64_t pol, int& i) {
-    GemmCtrl* ctrl = dp.pp.ctrl;
-    const int n_units = (int)(r.u1 - r.u0);
-    for (int k = 0; k < n_units; ++k, ++i) {
-        const int s = i % dp.SW;
-        if (i >= dp.SW && !mbar_wait(&ctrl->empty[s], ((i / dp.SW) - 1) & 1, dp.pp.abort_flag)) return false;
-        int tile, kb, nk;
-        unit_coords(p, r, k, tile, kb, nk);
-        const uint32_t bytes = (uint32_t)nk * kWChunk;
-        mbar_expect_tx(&ctrl->full[s], bytes);
-        bulk_load(dp.pp.stages + (size_t)s * (kUnitKb * kWChunk), p.Wp + ((size_t)tile * p.n_kb + kb) * kWChunk, bytes, &ctrl->full[s], pol);
-    }
-    return true;
-}
-
-// X producer (one thread): the activations of every unit into their own ring.
-__device__ __forceinline__ bool deep_produce_x(const GemmDev& p, const CtaRange& r, const DeepPipe& dp, uint64_t pol, int& i) {
-    const int n_units = (int)(r.u1 - r.u0);
-    for (int k = 0; k < n_units; ++k, ++i) {
-        const int s = i % dp.SX;
-        if (i >= dp.SX && !mbar_wait(&dp.dc->x_empty[s], ((i / dp.SX) - 1) & 1, dp.pp.abort_flag)) return false;
-        int tile, kb, nk;
-        unit_coords(p, r, k, tile, kb, nk);
-        const uint32_t bytes = (uint32_t)nk * p.x_chunk_bytes;
-        mbar_expect_tx(&dp.dc->x_full[s], bytes);
-        bulk_load(dp.xs + (size_t)s * dp.x_stage_bytes, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &dp.dc->x_full[s], pol);
-    }
-    return true;
-}
-
-// Copier (one thread): every landed W stage goes on into a free tensor-memory slot; the stage is free again as soon as
-// the copy has completed.
-__device__ __forceinline__ bool deep_copy_w(const GemmDev& p, const CtaRange& r, const DeepPipe& dp, int& i, int dbg = 0) {
-    GemmCtrl* ctrl = dp.pp.ctrl;
-    const int n_units = (int)(r.u1 - r.u0);
-    for (int k = 0; k < n_units; ++k, ++i) {
-        const int s = i % dp.SW, t = i % dp.NT;
-        if (!mbar_wait(&ctrl->full[s], (i / dp.SW) & 1, dp.pp.abort_flag)) return false;
-        if (i >= dp.NT && !mbar_wait(&dp.dc->t_empty[t], ((i / dp.NT) - 1) & 1, dp.pp.abort_flag)) return false;
-        tc_fence_after_sync();
-        int tile, kb, nk;
-        unit_coords(p, r, k, tile, kb, nk);
-        const uint32_t a_addr = smem_u32(dp.pp.stages + (size_t)s * (kUnitKb * kWChunk));
-        const uint32_t slot = dp.tmem_slots + (uint32_t)(t * kSlotCols);
-        for (int j = 0; j < nk; ++j) {
-            const uint64_t da = umma_desc_sw128(a_addr + j * kWChunk);
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) if (dbg != 1) tmem_cp_128x256b(slot + (uint32_t)(j * 32 + kk * 8), da + 2 * kk);
-        }
-        umma_commit(&ctrl->empty[s]);
-        umma_commit(&dp.dc->t_full[t]);
-    }
-    return true;
-}
-
-// MMA issuer (one thread): A from the tensor-memory slot, B from the X ring.
-// With two issuers (dp.pp.dual) issuer `half` takes the K = 16 steps 2 * half and 2 * half + 1 of every K block and
-// accumulates into its own half of the accumulator: issuing, not executing, an MMA is what costs time (about 100 ns each).
-__device__ __forceinline__ bool deep_mma(const GemmDev& p, const CtaRange& r, const DeepPipe& dp, int& i, int& seg, int half, int dbg = 0) {
-    GemmCtrl* ctrl = dp.pp.ctrl;
-    const uint32_t idesc = umma_idesc_bf16_m128(p.n_pad);
-    bool ok = true;
-    for (long long u = r.u0; u < r.u1 && ok; ++seg) {
-        const long long tile_end = (u / r.vlen + 1) * r.vlen;
-        const long long seg_end = min(r.u1, tile_end);
-        const int b = seg & 1;
-        if (seg >= 2) ok = mbar_wait(&ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, dp.pp.abort_flag);
-        tc_fence_after_sync();
-        const uint32_t d_addr = dp.pp.tmem_acc + (uint32_t)(b * dp.pp.acc_stride + half * p.n_pad);
-        const int k_lo = dp.pp.dual ? 2 * half : 0, k_hi = dp.pp.dual ? 2 * half + 2 : 4;
-        bool first = true;
-        for (; u < seg_end && ok; ++u, ++i) {
-            const int t = i % dp.NT, xsi = i % dp.SX;
-            ok = mbar_wait(&dp.dc->t_full[t], (i / dp.NT) & 1, dp.pp.abort_flag) &&
-                 mbar_wait(&dp.dc->x_full[xsi], (i / dp.SX) & 1, dp.pp.abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
-            const int kb = (r.koff + (int)(u % r.vlen)) * kUnitKb;
-            const int nk = min(kUnitKb, p.n_kb - kb);
-            const uint32_t slot = dp.tmem_slots + (uint32_t)(t * kSlotCols);
-            const uint32_t b_addr = smem_u32(dp.xs + (size_t)xsi * dp.x_stage_bytes);
-            for (int j = 0; j < nk; ++j) {
-                const uint64_t db = umma_desc_sw128(b_addr + j * p.x_chunk_bytes);
-                for (int k = k_lo; k < k_hi; ++k)
-                    if (dbg != 2 || (j == 0 && k == k_lo)) umma_bf16_ts(d_addr, slot + (uint32_t)(j * 32 + k * 8), db + 2 * k, idesc, !(first && k == k_lo));
-                first = false;
-            }
-            umma_commit(&dp.dc->t_empty[t]);
-            umma_commit(&dp.dc->x_empty[xsi]);
-        }
-        umma_commit(&ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
-    }
-    return ok;
-}
-
-// RMSNorm of row t by the 128 epilogue threads: resid[t] += sum of the partial sums (slot order), xn[t] = bf16(gain * resid
-// * rsqrt(mean square + eps)).  Rows of up to 5120 columns are held in registers (kNormCols float4 per thread): their
-// residual values are requested BEFORE the wait for the producing phase (they do not depend on it), the partial sums two
-// slots at a time after it.  Longer rows take the same steps in chunks and read the new residual back for the second pass.
-constexpr int kNormCols = 10;
-
-__device__ __forceinline__ void chain_norm_row(const NormDev& n, int t, int et, float* red, const int* ready, int target,
-                                               volatile int* abort_flag, bool& ok) {
-    const int n4 = n.H >> 2;                     // float4 columns
-    const int chunk = 128 * kNormCols;
-    float4* r4 = reinterpret_cast<float4*>(n.resid + (size_t)t * n.H);
-    const bool single = n4 <= chunk;
-    float4 a[kNormCols];
-    if (single) {
-#pragma unroll
-        for (int j = 0; j < kNormCols; ++j) {
-            const int cl = et + 128 * j;
-            a[j] = cl < n4 ? __ldcg(r4 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    }
-    if (et == 0 && ok) grid_wait(ready, target, abort_flag);
-    epi_barrier();
-    ok = ok && !*abort_flag;
-    if (!ok) return;
-    float ss = 0.f;
-    for (int base = 0; base < n4; base += chunk) {
-        if (!single) {
-#pragma unroll
-            for (int j = 0; j < kNormCols; ++j) {
-                const int cl = base + et + 128 * j;
-                a[j] = cl < n4 ? __ldcg(r4 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
-        for (int s = 0; s < n.n_part; s += 2) {
-            const float4* p0 = reinterpret_cast<const float4*>(n.part + (size_t)s * n.part_stride + (size_t)t * n.H);
-            const float4* p1 = reinterpret_cast<const float4*>(n.part + (size_t)(s + 1) * n.part_stride + (size_t)t * n.H);
-            const bool two = s + 1 < n.n_part;
-            float4 q0[kNormCols], q1[kNormCols];
-#pragma unroll
-            for (int j = 0; j < kNormCols; ++j) {
-                const int cl = base + et + 128 * j;
-                q0[j] = cl < n4 ? __ldcg(p0 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
-                q1[j] = (two && cl < n4) ? __ldcg(p1 + cl) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int j = 0; j < kNormCols; ++j) {
-                a[j].x += q0[j].x; a[j].y += q0[j].y; a[j].z += q0[j].z; a[j].w += q0[j].w;
-                if (two) { a[j].x += q1[j].x; a[j].y += q1[j].y; a[j].z += q1[j].z; a[j].w += q1[j].w; }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < kNormCols; ++j) {
-            const int cl = base + et + 128 * j;
-            if (cl < n4) {
-                ss += a[j].x * a[j].x + a[j].y * a[j].y + a[j].z * a[j].z + a[j].w * a[j].w;
-                if (n.n_part > 0) r4[cl] = a[j];
-            }
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-    if ((et & 31) == 0) red[et >> 5] = ss;
-    epi_barrier();
-    const float tot = (red[0] + red[1]) + (red[2] + red[3]);
-    const float rs = rsqrtf(tot / (float)n.H + n.eps);
-    for (int base = 0; base < n4; base += chunk) {
-#pragma unroll
-        for (int j = 0; j < kNormCols; ++j) {
-            const int cl = base + et + 128 * j;
-            if (cl < n4) {
-                const float4 x = single ? a[j] : r4[cl];
-                const uint2 g = __ldg(reinterpret_cast<const uint2*>(n.gain) + cl);
-                uint2 o;
-                o.x = pack_bf16x2(__uint_as_float(g.x << 16) * (x.x * rs), __uint_as_float(g.x & 0xFFFF0000u) * (x.y * rs));
-                o.y = pack_bf16x2(__uint_as_float(g.y << 16) * (x.z * rs), __uint_as_float(g.y & 0xFFFF0000u) * (x.w * rs));
-                *reinterpret_cast<uint2*>(n.xn + packed_act_offset(t, cl >> 1, n.n_pad) + (size_t)(cl & 1) * 8) = o;
-            }
-        }
-    }
-}
-
-// 9 warps: one of the SM's four register partitions (16 K registers each) holds three of them, hence at most 170 registers.
-template <int E0, int E1, int E2>
-__global__ void __maxnreg__(168) k_gemm_chain(const __grid_constant__ ChainDev c) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const int warp = threadIdx.x >> 5;
-    const int lane = threadIdx.x & 31;
-    const int cta = blockIdx.x;
-    const int G = (int)gridDim.x;
-    // shared memory: W stages | X stages | staging tile | control block
-    DeepPipe dp;
-    dp.SW = c.sw; dp.SX = c.sx; dp.NT = c.nt;
-    dp.x_stage_bytes = c.x_stage_bytes;
-    dp.pp.stages = smem_raw;
-    dp.xs = smem_raw + (size_t)c.sw * (kUnitKb * kWChunk);
-    dp.pp.acc_s = reinterpret_cast<float*>(dp.xs + (size_t)c.sx * c.x_stage_bytes);
-    dp.pp.landing = nullptr;
-    dp.pp.ctrl = reinterpret_cast<GemmCtrl*>(reinterpret_cast<uint8_t*>(dp.pp.acc_s) + (size_t)kStagingCols * 128 * 4);
-    dp.dc = reinterpret_cast<DeepCtrl*>(dp.pp.ctrl + 1);
-    dp.pp.abort_flag = &dp.pp.ctrl->abort_flag;
-    dp.pp.S = c.sw;
-    if ((smem_u32(smem_raw) & 1023u) != 0) {
-        if (threadIdx.x == 0) report(c.ph[0].d_status, CATS_ERR_UNSUPPORTED);
-        return;
-    }
-    GemmCtrl* ctrl = dp.pp.ctrl;
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < c.sw; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], 1); }
-        const uint32_t n_iss = c.dual ? 2u : 1u;      // every MMA issuer commits to the barriers its operands and results hang on
-        for (int s = 0; s < c.sx; ++s) { mbar_init(&dp.dc->x_full[s], 1); mbar_init(&dp.dc->x_empty[s], n_iss); }
-        for (int s = 0; s < c.nt; ++s) { mbar_init(&dp.dc->t_full[s], 1); mbar_init(&dp.dc->t_empty[s], n_iss); }
-        mbar_init(&ctrl->acc_full[0], n_iss);
-        mbar_init(&ctrl->acc_full[1], n_iss);
-        mbar_init(&ctrl->acc_empty[0], 128);
-        mbar_init(&ctrl->acc_empty[1], 128);
-        ctrl->abort_flag = 0;
-        mbar_fence_init();
-    }
-    if (warp == 1) {
-        tmem_alloc(&ctrl->tmem_base, 512);      // accumulators and W slots: the whole tensor memory of the SM
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    dp.pp.tmem_acc = ctrl->tmem_base;
-    dp.pp.dual = c.dual;
-    dp.pp.acc_stride = (c.dual ? 2 : 1) * c.ph[0].n_pad;
-    dp.tmem_slots = ctrl->tmem_base + (uint32_t)(2 * dp.pp.acc_stride);
-    pdl_launch_dependents();
-    int* const done = c.sync;                   // done[ph]: CTAs whose outputs of phase ph are written and fenced
-    int* const normed = c.sync + kMaxPhases;    // normed[ph]: rows the norm after phase ph has finished
-
-    if (warp == 0) {
-        // ---------------- W producer: all phases, never waits for anything but a free stage ----------------
-        if (lane == 0) {
-            const uint64_t pol = l2_policy_evict_first();
-            int i = 0;
-            bool ok = true;
-            CHAIN_TR(0);
-            for (int ph = 0; ph < c.n_phases && ok; ++ph) { ok = deep_produce_w(c.ph[ph], cta_range(c.ph[ph], cta), dp, pol, i); CHAIN_TR(1 + ph); }
-            if (*dp.pp.abort_flag) drain_after_abort(dp.pp, i);
-        }
-    } else if (warp == 7) {
-        // ---------------- copier: shared-memory W stages on into tensor memory ----------------
-        if (lane == 0) {
-            int i = 0;
-            bool ok = true;
-            for (int ph = 0; ph < c.n_phases && ok; ++ph) ok = deep_copy_w(c.ph[ph], cta_range(c.ph[ph], cta), dp, i
-#ifdef CATS_TRACE
-                    , c.dbg
-#endif
-                    );
-        }
-    } else if (warp == 6) {
-        // ---------------- X producer: phase 0 depends on the previous kernel, the others on the phase before ----------------
-        if (lane == 0) {
-            const uint64_t pol = l2_policy_evict_last();
-            pdl_wait();
-            CHAIN_TR(4);
-            int i = 0;
-            bool ok = true;
-            for (int ph = 0; ph < c.n_phases && ok; ++ph) {
-                if (ph > 0) {
-                    ok = (c.norm_after == ph - 1) ? grid_wait(normed + ph - 1, c.norm.T, dp.pp.abort_flag)
-                                                  : grid_wait(done + ph - 1, G, dp.pp.abort_flag);
-                    fence_proxy_async();
-                    CHAIN_TR(4 + ph);
-                }
-                if (ok) ok = deep_produce_x(c.ph[ph], cta_range(c.ph[ph], cta), dp, pol, i);
-            }
-            if (*dp.pp.abort_flag) {      // let the copies in flight land (bounded) before the CTA goes away
-                volatile int ignore = 0;
-                for (int j = max(0, i - dp.SX); j < i; ++j) mbar_wait(&dp.dc->x_full[j % dp.SX], (j / dp.SX) & 1, &ignore);
-            }
-        }
-    } else if (warp == 8) {
-        // ---------------- second MMA issuer ----------------
-        if (lane == 0 && c.dual) {
-            int i = 0, seg = 0;
-            bool ok = true;
-            for (int ph = 0; ph < c.n_phases && ok; ++ph) ok = deep_mma(c.ph[ph], cta_range(c.ph[ph], cta), dp, i, seg, 1);
-        }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            int i = 0, seg = 0;
-            bool ok = true;
-            for (int ph = 0; ph < c.n_phases && ok; ++ph) {
-#ifdef CATS_TRACE
-                if (cta_range(c.ph[ph], cta).u1 > cta_range(c.ph[ph], cta).u0) {
-                    mbar_wait(&dp.dc->t_full[i % dp.NT], (i / dp.NT) & 1, dp.pp.abort_flag);
-                    mbar_wait(&dp.dc->x_full[i % dp.SX], (i / dp.SX) & 1, dp.pp.abort_flag);
-                    CHAIN_TR(7 + ph);
-                }
-#endif
-                ok = deep_mma(c.ph[ph], cta_range(c.ph[ph], cta), dp, i, seg, 0
-#ifdef CATS_TRACE
-                    , c.dbg
-#endif
-                    );
-                CHAIN_TR(10 + ph);
-            }
-        }
-    } else if (warp < 6) {
-        // ---------------- epilogue warps; between phases: publish, and the RMSNorm rows ----------------
-        const int et = (warp - 2) * 32 + lane;
-        pdl_wait();
-        int seg = 0;
-        bool ok = true;
-#pragma unroll
-        for (int ph = 0; ph < kMaxPhases; ++ph) {
-            if (ph < c.n_phases) {
-                const GemmDev& p = c.ph[ph];
-                const CtaRange r = cta_range(p, cta);
-                if (ph == 0) epilogue_units<E0>(p, r, dp.pp, cta, warp, lane, seg, ok);
-                else if (ph == 1) epilogue_units<E1>(p, r, dp.pp, cta, warp, lane, seg, ok);
-                else epilogue_units<E2>(p, r, dp.pp, cta, warp, lane, seg, ok);
-                if (et == 0) CHAIN_TR(13 + ph);
-                if (ph + 1 < c.n_phases) {
-                    // this CTA's outputs of the phase are complete: after the barrier one thread fences for all and counts
-                    // the CTA in (the barrier orders the other threads' stores before that fence)
-                    epi_barrier();
-                    if (et == 0 && ok) { __threadfence(); atomicAdd(done + ph, 1); }
-                    if (c.norm_after == ph && cta < c.norm.T) {
-                        if (et == 0) CHAIN_TR(16);
-                        chain_norm_row(c.norm, cta, et, dp.pp.acc_s, done + ph, G, dp.pp.abort_flag, ok);
-                        if (et == 0) CHAIN_TR(17);
-                        epi_barrier();
-                        if (et == 0 && ok) { __threadfence(); atomicAdd(normed + ph, 1); CHAIN_TR(18); }
-                    }
-                }
-            }
-        }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after_sync();
-        tmem_dealloc(dp.pp.tmem_acc, 512);
-    }
-    if (threadIdx.x == 0 && ctrl->abort_flag) report(c.ph[0].d_status, CATS_ERR_TIMEOUT);
-}
-
-// ---------------------------------------------------------------------------------------------------
 // Weight packing: nn.Linear [rows][cols] bf16 -> 16 KB chunks (tile, K block) in the tcgen05 K-major
 // 128-byte-swizzle layout.  layout 0: n_src matrices stacked, each padded to whole 128-row tiles.
 // layout 1: two matrices (gate, up) interleaved as tiles of 64 + 64 rows.  Rows and columns beyond
@@ -1226,15 +766,17 @@ GemmPlan gemm_plan(const GemmProblem& p) {
         // it and run its epilogue.  Instead: one owner CTA per tile runs the first `a` K units and the epilogue; the
         // other CTAs ("helpers") share the remaining units of all tiles, with shorter shares than an owner's, so their
         // partial tiles are in L2 before an owner needs them.  How much shorter grows with the tree (the published tiles
-        // and the owner's epilogue grow with it).  Measured on the 7B forward, 32 units per tile, owner units a:
-        //   T = 16:  a = 22 / 23 / 24 / 25 -> 3.136 / 3.115 / 3.128 / 3.151 ms
-        //   T = 64:  a = 23 / 24 / 25 / 26 -> 3.539 / 3.506 / 3.484 / 3.503 ms
-        //   T = 128: a = 25 / 26 / 27 / 28 -> 4.199 / 4.144 / 4.163 / 4.187 ms
+        // and the owner's epilogue grow with it).  Measured on the 7B forward (two MMA issuers), 32 units per tile, owner units a:
+        //   T = 16:  a = 23 / 24 / 25 / 26 / 28 -> 2.926 / 2.896 / 2.889 / 2.906 / 2.937 ms
+        //   T = 64:  a = 24 / 25 / 26 / 27 / 28 -> 3.322 / 3.301 / 3.230 / 3.241 / 3.255 ms
+        //   T = 128: a = 25 / 26 / 27 / 28      -> 4.072 / 3.955 / 3.976 / 3.979 ms
+        // (an owner's SM pulls more once the helpers have finished, so the optimum is flat towards large shares: with
+        // a = 31, next to no help at all, the forward is only 2 % slower.)
         const int h = kGemmCtas - tiles;
         const double rho = (double)tiles / h;
         int lg = 0;                                    // log2(n_pad / 16): 0, 1, 2, 3 for trees of up to 16, 32, 64, 128 nodes
         for (int n = ((p.T + 15) / 16) * 16; n > 16; n = (n + 1) / 2) ++lg;
-        const double lead = (5.0 + 3.0 * lg) * n_ku / 32.0;
+        const double lead = (10.0 + 1.5 * lg) * n_ku / 32.0;
         int a = (int)((rho * n_ku + lead) / (1.0 + rho) + 0.999);
         if (a > n_ku - 1) a = n_ku - 1;
         const int R = n_ku - a;
@@ -1263,7 +805,6 @@ GemmPlan gemm_plan(const GemmProblem& p) {
 
 namespace {
 constexpr int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
-constexpr int kChainSmem = 226 * 1024; // the chained launch shares its SM with nothing
 constexpr size_t kStagingBytes = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
 
 // Device-side description of one projection.  max_stages: upper bound on the ring depth (a single launch needs no more
@@ -1320,9 +861,6 @@ size_t make_gemm_dev(const GemmProblem& p, const GemmPlan& pl, int max_stages, G
     d.cand = p.cand;
     d.d_status = p.d_status;
     d.dbg_skip_publish = g_debug_fault == 1 ? 1 : 0;
-#ifdef CATS_TRACE
-    { const char* e = getenv("CATS_MMA_DBG"); d.dbg_mma = e ? atoi(e) : 0; }
-#endif
     d.warm_ptr = nullptr;
     d.warm_chunks = 0;
     if (p.warm_next != nullptr && p.warm_next->W[0] != nullptr) {
@@ -1360,77 +898,6 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
         case EPI_LMHEAD: return launch_pdl(k_gemm_sk<EPI_LMHEAD>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
         default: return cudaErrorInvalidValue;
     }
-}
-
-// True when the chained launch can be used on the current device: all its CTAs wait on one another, so every one of
-// them must be resident at the same time (one per SM).
-#ifdef CATS_TRACE
-unsigned long long* g_chain_trace = nullptr;
-extern "C" void cats_trace_chain(void* d_buf) { g_chain_trace = (unsigned long long*)d_buf; }
-#endif
-
-bool gemm_chain_supported() {
-    static const int ok = [] {
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
-        return sms >= kGemmCtas ? 1 : 0;
-    }();
-    return ok != 0;
-}
-
-// O projection -> RMSNorm -> gate/up + SwiGLU -> down projection as one launch (k_gemm_chain).
-cudaError_t launch_layer_tail(const GemmProblem& o_proj, const NormProblem& norm, const GemmProblem& gate_up, const GemmProblem& down,
-                              int* sync, cudaStream_t st) {
-    auto kern = k_gemm_chain<EPI_PARTIAL, EPI_SWIGLU, EPI_PARTIAL>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    if (o_proj.epi != EPI_PARTIAL || gate_up.epi != EPI_SWIGLU || down.epi != EPI_PARTIAL) return cudaErrorInvalidValue;
-    ChainDev c = {};
-    c.n_phases = 3;
-    c.norm_after = 0;
-    const GemmProblem* probs[3] = {&o_proj, &gate_up, &down};
-    for (int i = 0; i < 3; ++i) {
-        const GemmPlan pl = gemm_plan(*probs[i]);
-        if (pl.n_ctas > kGemmCtas) return cudaErrorInvalidValue;
-        make_gemm_dev(*probs[i], pl, kMaxStages, c.ph[i]);
-        c.ph[i].warm_ptr = nullptr;
-        c.ph[i].warm_chunks = 0;
-    }
-    // shared memory: W stages, X stages, staging tile, control block; tensor memory: two accumulators, the rest W slots
-    const int n_pad = c.ph[0].n_pad;
-    c.x_stage_bytes = ((kUnitKb * c.ph[0].x_chunk_bytes + 1023) / 1024) * 1024;
-    c.sx = c.x_stage_bytes <= 16384 ? 3 : 2;
-    const size_t fixed = (size_t)c.sx * c.x_stage_bytes + (size_t)kStagingCols * 128 * 4 + kCtrlBytes;
-    c.sw = (int)((kChainSmem - fixed) / (kUnitKb * kWChunk));
-    if (c.sw > kMaxStages) c.sw = kMaxStages;
-    c.dual = 4 * n_pad + 2 * kSlotCols <= 512 ? 1 : 0;
-    c.nt = (512 - (c.dual ? 4 : 2) * n_pad) / kSlotCols;
-    if (c.nt > kMaxTSlots) c.nt = kMaxTSlots;
-    if (c.sw < 2 || c.nt < 2) return cudaErrorInvalidValue;
-    const size_t smem = (size_t)c.sw * (kUnitKb * kWChunk) + fixed;
-    c.norm.resid = norm.resid;
-    c.norm.part = norm.part;
-    c.norm.n_part = norm.n_part;
-    c.norm.part_stride = norm.part_stride;
-    c.norm.gain = (const uint16_t*)norm.gain;
-    c.norm.xn = (uint8_t*)norm.xn_packed;
-    c.norm.H = norm.H;
-    c.norm.T = norm.T;
-    c.norm.n_pad = (norm.T + 15) / 16 * 16;
-    c.norm.eps = norm.eps;
-    c.sync = sync;
-#ifdef CATS_TRACE
-    c.trace = g_chain_trace;
-    { const char* e = getenv("CATS_CHAIN_DBG"); c.dbg = e ? atoi(e) : 0; }
-#endif
-    cudaError_t e = launch_pdl(kern, dim3(kGemmCtas), dim3(kChainThreads), smem, st, c);
-    if (e != cudaSuccess) fprintf(stderr, "launch_layer_tail: %s (smem %zu sw %d sx %d nt %d dual %d)\n", cudaGetErrorString(e), smem, c.sw, c.sx, c.nt, c.dual);
-    return e;
 }
 
 }  // namespace cats

@@ -16,7 +16,6 @@ extern thread_local bool g_call_boundary;
 
 // Measurement / fault-injection state set through the cats_debug_* hooks (include/cats_debug.h); process-wide.
 extern int g_debug_attn_kernel;   // -1: attention kernel chosen by shape; 0: mma.sync kernel; 1: tcgen05 kernel
-extern int g_debug_chain;        // 1: the second half of a decoder layer runs as one chained launch where possible (default 0)
 extern int g_debug_fault;         // 0: none; 1: a helper CTA of a projection never publishes; 2: the attention loader drops Q
 cudaError_t set_wait_limit_gemm(unsigned long long ns);
 cudaError_t set_wait_limit_attn(unsigned long long ns);
@@ -126,24 +125,6 @@ struct GemmPlan {
     int head_units;      // > 0: one owner CTA per tile runs this many K units, helper CTAs share the rest
     int help_upc;        //      units per helper CTA
 };
-
-// The RMSNorm that sits between two projections of a chained launch.
-struct NormProblem {
-    float* resid;            // [T][H] fp32 in/out
-    const float* part;       // split-K partial sums of the projection before the norm, [n_part][T][H]
-    int n_part;
-    size_t part_stride;
-    const void* gain;        // [H] bf16
-    void* xn_packed;         // packed activations out
-    int T, H;
-    float eps;
-};
-constexpr int kChainSyncInts = 8;   // counters of a chained launch, kept behind the kFixSlots flags and zeroed with them
-bool gemm_chain_supported();
-// O projection -> RMSNorm -> gate/up + SwiGLU -> down projection of one decoder layer as ONE launch.  sync: kChainSyncInts
-// ints, zero at launch.  Only the down projection's warm_next is honoured.
-cudaError_t launch_layer_tail(const GemmProblem& o_proj, const NormProblem& norm, const GemmProblem& gate_up, const GemmProblem& down,
-                              int* sync, cudaStream_t st);
 
 // Number of 128-row tiles the problem has (SwiGLU: tiles of 64 gate + 64 up rows).
 int gemm_num_tiles(const GemmProblem& p);
