@@ -115,9 +115,6 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
     g.q_out = ws.q; g.kcache = kc; g.vcache = vc; g.rope = ws.rope; g.head_dim = c->head_dim; g.prefix_len = P; g.kv_rows = nodes;
     g.d_status = d_status;
-    GemmProblem nxt = {};
-    nxt.epi = EPI_PARTIAL; nxt.T = T; nxt.K = D; nxt.n_out = H; nxt.n_mats = 1; nxt.W[0] = w->wo;
-    g.warm_next = &nxt;
     if (stage_on(1)) CATS_CUDA(launch_gemm(g, st));
 
     AttnProblem a = {};
@@ -139,17 +136,10 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     gd.epi = EPI_PARTIAL; gd.T = T; gd.K = F; gd.n_out = H; gd.n_mats = 1; gd.W[0] = w->w_down; gd.X = ws.act;
     gd.fix_part = ws.fix_part; gd.fix_flags = ws.fix_flags; gd.part = ws.part; gd.part_stride = ws.part_stride; gd.d_status = d_status;
     const int pieces_d = gemm_plan(gd).max_pieces;
-    GemmProblem nxt_after = {};
-    if (next_is_head) { nxt_after.epi = EPI_LMHEAD; nxt_after.T = T; nxt_after.K = H; nxt_after.n_out = c->vocab; nxt_after.n_mats = 1; nxt_after.W[0] = next_w; }
-    else { nxt_after.epi = EPI_QKV; nxt_after.T = T; nxt_after.K = H; nxt_after.n_out = D; nxt_after.n_mats = 3; nxt_after.W[0] = next_w; }
-    gd.warm_next = next_w ? &nxt_after : nullptr;
-
-    go.warm_next = &ggu;
     if (stage_on(3)) CATS_CUDA(launch_gemm(go, st));
     if (stage_on(4))
         CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
                                  nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st, d_status));
-    ggu.warm_next = &gd;
     if (stage_on(5)) CATS_CUDA(launch_gemm(ggu, st));
     if (stage_on(6)) CATS_CUDA(launch_gemm(gd, st));
     return pieces_d;

@@ -36,7 +36,7 @@ namespace cats {
 #define CATS_GEMM_DUAL 1
 #endif
 constexpr int kGemmDualIssue = CATS_GEMM_DUAL;       // 1: two threads issue the MMAs (see mma_units)
-constexpr int kGemmThreads = kGemmDualIssue ? 256 : 224;
+constexpr int kGemmThreads = 384;      // warps: 0 W producer, 1 and 7 MMA issuers, 6 X producer, 2-5 and 8-11 epilogue groups
 constexpr int kCtrlBytes = 512;
 constexpr int kMaxStages = 14;
 constexpr int kWChunk = 16384;        // 128 rows x 64 bf16
@@ -69,10 +69,6 @@ struct GemmDev {
     const int32_t *tree_parent, *tree_tokens;   //   [T]
     float* cand;                  //   [T]: logit of every node's own token at its parent
     int32_t* d_status;
-    const uint8_t* warm_ptr;     // next projection's packed weights: this CTA's first chunks of it
-    int warm_chunks;             // 16 KB chunks to pull through a landing buffer (warms L2)
-    int warm_upc, warm_n_ku, warm_n_kb;
-    long long warm_total_chunks;
     int dbg_skip_publish;        // fault injection: contributors of shared tiles keep their flags to themselves
 };
 
@@ -81,13 +77,15 @@ struct GemmCtrl {
     uint64_t empty[kMaxStages];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
-    uint64_t warm;
     uint32_t tmem_base;
     int abort_flag;
 };
 static_assert(sizeof(GemmCtrl) <= kCtrlBytes, "control block too large");
 
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+constexpr int kEpiGroups = 2;         // groups of four epilogue warps (warps 2-5 and 8-11)
+constexpr size_t kStagingBytes = (size_t)kEpiGroups * kStagingCols * 128 * 4;   // one staging tile per group
+__device__ __forceinline__ void epi_barrier(int group) { asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory"); }
+__device__ __forceinline__ void epi_barrier_all() { asm volatile("bar.sync 3, %0;" ::"n"(128 * kEpiGroups) : "memory"); }
 
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar, uint64_t policy) {
     asm volatile(
@@ -113,8 +111,8 @@ __device__ __forceinline__ void acc_ld16(uint32_t taddr, uint32_t dual, float* v
 }
 
 __device__ __forceinline__ void store_tile_transposed(uint32_t taddr, uint32_t dual, int n_pad, int n_valid, float* acc_s, int f, int et,
-                                                      float* dst, size_t row_stride, int feat_limit) {
-    for (int c0 = 0; c0 < n_valid; c0 += kStagingCols) {
+                                                      int group, float* dst, size_t row_stride, int feat_limit) {
+    for (int c0 = group * kStagingCols; c0 < n_valid; c0 += kEpiGroups * kStagingCols) {
 #pragma unroll
         for (int hc = 0; hc < kStagingCols / 16; ++hc) {
             if (c0 + hc * 16 >= n_pad) break;
@@ -123,7 +121,7 @@ __device__ __forceinline__ void store_tile_transposed(uint32_t taddr, uint32_t d
 #pragma unroll
             for (int i = 0; i < 16; ++i) acc_s[(hc * 16 + i) * 128 + f] = v[i];
         }
-        epi_barrier();
+        epi_barrier(group);
         const int l4 = et & 31;
 #pragma unroll
         for (int k = 0; k < kStagingCols / 4; ++k) {
@@ -132,7 +130,7 @@ __device__ __forceinline__ void store_tile_transposed(uint32_t taddr, uint32_t d
                 *reinterpret_cast<float4*>(dst + (size_t)(c0 + nl) * row_stride + l4 * 4) =
                     *reinterpret_cast<const float4*>(acc_s + nl * 128 + l4 * 4);
         }
-        epi_barrier();
+        epi_barrier(group);
     }
 }
 
@@ -192,7 +190,6 @@ __device__ __forceinline__ CtaRange cta_range(const GemmDev& p, int cta) {
 struct Pipe {               // the CTA's pipeline resources, the same for every phase of a launch
     uint8_t* stages;        // ring of S stages
     float* acc_s;           // [32][128] fp32 epilogue staging tile
-    uint8_t* landing;       // 16 KB, contents never read
     GemmCtrl* ctrl;
     volatile int* abort_flag;
     uint32_t tmem_acc;
@@ -227,25 +224,6 @@ __device__ __forceinline__ bool produce_units(const GemmDev& p, const CtaRange& 
         }
     }
     return true;
-}
-
-// Real copies of the first chunks the same CTA of the NEXT launch's projection will read, into a landing buffer nobody
-// reads: they leave those lines in L2 while this kernel drains and runs its last epilogue.
-__device__ __forceinline__ void warm_next_projection(const GemmDev& p, const Pipe& pp, int cta) {
-    if (p.warm_ptr == nullptr || p.warm_chunks <= 0) return;
-    // first chunk of this CTA's range in the next matrix: unit cta * upc -> (tile, K block)
-    const long long wu = (long long)cta * p.warm_upc;
-    const long long wt = wu / p.warm_n_ku;
-    long long first = wt * p.warm_n_kb + (wu - wt * p.warm_n_ku) * kUnitKb;
-    long long n = min((long long)p.warm_chunks, p.warm_total_chunks - first);
-    if (n < 0) n = 0;
-    mbar_expect_tx(&pp.ctrl->warm, (uint32_t)n * kWChunk);
-    for (long long j = 0; j < n; ++j)
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                     ::"r"(smem_u32(pp.landing)), "l"(p.warm_ptr + (size_t)(first + j) * kWChunk), "r"(kWChunk), "r"(smem_u32(&pp.ctrl->warm))
-                     : "memory");
-    volatile int ignore = 0;
-    mbar_wait(&pp.ctrl->warm, 0, &ignore);   // the landing buffer must stay alive until the copies have landed
 }
 
 // After an abort: let the copies in flight land (bounded) before the CTA goes away.  i: units issued by this producer.
@@ -290,13 +268,18 @@ __device__ __forceinline__ bool mma_units(const GemmDev& p, const CtaRange& r, c
     return ok;
 }
 
-// The four epilogue warps (128 threads) over one phase.  seg: accumulator segments so far over all phases.
+// One group of four epilogue warps (128 threads) over the CTA's share of the projection.  seg: accumulator segments so far.
 template <int EPI>
 __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, int cta, int warp, int lane,
-                                               int& seg, bool& ok) {
+                                               int group, int& seg, bool& ok) {
+    // Two groups of four warps share every accumulator: group g takes the 32-node staging rounds g, g + 2, ... (trees of
+    // up to 32 nodes leave group 1 nothing to do but arrive).  Each group has its own staging tile and its own barrier.
     const int q4 = warp & 3;               // TMEM lane quadrant this warp may read
     const int f = q4 * 32 + lane;          // accumulator row = weight row inside the tile
-    const int et = (warp - 2) * 32 + lane; // 0..127 among the epilogue threads
+    const int ew = group == 0 ? warp - 2 : warp - 8;   // warp index inside the group
+    const int et = ew * 32 + lane;         // 0..127 among the group's threads
+    float* const acc_s = pp.acc_s + (size_t)group * kStagingCols * 128;
+    const int c_first = group * kStagingCols, c_step = kEpiGroups * kStagingCols;
     for (long long u = r.u0; u < r.u1; ++seg) {
         const int tile = (int)(u / r.vlen);
         const long long tile_begin = (long long)tile * r.vlen;
@@ -322,9 +305,9 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
             g_n = (head && !tail) ? last_cta - cta : 0;
         }
         // A tile this CTA owns but shares with other CTAs: their partial tiles are usually published long before
-        // this CTA's own part is accumulated, so fetch them (first 64 nodes) while waiting for the accumulator.
+        // this CTA's own part is accumulated, so fetch them (the group's first 32 nodes) while waiting for the accumulator.
         const bool gather = head && g_n > 0 && EPI != EPI_PARTIAL;
-        float pre[64];
+        float pre[kStagingCols];
         if (ok && gather) {
             if (et == 0) {
                 unsigned long long t0 = globaltimer_ns();
@@ -334,15 +317,15 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                     }
                 }
             }
-            epi_barrier();
+            epi_barrier(group);
             ok = !*pp.abort_flag;
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
+            for (int cc = 0; cc < kStagingCols / 16; ++cc) {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) pre[cc * 16 + i] = 0.f;
-                if (ok && cc * 16 < p.n_pad) {
+                if (ok && c_first + cc * 16 < p.n_pad) {
                     for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
-                        const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(cc * 16) * 128 + f;
+                        const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c_first + cc * 16) * 128 + f;
 #pragma unroll
                         for (int i = 0; i < 16; ++i) pre[cc * 16 + i] += __ldcg(src + (size_t)i * 128);
                     }
@@ -363,9 +346,9 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
         } else if (EPI == EPI_PARTIAL) {
             const int feat = row0 + f;
             const int piece = p.split_s > 0 ? cta % p.split_s : cta - head_cta;
-            store_tile_transposed(taddr, dual, p.n_pad, p.T, pp.acc_s, f, et, p.part + (size_t)piece * p.part_stride + row0,
+            store_tile_transposed(taddr, dual, p.n_pad, p.T, acc_s, f, et, group, p.part + (size_t)piece * p.part_stride + row0,
                                   (size_t)p.n_out, p.n_out - row0);
-            if (head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
+            if (group == 0 && head && p.split_s == 0 && feat < p.n_out) {   // slots no piece of this tile writes must read as zero
                 for (int sl = last_cta - head_cta + 1; sl < p.max_pieces; ++sl) {
                     float* z = p.part + (size_t)sl * p.part_stride + feat;
                     for (int n = 0; n < p.T; ++n) z[(size_t)n * p.n_out] = 0.f;
@@ -373,15 +356,15 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
             }
         } else if (!head) {
             // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
-            store_tile_transposed(taddr, dual, p.n_pad, p.n_pad, pp.acc_s, f, et, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
+            store_tile_transposed(taddr, dual, p.n_pad, p.n_pad, acc_s, f, et, group, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
             __threadfence();
-            epi_barrier();
-            if (et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
+            epi_barrier_all();       // both groups have stored and fenced their rounds
+            if (group == 0 && et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
         } else {
             // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
 #pragma unroll
-            for (int qc = 0; qc < CATS_MAX_TREE / kStagingCols; ++qc) {
-                const int c0 = qc * kStagingCols;
+            for (int qi = 0; qi < CATS_MAX_TREE / kStagingCols / kEpiGroups; ++qi) {
+                const int c0 = c_first + qi * c_step;
                 if (c0 >= p.T || !ok) break;
 #pragma unroll
                 for (int hc = 0; hc < kStagingCols / 16; ++hc) {
@@ -390,9 +373,9 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                     float v[16];
                     acc_ld16(taddr + c0 + c, dual, v);
                     if (gather) {
-                        if (qc * (kStagingCols / 16) + hc < 4) {
+                        if (qi == 0) {
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) v[i] += pre[((qc * (kStagingCols / 16) + hc) & 3) * 16 + i];
+                            for (int i = 0; i < 16; ++i) v[i] += pre[hc * 16 + i];
                         } else {
                             for (int c2 = g_first; c2 < g_first + g_n; ++c2) {
                                 const float* src = p.fix_part + (size_t)c2 * p.n_pad * 128 + (size_t)(c0 + c) * 128 + f;
@@ -409,9 +392,9 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                         }
                     }
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) pp.acc_s[(c + i) * 128 + f] = v[i];
+                    for (int i = 0; i < 16; ++i) acc_s[(c + i) * 128 + f] = v[i];
                 }
-                epi_barrier();
+                epi_barrier(group);
                 const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
                 if (EPI == EPI_QKV) {
                     // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
@@ -439,10 +422,10 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
 #pragma unroll
                             for (int it = 0; it < NI; ++it) {
                                 const int nl = (et >> 4) + 8 * it;
-                                const float4 x0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
-                                const float4 x1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
-                                const float4 y0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + partner);
-                                const float4 y1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + partner + 4);
+                                const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                                const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
+                                const float4 y0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner);
+                                const float4 y1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner + 4);
                                 packed[it].x = pack_bf16x2(x0.x * cs[it][0].x + sgn * y0.x * cs[it][0].y, x0.y * cs[it][0].z + sgn * y0.y * cs[it][0].w);
                                 packed[it].y = pack_bf16x2(x0.z * cs[it][1].x + sgn * y0.z * cs[it][1].y, x0.w * cs[it][1].z + sgn * y0.w * cs[it][1].w);
                                 packed[it].z = pack_bf16x2(x1.x * cs[it][2].x + sgn * y1.x * cs[it][2].y, x1.y * cs[it][2].z + sgn * y1.y * cs[it][2].w);
@@ -452,8 +435,8 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
 #pragma unroll
                             for (int it = 0; it < NI; ++it) {
                                 const int nl = (et >> 4) + 8 * it;
-                                const float4 x0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
-                                const float4 x1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
+                                const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                                const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
                                 packed[it] = make_uint4(pack_bf16x2(x0.x, x0.y), pack_bf16x2(x0.z, x0.w), pack_bf16x2(x1.x, x1.y),
                                                         pack_bf16x2(x1.z, x1.w));
                             }
@@ -487,10 +470,10 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
 #pragma unroll
                     for (int it = 0; it < NI; ++it) {
                         const int nl = (et >> 3) + 16 * it;
-                        const float4 g0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8);
-                        const float4 g1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + j8 + 4);
-                        const float4 u0 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + 64 + j8);
-                        const float4 u1 = *reinterpret_cast<const float4*>(pp.acc_s + nl * 128 + 64 + j8 + 4);
+                        const float4 g0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
+                        const float4 g1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
+                        const float4 u0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8);
+                        const float4 u1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + 64 + j8 + 4);
                         uint4 o;
                         o.x = pack_bf16x2(__fdividef(g0.x, 1.f + __expf(-g0.x)) * u0.x, __fdividef(g0.y, 1.f + __expf(-g0.y)) * u0.y);
                         o.y = pack_bf16x2(__fdividef(g0.z, 1.f + __expf(-g0.z)) * u0.z, __fdividef(g0.w, 1.f + __expf(-g0.w)) * u0.w);
@@ -499,13 +482,13 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                         if (nl < n_hi) *reinterpret_cast<uint4*>(p.act_out + packed_act_offset(c0 + nl, feat >> 3, p.n_pad)) = o;
                     }
                 } else if (EPI == EPI_LMHEAD) {
-                    for (int nl = warp - 2; nl < n_hi; nl += 4) {
+                    for (int nl = ew; nl < n_hi; nl += 4) {
                         float best = -INFINITY;
                         int bi = 0x7fffffff;
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             int ff = lane + 32 * i;
-                            float v = pp.acc_s[nl * 128 + ff];
+                            float v = acc_s[nl * 128 + ff];
                             if (row0 + ff < p.n_out && v > best) { best = v; bi = row0 + ff; }
                         }
 #pragma unroll
@@ -526,7 +509,7 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                             for (int i = 0; i < 4; ++i) {
                                 int ff = lane + 32 * i;
                                 if (row0 + ff < p.n_out) {
-                                    float d = pp.acc_s[nl * 128 + ff] - best;
+                                    float d = acc_s[nl * 128 + ff] - best;
                                     float e = exp2f(d * p.inv_temp_log2e);
                                     z += e;
                                     s1 = fmaf(e, d, s1);
@@ -547,13 +530,16 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                         // logit of tree node et's own token under its parent's distribution, if this tile holds it
                         const int pa = __ldg(p.tree_parent + et), tk = __ldg(p.tree_tokens + et);
                         if (pa >= c0 && pa < c0 + n_hi && tk >= row0 && tk < row0 + 128 && tk < p.n_out)
-                            p.cand[et] = pp.acc_s[(pa - c0) * 128 + (tk - row0)];
+                            p.cand[et] = acc_s[(pa - c0) * 128 + (tk - row0)];
                     }
                 }
-                epi_barrier();
+                epi_barrier(group);
             }
-            if (gather && et == 0)
-                for (int c2 = g_first; c2 < g_first + g_n; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
+            if (gather) {
+                epi_barrier_all();       // both groups have seen the flags
+                if (group == 0 && et == 0)
+                    for (int c2 = g_first; c2 < g_first + g_n; ++c2) p.fix_flags[c2] = 0;   // leave the flags clear for the next launch
+            }
         }
         tc_fence_before_sync();
         mbar_arrive(&pp.ctrl->acc_empty[b]);
@@ -565,9 +551,8 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
 __device__ __forceinline__ bool pipe_setup(Pipe& pp, uint8_t* smem_raw, int n_stages, uint32_t stage_bytes, uint32_t tmem_cols,
                                            int n_pad, int32_t* d_status) {
     pp.stages = smem_raw;                                                                   // 1024-byte aligned (checked)
-    pp.acc_s = reinterpret_cast<float*>(pp.stages + (size_t)n_stages * stage_bytes);        // [32][128] fp32
-    pp.landing = reinterpret_cast<uint8_t*>(pp.acc_s) + (size_t)kStagingCols * 128 * 4;     // 16 KB, contents never read
-    pp.ctrl = reinterpret_cast<GemmCtrl*>(pp.landing + kWChunk);
+    pp.acc_s = reinterpret_cast<float*>(pp.stages + (size_t)n_stages * stage_bytes);        // [kEpiGroups][32][128] fp32
+    pp.ctrl = reinterpret_cast<GemmCtrl*>(reinterpret_cast<uint8_t*>(pp.acc_s) + kStagingBytes);
     pp.abort_flag = &pp.ctrl->abort_flag;
     pp.S = n_stages;
     pp.dual = kGemmDualIssue;
@@ -584,9 +569,8 @@ __device__ __forceinline__ bool pipe_setup(Pipe& pp, uint8_t* smem_raw, int n_st
         }
         mbar_init(&ctrl->acc_full[0], kGemmDualIssue ? 2 : 1);
         mbar_init(&ctrl->acc_full[1], kGemmDualIssue ? 2 : 1);
-        mbar_init(&ctrl->acc_empty[0], 128);
-        mbar_init(&ctrl->acc_empty[1], 128);
-        mbar_init(&ctrl->warm, 1);
+        mbar_init(&ctrl->acc_empty[0], 128 * kEpiGroups);
+        mbar_init(&ctrl->acc_empty[1], 128 * kEpiGroups);
         ctrl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -612,13 +596,11 @@ __device__ __forceinline__ void pipe_teardown(const Pipe& pp, uint32_t tmem_cols
     if (threadIdx.x == 0 && pp.ctrl->abort_flag) report(d_status, CATS_ERR_TIMEOUT);
 }
 
-// Register and shared-memory footprint are chosen so that one CTA of the RMSNorm kernel (256 threads, <= 80 registers,
-// no dynamic shared memory) fits on the SM beside a resident CTA of this kernel: 224 x 192 + 256 x 80 registers <= 64 K,
-// and 224.5 KB + 2 x 1 KB reserved + the norm's static 32 B <= 228 KB.  With programmatic dependent launch the CTAs of
-// the projection that FOLLOWS a norm then take the SMs as soon as the previous projection leaves them and fill their
-// weight ring while the norm is still running.
+// Twelve warps: W producer, two MMA issuers, X producer, two groups of four epilogue warps.  Three warps share each of
+// the SM's four register partitions (16 K registers), hence at most 170 registers per thread; all four epilogues fit
+// without spilling.
 #ifndef CATS_GEMM_MAXREG
-#define CATS_GEMM_MAXREG 192
+#define CATS_GEMM_MAXREG 168      // 12 warps: three of them share one of the SM's four 16 K register partitions
 #endif
 template <int EPI>
 __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
@@ -639,7 +621,6 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             if (!is_w) pdl_wait();    // activations come from the previous kernel; weights never do
             int i = 0;
             produce_units(p, r, pp, is_w, pol, i);
-            if (is_w) warm_next_projection(p, pp, cta);
             if (*pp.abort_flag) drain_after_abort(pp, i);
         }
     } else if (warp == 1) {
@@ -654,12 +635,12 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
             int i = 0, seg = 0;
             mma_units(p, r, pp, i, seg, 1);
         }
-    } else if (warp < 6) {
-        // ---------------- epilogue warps ----------------
+    } else {
+        // ---------------- epilogue warps: group 0 = warps 2-5, group 1 = warps 8-11 ----------------
         pdl_wait();
         int seg = 0;
         bool ok = true;
-        epilogue_units<EPI>(p, r, pp, cta, warp, lane, seg, ok);
+        epilogue_units<EPI>(p, r, pp, cta, warp, lane, warp < 6 ? 0 : 1, seg, ok);
     }
     pipe_teardown(pp, p.tmem_cols, p.d_status);
 }
@@ -805,7 +786,6 @@ GemmPlan gemm_plan(const GemmProblem& p) {
 
 namespace {
 constexpr int kMaxSmem = 225 * 1024;   // leaves room for a co-resident RMSNorm CTA (see k_gemm_sk)
-constexpr size_t kStagingBytes = (size_t)kStagingCols * 128 * 4 + kWChunk;   // epilogue staging tile + landing buffer of the warm copies
 
 // Device-side description of one projection.  max_stages: upper bound on the ring depth (a single launch needs no more
 // stages than a CTA has units).  Returns the dynamic shared memory the kernel needs.
@@ -861,19 +841,6 @@ size_t make_gemm_dev(const GemmProblem& p, const GemmPlan& pl, int max_stages, G
     d.cand = p.cand;
     d.d_status = p.d_status;
     d.dbg_skip_publish = g_debug_fault == 1 ? 1 : 0;
-    d.warm_ptr = nullptr;
-    d.warm_chunks = 0;
-    if (p.warm_next != nullptr && p.warm_next->W[0] != nullptr) {
-        const int n_warm = 4;   // 64 KB per CTA, 9.5 MB in all: what lands while the last epilogue runs
-        GemmPlan np = gemm_plan(*p.warm_next);
-        // the per-CTA base differs by CTA: pass the matrix base and let the CTA add its own offset
-        d.warm_ptr = (const uint8_t*)p.warm_next->W[0];
-        d.warm_chunks = (d.n_pad > 64 || np.head_units > 0) ? 0 : n_warm;   // measured: a small gain for T <= 64, a small loss above
-        d.warm_upc = np.units_per_cta;
-        d.warm_n_ku = ((p.warm_next->K + 63) / 64 + kUnitKb - 1) / kUnitKb;
-        d.warm_n_kb = (p.warm_next->K + 63) / 64;
-        d.warm_total_chunks = (long long)gemm_num_tiles(*p.warm_next) * d.warm_n_kb;
-    }
     return (size_t)stages * d.stage_bytes + kStagingBytes + kCtrlBytes;
 }
 }  // namespace

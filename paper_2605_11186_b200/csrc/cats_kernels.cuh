@@ -114,7 +114,6 @@ struct GemmProblem {
     const int32_t* tree_tokens;   //   [T] token of every tree node
     float* cand;           //   [T] out: logits[parent[i]][tokens[i]]
     int32_t* d_status;
-    const GemmProblem* warm_next;   // the projection that follows (only W[0], K, n_out, n_mats, epi are read), or null
 };
 
 struct GemmPlan {
