@@ -33,9 +33,9 @@ UNIT = "tree tokens/s"
 PREFIX = 512
 SWEEP = (16, 32, 64, 128)
 # dram__bytes_read + dram__bytes_write of the four projection launches of a layer at T=64, from the ncu capture of a
-# 2-layer stack summarised under profiles/ (QKV 109.7+3.8, O 42.5+0.0, gate/up 189.2+4.8, down 91.6+3.3 MB), scaled to the
+# 2-layer stack summarised under profiles/ (QKV 101.3+3.2, O 34.1+0.0, gate/up 180.9+6.5, down 91.6+3.2 MB), scaled to the
 # 128 layer launches of a forward; the LM head (not captured) is counted at its packed size.
-NCU_TRAFFIC_PER_LAUNCH = (32 * (113.5e6 + 42.5e6 + 194.0e6 + 94.9e6) + 262.1e6) / 129
+NCU_TRAFFIC_PER_LAUNCH = (32 * (104.5e6 + 34.1e6 + 187.4e6 + 94.8e6) + 262.1e6) / 129
 TARGET_FORWARD_FRAC_OF_8TBS = 0.70
 
 
