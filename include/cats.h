@@ -299,6 +299,50 @@ int cats_verify_forward_host(const cats_forward_args *a, const int32_t *h_parent
                              int32_t *d_parent_stage, int32_t *d_tokens_stage, int32_t *h_scalars,
                              int32_t *h_out_tokens, int32_t *h_path, void *stream);
 
+/* ---- Tensor-parallel verification over R GPUs -------------------------------
+ * (The paper runs on an 8-GPU server, Section 4 "Experimental setup", but gives
+ * no mechanism; this split is this library's.)  Rank r holds the attention
+ * heads [r*nh/R, (r+1)*nh/R) -- the matching rows of Wq, Wk, Wv, columns of Wo
+ * and its own slice [max_seq][nh/R*hd] of every layer's K/V cache -- and the
+ * MLP rows [r*F/R, (r+1)*F/R) of W_gate, W_up (columns of W_down); norm gains
+ * and the residual stream are replicated.  A layer is two calls per rank, each
+ * leaving this rank's CONTRIBUTION to the residual stream as one [T][hidden]
+ * fp32 tensor that the caller sums over the ranks (one all-reduce, e.g. NCCL
+ * over NVLink) and hands to the next call as d_pending, where the norm folds it
+ * into the rank's copy of the residual stream:
+ *
+ *   cats_tp_attention_half: resid += pending (NULL for the first layer);
+ *       norm, QKV + RoPE + KV append, tree attention, O projection of this
+ *       rank's heads -> d_partial_out
+ *   cats_tp_mlp_half:       resid += pending (the all-reduced attention sums);
+ *       norm, gate/up + SwiGLU, down projection of this rank's rows
+ *       -> d_partial_out
+ *
+ * cfg is the SHARD's shape: hidden as in the full model, n_heads = nh/R,
+ * ffn = F/R, vocab = V/R (head_dim 64 or 128, n_heads*head_dim a multiple of
+ * 64, ffn a multiple of 8); w holds the packed shard matrices.  All ranks see
+ * identical residual streams as long as the all-reduce delivers identical sums.
+ *
+ * cats_tp_lm_head_shard: resid += pending (the last layer's all-reduced MLP
+ * sums); final norm; logits of vocabulary rows [vocab_offset, vocab_offset +
+ * cfg->vocab); d_max_out [T] fp32 = this shard's maximum per node, d_argmax_out
+ * [T] = its lowest GLOBAL index; d_logits [T][cfg->vocab] optional.  The caller
+ * gathers (max, index) of all shards as [R][T] arrays; cats_tp_argmax_merge picks
+ * per node the greatest maximum, lowest index on ties (= the argmax of the
+ * unsplit head).  Walk and compaction then run on every rank as usual, the
+ * compaction on the rank's cache slice (row_elems = nh/R*hd). */
+int cats_tp_attention_half(const cats_model_cfg *cfg, const cats_layer_weights *w, float *d_resid, const float *d_pending,
+                           void *d_kcache, void *d_vcache, const uint64_t *d_mask, const int32_t *d_pos, int32_t T,
+                           int32_t prefix_len, float *d_partial_out, void *d_ws, size_t ws_bytes, int32_t *d_status,
+                           void *stream);
+int cats_tp_mlp_half(const cats_model_cfg *cfg, const cats_layer_weights *w, float *d_resid, const float *d_pending, int32_t T,
+                     float *d_partial_out, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
+int cats_tp_lm_head_shard(const cats_model_cfg *cfg, const void *d_final_norm, const void *d_w_lm, float *d_resid,
+                          const float *d_pending, int32_t T, int32_t vocab_offset, float *d_logits, float *d_max_out,
+                          int32_t *d_argmax_out, void *d_ws, size_t ws_bytes, int32_t *d_status, void *stream);
+int cats_tp_argmax_merge(const float *d_max, const int32_t *d_idx, int32_t n_shards, int32_t T, int32_t *d_argmax,
+                         void *stream);
+
 /* Number of kernel launches the last call of this thread issued (for reports). */
 int cats_last_launch_count(void);
 

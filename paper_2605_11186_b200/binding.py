@@ -77,6 +77,11 @@ lib.cats_accept_path_typical.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _i32, C.c
 lib.cats_compact_kv.argtypes = [_vp, _vp, _i32, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.cats_verify_forward.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp]
 lib.cats_verify_forward_host.argtypes = [C.POINTER(ForwardArgs), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.cats_tp_attention_half.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp,
+                                       _vp, C.c_size_t, _vp, _vp]
+lib.cats_tp_mlp_half.argtypes = [C.POINTER(ModelCfg), C.POINTER(LayerWeights), _vp, _vp, _i32, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.cats_tp_lm_head_shard.argtypes = [C.POINTER(ModelCfg), _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.cats_tp_argmax_merge.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
 lib.cats_packed_weight_bytes.restype = C.c_size_t
 lib.cats_packed_weight_bytes.argtypes = [_i32, _i32, _i32, _i32]
 lib.cats_pack_weights.argtypes = [C.POINTER(C.c_void_p), _i32, _i32, _i32, _i32, _vp, _vp]
@@ -293,6 +298,27 @@ def cats_compact_kv(kcache, vcache, n_layers, layer_stride, row_elems, prefix_le
     _check(lib.cats_compact_kv(_ptr(kcache), _ptr(vcache), n_layers, layer_stride, row_elems, prefix_len, _ptr(path),
                                _ptr(path_len), _ptr(new_len), _ptr(src_rows), _ptr(dst_rows), _ptr(status), _stream()),
            "cats_compact_kv")
+
+
+def cats_tp_attention_half(cfg, w: LayerWeights, resid, pending, kcache, vcache, mask, pos, T, prefix_len, partial_out, ws, status):
+    _check(lib.cats_tp_attention_half(C.byref(cfg), C.byref(w), _ptr(resid), _ptr(pending), _ptr(kcache), _ptr(vcache), _ptr(mask),
+                                      _ptr(pos), T, prefix_len, _ptr(partial_out), _ptr(ws), ws.numel(), _ptr(status), _stream()),
+           "cats_tp_attention_half")
+
+
+def cats_tp_mlp_half(cfg, w: LayerWeights, resid, pending, T, partial_out, ws, status):
+    _check(lib.cats_tp_mlp_half(C.byref(cfg), C.byref(w), _ptr(resid), _ptr(pending), T, _ptr(partial_out), _ptr(ws), ws.numel(),
+                                _ptr(status), _stream()), "cats_tp_mlp_half")
+
+
+def cats_tp_lm_head_shard(cfg, final_norm, w_lm, resid, pending, T, vocab_offset, logits, max_out, argmax_out, ws, status):
+    _check(lib.cats_tp_lm_head_shard(C.byref(cfg), _ptr(final_norm), _ptr(w_lm), _ptr(resid), _ptr(pending), T, vocab_offset,
+                                     _ptr(logits), _ptr(max_out), _ptr(argmax_out), _ptr(ws), ws.numel(), _ptr(status), _stream()),
+           "cats_tp_lm_head_shard")
+
+
+def cats_tp_argmax_merge(max_all, idx_all, n_shards, T, argmax):
+    _check(lib.cats_tp_argmax_merge(_ptr(max_all), _ptr(idx_all), n_shards, T, _ptr(argmax), _stream()), "cats_tp_argmax_merge")
 
 
 class VerifyForward:

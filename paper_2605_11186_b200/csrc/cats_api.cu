@@ -96,19 +96,25 @@ inline bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintp
         if (e__ != cudaSuccess) return CATS_ERR_CUDA; \
     } while (0)
 
-// One decoder layer over T rows.  nodes == nullptr: the rows are the T tree nodes.  Else row t is tree node nodes[t] of
-// a tree of T_tree nodes (mask and pos describe that whole tree): its K/V go to cache row P + nodes[t], it is rotated
-// to pos[nodes[t]] and attends under mask row nodes[t]; the other tree rows are read from the cache.  n_pending: split-K partial sums of the previous layer's down projection still
-// to be folded into resid; copy_from: resid starts from this buffer.  Returns the number of partial
-// sums this layer's down projection left pending (>0) or a negative status.
-int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
-               void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               const void* next_w, bool next_is_head, int32_t* d_status, cudaStream_t st,
-               const int32_t* nodes = nullptr, int T_tree = 0) {
-    const int H = c->hidden, D = c->n_heads * c->head_dim, F = c->ffn;
+// Split-K partial sums still to be folded into the residual stream by the next norm: n slices [T][hidden] fp32.
+struct Pending {
+    const float* part;
+    int n;
+    size_t stride;
+};
+
+// First half of a decoder layer over T rows: RMSNorm (folding `pend` into resid), QKV + RoPE + KV append, tree attention,
+// O projection.  nodes == nullptr: the rows are the T tree nodes.  Else row t is tree node nodes[t] of a tree of T_tree
+// nodes (mask and pos describe that whole tree): its K/V go to cache row P + nodes[t], it is rotated to pos[nodes[t]] and
+// attends under mask row nodes[t]; the other tree rows are read from the cache.  copy_from: resid starts from this buffer.
+// Returns the number of partial sums the O projection left in ws.part (> 0) or a negative status.
+int layer_front(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc, void* vc,
+                const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, Pending pend, int32_t* d_status,
+                cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0) {
+    const int H = c->hidden, D = c->n_heads * c->head_dim;
     const int tpad = (T + 15) / 16 * 16;
     if (stage_on(0))
-        CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
+        CATS_CUDA(launch_rmsnorm(resid, copy_from, pend.part, pend.n, pend.stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
                                  nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
@@ -129,6 +135,15 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     go.epi = EPI_PARTIAL; go.T = T; go.K = D; go.n_out = H; go.n_mats = 1; go.W[0] = w->wo; go.X = ws.o;
     go.fix_part = ws.fix_part; go.fix_flags = ws.fix_flags; go.part = ws.part; go.part_stride = ws.part_stride; go.d_status = d_status;
     const int pieces_o = gemm_plan(go).max_pieces;
+    if (stage_on(3)) CATS_CUDA(launch_gemm(go, st));
+    return pieces_o;
+}
+
+// Second half: RMSNorm (folding `pend`, the O projection's sums, into resid), gate/up + SwiGLU, down projection.
+// Returns the number of partial sums the down projection left in ws.part (> 0) or a negative status.
+int layer_back(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, int T, const Workspace& ws, Pending pend,
+               int32_t* d_status, cudaStream_t st) {
+    const int H = c->hidden, F = c->ffn;
     GemmProblem ggu = {};
     ggu.epi = EPI_SWIGLU; ggu.T = T; ggu.K = H; ggu.n_out = F; ggu.n_mats = 2; ggu.W[0] = w->w_gate_up; ggu.X = ws.xn;
     ggu.fix_part = ws.fix_part; ggu.fix_flags = ws.fix_flags; ggu.act_out = ws.act; ggu.d_status = d_status;
@@ -136,13 +151,23 @@ int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
     gd.epi = EPI_PARTIAL; gd.T = T; gd.K = F; gd.n_out = H; gd.n_mats = 1; gd.W[0] = w->w_down; gd.X = ws.act;
     gd.fix_part = ws.fix_part; gd.fix_flags = ws.fix_flags; gd.part = ws.part; gd.part_stride = ws.part_stride; gd.d_status = d_status;
     const int pieces_d = gemm_plan(gd).max_pieces;
-    if (stage_on(3)) CATS_CUDA(launch_gemm(go, st));
     if (stage_on(4))
-        CATS_CUDA(launch_rmsnorm(resid, nullptr, ws.part, pieces_o, ws.part_stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
+        CATS_CUDA(launch_rmsnorm(resid, nullptr, pend.part, pend.n, pend.stride, w->mlp_norm, T, H, c->rms_eps, ws.xn, nullptr,
                                  nullptr, nullptr, c->head_dim, c->rope_base, nullptr, 0, st, d_status));
     if (stage_on(5)) CATS_CUDA(launch_gemm(ggu, st));
     if (stage_on(6)) CATS_CUDA(launch_gemm(gd, st));
     return pieces_d;
+}
+
+// One whole decoder layer.  n_pending: split-K partial sums of the previous layer's down projection still to be folded
+// into resid.  Returns the number of partial sums this layer's down projection left pending (> 0) or a negative status.
+int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
+               void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
+               int32_t* d_status, cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0) {
+    const int pieces_o = layer_front(c, w, resid, copy_from, kc, vc, mask, pos, T, P, ws, Pending{ws.part, n_pending, ws.part_stride},
+                                     d_status, st, nodes, T_tree);
+    if (pieces_o < 0) return pieces_o;
+    return layer_back(c, w, resid, T, ws, Pending{ws.part, pieces_o, ws.part_stride}, d_status, st);
 }
 
 // Typical acceptance: what the LM head must leave behind besides the argmax.
@@ -152,11 +177,12 @@ struct TypicalOut {
     float *lse, *entropy, *cand;      // [T] each
 };
 
+// vmax_out / idx_offset: a vocabulary shard also leaves every node's maximum and adds its first row to the indices.
 int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm, float* resid, const float* copy_from,
-              int T, int n_pending, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st,
-              const TypicalOut* ty = nullptr) {
+              int T, Pending pend, float* logits, int32_t* amax, const Workspace& ws, int32_t* d_status, cudaStream_t st,
+              const TypicalOut* ty = nullptr, float* vmax_out = nullptr, int idx_offset = 0) {
     const int H = c->hidden, V = c->vocab;
-    CATS_CUDA(launch_rmsnorm(resid, copy_from, ws.part, n_pending, ws.part_stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
+    CATS_CUDA(launch_rmsnorm(resid, copy_from, pend.part, pend.n, pend.stride, final_norm, T, H, c->rms_eps, ws.xn, nullptr,
                              nullptr, nullptr, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
     GemmProblem g = {};
     g.epi = EPI_LMHEAD; g.T = T; g.K = H; g.n_out = V; g.n_mats = 1; g.W[0] = w_lm; g.X = ws.xn;
@@ -171,7 +197,7 @@ int head_impl(const cats_model_cfg* c, const void* final_norm, const void* w_lm,
         CATS_CUDA(launch_head_reduce(ws.pmax, ws.pidx, ws.psum, ws.ps1, (V + 127) / 128, 128, T, ty->inv_temperature, amax,
                                      ty->lse, ty->entropy, st));
     else
-        CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, st));
+        CATS_CUDA(launch_argmax_reduce(ws.pmax, ws.pidx, (V + 127) / 128, 128, T, amax, vmax_out, idx_offset, st));
     return CATS_OK;
 }
 
@@ -301,8 +327,7 @@ int cats_verify_layer(const cats_model_cfg* cfg, const cats_layer_weights* w, fl
     Workspace ws = carve(cfg, T, d_ws);
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, nullptr,
-                             false, d_status, st);
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws, 0, d_status, st);
     if (pending < 0) return pending;
     if (stage_on(6))
         CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, T, cfg->hidden, cfg->rms_eps, nullptr,
@@ -331,8 +356,8 @@ int cats_verify_layer_nodes(const cats_model_cfg* cfg, const cats_layer_weights*
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     CATS_CUDA(launch_check_nodes(d_nodes, m, T, ws.nodes, d_status, st));
-    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, m, prefix_len, ws, 0, nullptr,
-                             false, d_status, st, ws.nodes, T);
+    int pending = layer_impl(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, m, prefix_len, ws, 0, d_status, st,
+                             ws.nodes, T);
     if (pending < 0) return pending;
     CATS_CUDA(launch_rmsnorm(d_resid, nullptr, ws.part, pending, ws.part_stride, nullptr, m, cfg->hidden, cfg->rms_eps, nullptr,
                              nullptr, nullptr, nullptr, cfg->head_dim, cfg->rope_base, nullptr, 0, st, d_status));
@@ -380,7 +405,8 @@ int cats_lm_head_argmax(const cats_model_cfg* cfg, const void* d_final_norm, con
     Workspace ws = carve(cfg, T, d_ws);
     if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
     // the caller's residual is read-only here: normalise a copy held in the scratch area
-    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, 0, d_logits, d_argmax, ws, d_status, (cudaStream_t)stream);
+    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, Pending{nullptr, 0, 0}, d_logits, d_argmax, ws, d_status,
+                     (cudaStream_t)stream);
 }
 
 int cats_lm_head_typical(const cats_model_cfg* cfg, const void* d_final_norm, const void* d_w_lm, const float* d_resid,
@@ -404,7 +430,7 @@ int cats_lm_head_typical(const cats_model_cfg* cfg, const void* d_final_norm, co
     CATS_CUDA(cudaMemsetAsync(d_cand_logit, 0, (size_t)T * sizeof(float), st));
     g_call_boundary = true;   // the memset is not a kernel: the first kernel still takes full stream ordering
     TypicalOut ty = {d_parent, d_tokens, inv_temperature, d_lse, d_entropy, d_cand_logit};
-    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, 0, d_logits, d_argmax, ws, d_status, st, &ty);
+    return head_impl(cfg, d_final_norm, d_w_lm, ws.scratch, d_resid, T, Pending{nullptr, 0, 0}, d_logits, d_argmax, ws, d_status, st, &ty);
 }
 
 int cats_accept_path_typical(const int32_t* d_parent, const int32_t* d_tokens, const int32_t* d_argmax, const float* d_cand_logit,
@@ -449,6 +475,87 @@ int cats_compact_kv(void* d_kcache, void* d_vcache, int32_t n_layers, int64_t la
     return CATS_OK;
 }
 
+/* ---- tensor-parallel halves (see cats.h) ---- */
+static int tp_common_checks(const cats_model_cfg* cfg, const float* d_resid, int32_t T, void* d_ws, int32_t* d_status) {
+    int rc = check_cfg(cfg);
+    if (rc) return rc;
+    if (!d_resid || !d_ws || !d_status) return CATS_ERR_INVALID_ARG;
+    if (T < 1 || T > CATS_MAX_TREE) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_ws, 1024)) return CATS_ERR_WORKSPACE;
+    if (misaligned(d_resid, 16)) return CATS_ERR_INVALID_ARG;
+    return CATS_OK;
+}
+
+int cats_tp_attention_half(const cats_model_cfg* cfg, const cats_layer_weights* w, float* d_resid, const float* d_pending,
+                           void* d_kcache, void* d_vcache, const uint64_t* d_mask, const int32_t* d_pos, int32_t T,
+                           int32_t prefix_len, float* d_partial_out, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    NvtxRange nvtx_range("cats_tp_attention_half");
+    g_call_boundary = true;
+    int rc = tp_common_checks(cfg, d_resid, T, d_ws, d_status);
+    if (rc) return rc;
+    if (!w || !w->attn_norm || !w->wqkv || !w->wo || !d_kcache || !d_vcache || !d_mask || !d_pos || !d_partial_out)
+        return CATS_ERR_INVALID_ARG;
+    if (prefix_len < 0 || prefix_len + T > cfg->max_seq) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_partial_out, 16) || misaligned(d_pending, 16) || misaligned(d_kcache, 16) || misaligned(d_vcache, 16))
+        return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = (size_t)T * cfg->hidden;
+    const int pieces = layer_front(cfg, w, d_resid, nullptr, d_kcache, d_vcache, d_mask, d_pos, T, prefix_len, ws,
+                                   Pending{d_pending, d_pending ? 1 : 0, n}, d_status, st);
+    if (pieces < 0) return pieces;
+    CATS_CUDA(launch_sum_parts(ws.part, pieces, ws.part_stride, n, d_partial_out, st));
+    return CATS_OK;
+}
+
+int cats_tp_mlp_half(const cats_model_cfg* cfg, const cats_layer_weights* w, float* d_resid, const float* d_pending, int32_t T,
+                     float* d_partial_out, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    NvtxRange nvtx_range("cats_tp_mlp_half");
+    g_call_boundary = true;
+    int rc = tp_common_checks(cfg, d_resid, T, d_ws, d_status);
+    if (rc) return rc;
+    if (!w || !w->mlp_norm || !w->w_gate_up || !w->w_down || !d_pending || !d_partial_out) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_partial_out, 16) || misaligned(d_pending, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = (size_t)T * cfg->hidden;
+    // the stream-K fix-up flags of the gate/up projection must start at zero; the first half of the layer left them so
+    const int pieces = layer_back(cfg, w, d_resid, T, ws, Pending{d_pending, 1, n}, d_status, st);
+    if (pieces < 0) return pieces;
+    CATS_CUDA(launch_sum_parts(ws.part, pieces, ws.part_stride, n, d_partial_out, st));
+    return CATS_OK;
+}
+
+int cats_tp_lm_head_shard(const cats_model_cfg* cfg, const void* d_final_norm, const void* d_w_lm, float* d_resid,
+                          const float* d_pending, int32_t T, int32_t vocab_offset, float* d_logits, float* d_max_out,
+                          int32_t* d_argmax_out, void* d_ws, size_t ws_bytes, int32_t* d_status, void* stream) {
+    g_launch_count = 0;
+    NvtxRange nvtx_range("cats_tp_lm_head_shard");
+    g_call_boundary = true;
+    int rc = tp_common_checks(cfg, d_resid, T, d_ws, d_status);
+    if (rc) return rc;
+    if (!d_final_norm || !d_w_lm || !d_max_out || !d_argmax_out || cfg->vocab < 1 || vocab_offset < 0) return CATS_ERR_INVALID_ARG;
+    if (misaligned(d_pending, 16) || misaligned(d_w_lm, 16) || misaligned(d_final_norm, 16)) return CATS_ERR_INVALID_ARG;
+    Workspace ws = carve(cfg, T, d_ws);
+    if (ws.bytes > ws_bytes) return CATS_ERR_WORKSPACE;
+    const size_t n = (size_t)T * cfg->hidden;
+    return head_impl(cfg, d_final_norm, d_w_lm, d_resid, nullptr, T, Pending{d_pending, d_pending ? 1 : 0, n}, d_logits, d_argmax_out,
+                     ws, d_status, (cudaStream_t)stream, nullptr, d_max_out, vocab_offset);
+}
+
+int cats_tp_argmax_merge(const float* d_max, const int32_t* d_idx, int32_t n_shards, int32_t T, int32_t* d_argmax, void* stream) {
+    g_launch_count = 0;
+    NvtxRange nvtx_range("cats_tp_argmax_merge");
+    g_call_boundary = true;
+    if (!d_max || !d_idx || !d_argmax || n_shards < 1 || T < 1 || T > CATS_MAX_TREE) return CATS_ERR_INVALID_ARG;
+    CATS_CUDA(launch_argmax_reduce(d_max, d_idx, n_shards, T, T, d_argmax, nullptr, 0, (cudaStream_t)stream));
+    return CATS_OK;
+}
+
 int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, const int32_t* d_tokens, void* stream) {
     g_launch_count = 0;
     NvtxRange nvtx_range("cats_verify_forward");
@@ -481,16 +588,14 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     if (!copy_from) CATS_CUDA(launch_embed(a->d_embed, d_tokens, T, c->hidden, c->vocab, a->d_resid, a->d_status, st));
     int pending = 0;
     for (int l = 0; l < c->n_layers; ++l) {
-        const bool last = (l + 1 == c->n_layers);
-        const void* next_w = last ? a->d_w_lm : a->layers[l + 1].wqkv;
         pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
-                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, next_w,
-                             last, a->d_status, st);
+                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, a->d_status, st);
         if (pending < 0) return pending;
     }
     TypicalOut ty = {d_parent, d_tokens, a->inv_temperature, a->d_typical, a->d_typical ? a->d_typical + T : nullptr,
                      a->d_typical ? a->d_typical + 2 * T : nullptr};
-    rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T, pending, a->d_logits,
+    rc = head_impl(c, a->d_final_norm, a->d_w_lm, a->d_resid, c->n_layers == 0 ? copy_from : nullptr, T,
+                   Pending{ws.part, pending, ws.part_stride}, a->d_logits,
                    a->d_argmax, ws, a->d_status, st, typical ? &ty : nullptr);
     if (rc) return rc;
     if (typical)

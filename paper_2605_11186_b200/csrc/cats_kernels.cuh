@@ -52,7 +52,9 @@ cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* pa
 // Checks a partial-tree node list (strictly ascending, inside [0, T)) and writes a copy clamped into range.
 cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
-                                 cudaStream_t st);
+                                 float* vmax, int idx_offset, cudaStream_t st);
+// out[i] = sum over the n_part slices part[s * part_stride + i], i < n (n and part_stride multiples of 4).
+cudaError_t launch_sum_parts(const float* part, int n_part, size_t part_stride, size_t n, float* out, cudaStream_t st);
 // The same reduction plus the merge of the per-tile softmax statistics: lse[n] = log sum_v exp(logit/t),
 // entropy[n] = H(softmax(logit/t)).
 cudaError_t launch_head_reduce(const float* pmax, const int32_t* pidx, const float* psum, const float* ps1, int n_tiles,

@@ -176,8 +176,11 @@ __global__ void __launch_bounds__(128) k_check_nodes(const int32_t* __restrict__
 // tile's maximum and the lowest index attaining it; one warp per node picks the overall winner
 // (lowest index among equal maxima).
 // ---------------------------------------------------------------------------------------------
+// vmax (optional) receives the maximum itself, idx_offset is added to the winning index (a vocabulary shard reports global
+// indices); the same kernel merges the shards' results, one "tile" per shard.
 __global__ void __launch_bounds__(128) k_argmax_reduce(const float* __restrict__ pmax, const int32_t* __restrict__ pidx,
-                                                       int n_tiles, int t_stride, int T, int32_t* __restrict__ amax) {
+                                                       int n_tiles, int t_stride, int T, int32_t* __restrict__ amax,
+                                                       float* __restrict__ vmax, int idx_offset) {
     pdl_launch_dependents();
     pdl_wait();
     int t = blockIdx.x * 4 + (threadIdx.x >> 5);
@@ -196,7 +199,26 @@ __global__ void __launch_bounds__(128) k_argmax_reduce(const float* __restrict__
         int oi = __shfl_xor_sync(0xffffffffu, bi, o);
         if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
     }
-    if (lane == 0) amax[t] = bi;
+    if (lane == 0) {
+        amax[t] = bi + idx_offset;
+        if (vmax != nullptr) vmax[t] = best;
+    }
+}
+
+// out[i] = part[0][i] + part[1][i] + ... (slot order): the split-K partial sums of a projection as ONE [T][hidden] fp32
+// tensor, for a caller that reduces it across GPUs before the next norm folds it into the residual stream.
+__global__ void __launch_bounds__(256) k_sum_parts(const float4* __restrict__ part, int n_part, size_t stride4, size_t n4,
+                                                   float4* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 a = __ldcg(part + i);
+        for (int s = 1; s < n_part; ++s) {
+            const float4 q = __ldcg(part + (size_t)s * stride4 + i);
+            a.x += q.x; a.y += q.y; a.z += q.z; a.w += q.w;
+        }
+        out[i] = a;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -625,8 +647,16 @@ cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clam
 }
 
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
-                                 cudaStream_t st) {
-    return launch_pdl(k_argmax_reduce, dim3((T + 3) / 4), dim3(128), 0, st, pmax, pidx, n_tiles, t_stride, T, amax);
+                                 float* vmax, int idx_offset, cudaStream_t st) {
+    return launch_pdl(k_argmax_reduce, dim3((T + 3) / 4), dim3(128), 0, st, pmax, pidx, n_tiles, t_stride, T, amax, vmax, idx_offset);
+}
+
+cudaError_t launch_sum_parts(const float* part, int n_part, size_t part_stride, size_t n, float* out, cudaStream_t st) {
+    const size_t n4 = n / 4;
+    int blocks = (int)((n4 + 255) / 256);
+    if (blocks > 148 * 4) blocks = 148 * 4;
+    if (blocks < 1) blocks = 1;
+    return launch_pdl(k_sum_parts, dim3(blocks), dim3(256), 0, st, (const float4*)part, n_part, part_stride / 4, n4, (float4*)out);
 }
 
 cudaError_t launch_head_reduce(const float* pmax, const int32_t* pidx, const float* psum, const float* ps1, int n_tiles,
