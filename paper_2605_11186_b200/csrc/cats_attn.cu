@@ -570,10 +570,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     // Every barrier that a thread may find more than one phase ahead of itself would give a wrong answer to a parity
     // wait, so each one is either indexed by block parity (its next completion needs the waiter's own progress) or by
     // ring stage (the classical full / empty pair).
-    uint64_t* bar_s = rbar + 1;           // [2]  S(b) complete, by block parity
-    uint64_t* bar_o = rbar + 3;           // [2]  P(b) V(b) complete, by block parity
-    uint64_t* bar_p = rbar + 5;           // [2]  P(b) written (256 arrivals), by block parity
-    uint64_t* bar_kv = rbar + 7;          // [kTcMaxStages]  block landed in the stage (bytes counted)
+    // Streamed shares keep FOUR score / probability buffers in tensor memory (one-block shares use one): the loop
+    // S(b) -> softmax -> P(b) V(b) -> buffer free again is a chain of three hand-offs of several hundred nanoseconds each,
+    // and with two buffers that chain, not any unit's throughput, set the pace (halving the MMAs, the TMA issues or the
+    // softmax work per thread each changed next to nothing).
+    constexpr int NSB = STREAM ? 4 : 2;
+    uint64_t* bar_s = rbar + 1;           // [4]  S(b) complete, by buffer (b mod NSB)
+    uint64_t* bar_o = rbar + 5;           // [4]  P(b) V(b) complete, by buffer
+    uint64_t* bar_p = rbar + 9;           // [4]  P(b) written (256 arrivals), by buffer
+    uint64_t* bar_kv = rbar + 13;         // [kTcMaxStages]  block landed in the stage (bytes counted)
     uint64_t* bar_free = bar_kv + kTcMaxStages;  // [kTcMaxStages]  the P V product that read the stage has completed
     uint64_t* bar_q = bar_free + kTcMaxStages;   //      Q landed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_q + 1);
@@ -615,12 +620,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         tmem_relinquish();
         if (lane == 0) {
             *wait_expired = 0;
-            mbar_init(bar_s, 1);
-            mbar_init(bar_s + 1, 1);
-            mbar_init(bar_o, 1);
-            mbar_init(bar_o + 1, 1);
-            mbar_init(bar_p, 256);
-            mbar_init(bar_p + 1, 256);
+            for (int i = 0; i < NSB; ++i) {
+                mbar_init(bar_s + i, 1);
+                mbar_init(bar_o + i, 1);
+                mbar_init(bar_p + i, 256);
+            }
             mbar_fence_init();
         }
     }
@@ -644,27 +648,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_wait();
     const uint32_t tbase = *tmem_slot;
+    // tensor-memory columns.  One-block share: S / P [0,192), O [384,512).  Streamed: S / P buffers [64 k, 64 k + 64), k < 4.
     const uint32_t tO = tbase + 384;
+    auto sbuf = [&](int b) { return STREAM ? (b & 3) : (b & 1); };              // buffer of block b
+    auto sphase = [&](int b) { return (uint32_t)(STREAM ? (b >> 2) : (b >> 1)) & 1u; };   // and the phase of its barriers
+    auto s_addr = [&](int b) { return tbase + (uint32_t)(STREAM ? (b & 3) * 64 : (b & 1) * kTcSStride); };
     const uint32_t q_u32 = smem_u32(q_s);
 
     // O += P(b) V(b), issued as soon as the softmax warps have written P(b)
     auto issue_pv = [&](int b) -> bool {
         const uint32_t idv = umma_idesc_bf16_m128_bmn(HD);
         if (!(mbar_wait(bar_kv + b % NST, (uint32_t)(b / NST) & 1u, wait_expired) &&      // V(b) (long since landed)
-              mbar_wait(bar_p + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired)))
+              mbar_wait(bar_p + sbuf(b), sphase(b), wait_expired)))
             return false;
         tc_fence_after_sync();
         const int r0 = c_begin + b * NB;
         const int n16 = min(NB, (c_end - r0 + 15) & ~15);
         const uint32_t vs_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes) + (uint32_t)NB * 256u;
-        const uint32_t tP = tbase + (uint32_t)(b & 1) * kTcSStride;
+        const uint32_t tP = s_addr(b);
         const uint64_t dv0 = umma_desc_sw128_mn(vs_u32, half);
         const int nk = n16 / 16;
         for (int kk = 0; kk < nk; ++kk)
             umma_bf16_ts(tO, tP + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, b > 0 || kk > 0);
         for (int kk = 0; kk < nk; ++kk)
             umma_bf16_ts(tO, tP + (uint32_t)(NB / 2) + (uint32_t)kk * 8u, dv0 + (uint64_t)(kk * (2048 >> 4)), idv, true);
-        umma_commit(bar_o + (b & 1));
+        umma_commit(bar_o + sbuf(b));
         umma_commit(bar_free + b % NST);
         return true;
     };
@@ -676,13 +684,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             bool ok = mbar_wait(bar_q, 0, wait_expired);
             for (int b = 0; b < nb && ok; ++b) {
                 ok = mbar_wait(bar_kv + b % NST, (uint32_t)(b / NST) & 1u, wait_expired);
-                if (ok && b >= 2) ok = mbar_wait(bar_o + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
+                if (ok && b >= NSB) ok = mbar_wait(bar_o + sbuf(b), sphase(b - NSB), wait_expired);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
                 const int n16 = min(NB, (c_end - r0 + 15) & ~15);
                 const uint32_t ks_u32 = smem_u32(kv_s + (size_t)(b % NST) * stage_bytes);
-                const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
+                const uint32_t tS = s_addr(b);
                 const uint32_t idesc = umma_idesc_bf16_m128(n16);
                 const uint64_t da0 = umma_desc_sw128(q_u32), db0 = umma_desc_sw128(ks_u32);      // the address field takes plain additions
 #pragma unroll
@@ -691,7 +699,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                     const uint64_t db = db0 + (uint64_t)(((uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u) >> 4);
                     umma_bf16(tS, da, db, idesc, ks > 0);
                 }
-                umma_commit(bar_s + (b & 1));
+                umma_commit(bar_s + sbuf(b));
             }
             if (!STREAM && ok) issue_pv(0);      // one-block share: the same thread issues P V as well
         }
@@ -732,10 +740,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         bool ok = true;
         for (int b = 0; b < nb; ++b) {
             const int r0 = c_begin + b * NB;
-            const uint32_t tS = tbase + (uint32_t)(b & 1) * kTcSStride;
+            const uint32_t tS = s_addr(b);
             float v[CPT];
             float corr = 1.f, ref = 0.f;
-            if (ok) ok = mbar_wait(bar_s + (b & 1), (uint32_t)(b >> 1) & 1u, wait_expired);
+            if (ok) ok = mbar_wait(bar_s + sbuf(b), sphase(b), wait_expired);
             tc_fence_after_sync();
             if (act) {
 #pragma unroll
@@ -785,7 +793,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             }
             if (STREAM && b > 0 && act && __any_sync(0xffffffffu, corr != 1.f)) {
                 // O follows the reference; P(b-1) V(b-1) must have completed first
-                if (ok) ok = mbar_wait(bar_o + ((b - 1) & 1), (uint32_t)((b - 1) >> 1) & 1u, wait_expired);
+                if (ok) ok = mbar_wait(bar_o + sbuf(b - 1), sphase(b - 1), wait_expired);
                 tc_fence_after_sync();
                 {
 #pragma unroll
@@ -824,16 +832,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 tmem_wait_st();
             }
             tc_fence_before_sync();
-            // Two hand-off barriers alternate by block, each counting one arrival per thread and block: no arrival for
-            // block b before every thread has arrived for block b - 2 (which holds anyway: S(b) is issued only after
-            // P(b - 2) V(b - 2) has completed).
-            if (STREAM && b > 1 && ok) ok = mbar_wait(bar_p + (b & 1), (uint32_t)((b - 2) >> 1) & 1u, wait_expired);
-            mbar_arrive(bar_p + (b & 1));
+            // One hand-off barrier per buffer, counting one arrival per thread and block: no arrival for block b can come
+            // before every thread has arrived for the buffer's previous block (S(b) is issued only after that block's
+            // P V has completed, which needed all of its P).
+            mbar_arrive(bar_p + sbuf(b));
         }
         // ---- this thread's half of the row's O, and the row's (m, l), go straight into the shared memory of the CTA
         //      that merges the row: stores through distributed shared memory, made visible by the cluster barrier ----
         if (nb > 0) {
-            if (ok) ok = mbar_wait(bar_o + ((nb - 1) & 1), (uint32_t)((nb - 1) >> 1) & 1u, wait_expired);
+            if (ok) ok = mbar_wait(bar_o + sbuf(nb - 1), sphase(nb - 1), wait_expired);
             tc_fence_after_sync();
         }
         if (p.csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA of the cluster has started
