@@ -110,12 +110,14 @@ struct Pending {
 // Returns the number of partial sums the O projection left in ws.part (> 0) or a negative status.
 int layer_front(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc, void* vc,
                 const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, Pending pend, int32_t* d_status,
-                cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0) {
+                cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0, bool rope_ready = false) {
     const int H = c->hidden, D = c->n_heads * c->head_dim;
     const int tpad = (T + 15) / 16 * 16;
+    // rope_ready: an earlier layer of the same call has already left the rotary table of these rows in the workspace
     if (stage_on(0))
         CATS_CUDA(launch_rmsnorm(resid, copy_from, pend.part, pend.n, pend.stride, w->attn_norm, T, H, c->rms_eps, ws.xn, pos,
-                                 nodes, ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st, d_status));
+                                 nodes, rope_ready ? nullptr : ws.rope, c->head_dim, c->rope_base, ws.fix_flags, kFixSlots, st,
+                                 d_status));
     GemmProblem g = {};
     g.epi = EPI_QKV; g.T = T; g.K = H; g.n_out = D; g.n_mats = 3;
     g.W[0] = w->wqkv; g.X = ws.xn; g.fix_part = ws.fix_part; g.fix_flags = ws.fix_flags;
@@ -163,9 +165,9 @@ int layer_back(const cats_model_cfg* c, const cats_layer_weights* w, float* resi
 // into resid.  Returns the number of partial sums this layer's down projection left pending (> 0) or a negative status.
 int layer_impl(const cats_model_cfg* c, const cats_layer_weights* w, float* resid, const float* copy_from, void* kc,
                void* vc, const uint64_t* mask, const int32_t* pos, int T, int P, const Workspace& ws, int n_pending,
-               int32_t* d_status, cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0) {
+               int32_t* d_status, cudaStream_t st, const int32_t* nodes = nullptr, int T_tree = 0, bool rope_ready = false) {
     const int pieces_o = layer_front(c, w, resid, copy_from, kc, vc, mask, pos, T, P, ws, Pending{ws.part, n_pending, ws.part_stride},
-                                     d_status, st, nodes, T_tree);
+                                     d_status, st, nodes, T_tree, rope_ready);
     if (pieces_o < 0) return pieces_o;
     return layer_back(c, w, resid, T, ws, Pending{ws.part, pieces_o, ws.part_stride}, d_status, st);
 }
@@ -589,7 +591,8 @@ int cats_verify_forward(const cats_forward_args* a, const int32_t* d_parent, con
     int pending = 0;
     for (int l = 0; l < c->n_layers; ++l) {
         pending = layer_impl(c, &a->layers[l], a->d_resid, l == 0 ? copy_from : nullptr, (uint16_t*)a->d_kcache + l * lstride,
-                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, a->d_status, st);
+                             (uint16_t*)a->d_vcache + l * lstride, a->d_mask, a->d_pos, T, P, ws, pending, a->d_status, st,
+                             nullptr, 0, /*rope_ready=*/l > 0 && stage_on(0));
         if (pending < 0) return pending;
     }
     TypicalOut ty = {d_parent, d_tokens, a->inv_temperature, a->d_typical, a->d_typical ? a->d_typical + T : nullptr,

@@ -332,14 +332,34 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                 }
             }
         }
+        int mat = 0, row0;
+        if (EPI == EPI_SWIGLU) row0 = tile * 64;
+        else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
+        // EPI_QKV: a thread rotates 4 feature pairs (lo, lo + head_dim / 2) of every eighth node, so it needs the 4
+        // (cos, sin) of each of its nodes once.  Those of the group's first staging round are fetched here, while the
+        // accumulator is still being summed: their trip from L2 otherwise sits between the last MMA and the stores
+        // (1.5 us per q/k tile, measured).
+        constexpr int kRopeNodes = kStagingCols / 8;       // nodes per thread and staging round
+        const int rope_half = p.head_dim >> 1;
+        const int rope_pj = (et & 15) * 4;                  // first of the thread's 4 pairs among the tile's 64
+        const int rope_hin = EPI == EPI_QKV ? rope_pj / rope_half : 0;          // head inside the tile
+        const int rope_ri = rope_pj - rope_hin * rope_half;                     // rotary index of the first pair
+        float4 cs0[kRopeNodes][2];
+        if (EPI == EPI_QKV && ok && head && mat < 2) {
+            const int n_hi0 = min(kStagingCols, p.T - c_first);
+#pragma unroll
+            for (int it = 0; it < kRopeNodes; ++it) {
+                const int nl = (et >> 4) + 8 * it;
+                const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c_first + nl) * rope_half + rope_ri);
+                cs0[it][0] = nl < n_hi0 ? __ldg(src) : make_float4(1.f, 0.f, 1.f, 0.f);
+                cs0[it][1] = nl < n_hi0 ? __ldg(src + 1) : make_float4(1.f, 0.f, 1.f, 0.f);
+            }
+        }
         if (ok) ok = mbar_wait(&pp.ctrl->acc_full[b], (seg >> 1) & 1, pp.abort_flag);
         ok = ok && !*pp.abort_flag;
         tc_fence_after_sync();
         const uint32_t taddr = pp.tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * pp.acc_stride);
         const uint32_t dual = pp.dual ? (uint32_t)p.n_pad : 0u;
-        int mat = 0, row0;
-        if (EPI == EPI_SWIGLU) row0 = tile * 64;
-        else { mat = tile / p.tiles_per_mat; row0 = (tile - mat * p.tiles_per_mat) * 128; }
 
         if (!ok) {
             // nothing: fall through to the arrive below so that nobody waits on this accumulator
@@ -357,9 +377,11 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
         } else if (!head) {
             // a later piece of a tile another CTA owns: publish the raw fp32 partial tile
             store_tile_transposed(taddr, dual, p.n_pad, p.n_pad, acc_s, f, et, group, p.fix_part + (size_t)my_slot * p.n_pad * 128, 128, 128);
-            __threadfence();
-            epi_barrier_all();       // both groups have stored and fenced their rounds
-            if (group == 0 && et == 0 && !p.dbg_skip_publish) st_release(p.fix_flags + my_slot, 1);
+            epi_barrier_all();       // both groups have stored their rounds; the barrier orders those stores before the release below
+            if (group == 0 && et == 0 && !p.dbg_skip_publish) {
+                __threadfence();
+                st_release(p.fix_flags + my_slot, 1);
+            }
         } else {
             // this CTA owns the tile: add the other pieces (if any), then the fused epilogue
 #pragma unroll
@@ -397,66 +419,57 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
                 epi_barrier(group);
                 const int n_hi = min(kStagingCols, p.T - c0);   // valid nodes in this staging tile
                 if (EPI == EPI_QKV) {
-                    // thread -> 8 consecutive features (one 16-byte store per node), every eighth node.  All loads of
-                    // the thread are issued before the first store, so their latencies overlap.
-                    const int j8 = (et & 15) * 8;
-                    const int feat = row0 + j8;
-                    const int hd = p.head_dim, half = hd >> 1;
-                    const int in_head = feat % hd;
-                    const bool first_half = in_head < half;
-                    const int partner = first_half ? j8 + half : j8 - half;
-                    const int ri = in_head % half;
-                    const float sgn = first_half ? -1.f : 1.f;
-                    constexpr int NI = kStagingCols / 8;
-                    if (feat < p.n_out) {
-                        uint4 packed[NI];
+                    // thread -> 4 rotary pairs: features [lo, lo + 4) and [lo + half, lo + half + 4) of every eighth node,
+                    // two 8-byte stores per node.  All loads of the thread are issued before the first store.
+                    const int lo = rope_hin * p.head_dim + rope_ri, hi = lo + rope_half;
+                    constexpr int NI = kRopeNodes;
+                    if (row0 + hi < p.n_out) {
+                        uint2 plo[NI], phi[NI];
                         if (mat < 2) {
-                            float4 cs[NI][4];     // (cos, sin) of the 8 feature pairs
+                            float4 cs[NI][2];     // (cos, sin) of the 4 pairs
 #pragma unroll
                             for (int it = 0; it < NI; ++it) {
                                 const int nl = (et >> 4) + 8 * it;
-                                const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * half + ri);
+                                const float4* src = reinterpret_cast<const float4*>(p.rope + (size_t)(c0 + nl) * rope_half + rope_ri);
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) cs[it][q] = nl < n_hi ? __ldg(src + q) : make_float4(1.f, 0.f, 1.f, 0.f);
+                                for (int q = 0; q < 2; ++q) {
+                                    if (qi == 0) cs[it][q] = cs0[it][q];       // fetched before the accumulator wait
+                                    else cs[it][q] = nl < n_hi ? __ldg(src + q) : make_float4(1.f, 0.f, 1.f, 0.f);
+                                }
                             }
 #pragma unroll
                             for (int it = 0; it < NI; ++it) {
                                 const int nl = (et >> 4) + 8 * it;
-                                const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
-                                const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
-                                const float4 y0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner);
-                                const float4 y1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + partner + 4);
-                                packed[it].x = pack_bf16x2(x0.x * cs[it][0].x + sgn * y0.x * cs[it][0].y, x0.y * cs[it][0].z + sgn * y0.y * cs[it][0].w);
-                                packed[it].y = pack_bf16x2(x0.z * cs[it][1].x + sgn * y0.z * cs[it][1].y, x0.w * cs[it][1].z + sgn * y0.w * cs[it][1].w);
-                                packed[it].z = pack_bf16x2(x1.x * cs[it][2].x + sgn * y1.x * cs[it][2].y, x1.y * cs[it][2].z + sgn * y1.y * cs[it][2].w);
-                                packed[it].w = pack_bf16x2(x1.z * cs[it][3].x + sgn * y1.z * cs[it][3].y, x1.w * cs[it][3].z + sgn * y1.w * cs[it][3].w);
+                                const float4 x = *reinterpret_cast<const float4*>(acc_s + nl * 128 + lo);
+                                const float4 y = *reinterpret_cast<const float4*>(acc_s + nl * 128 + hi);
+                                const float4 c0s = cs[it][0], c1s = cs[it][1];
+                                plo[it].x = pack_bf16x2(x.x * c0s.x - y.x * c0s.y, x.y * c0s.z - y.y * c0s.w);
+                                plo[it].y = pack_bf16x2(x.z * c1s.x - y.z * c1s.y, x.w * c1s.z - y.w * c1s.w);
+                                phi[it].x = pack_bf16x2(y.x * c0s.x + x.x * c0s.y, y.y * c0s.z + x.y * c0s.w);
+                                phi[it].y = pack_bf16x2(y.z * c1s.x + x.z * c1s.y, y.w * c1s.z + x.w * c1s.w);
                             }
                         } else {
 #pragma unroll
                             for (int it = 0; it < NI; ++it) {
                                 const int nl = (et >> 4) + 8 * it;
-                                const float4 x0 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8);
-                                const float4 x1 = *reinterpret_cast<const float4*>(acc_s + nl * 128 + j8 + 4);
-                                packed[it] = make_uint4(pack_bf16x2(x0.x, x0.y), pack_bf16x2(x0.z, x0.w), pack_bf16x2(x1.x, x1.y),
-                                                        pack_bf16x2(x1.z, x1.w));
+                                const float4 x = *reinterpret_cast<const float4*>(acc_s + nl * 128 + lo);
+                                const float4 y = *reinterpret_cast<const float4*>(acc_s + nl * 128 + hi);
+                                plo[it] = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+                                phi[it] = make_uint2(pack_bf16x2(y.x, y.y), pack_bf16x2(y.z, y.w));
                             }
                         }
-                        if (mat == 0 || p.kv_rows == nullptr) {
-                            uint16_t* base = mat == 0 ? p.q_out + (size_t)c0 * p.n_out
-                                                      : (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + c0) * p.n_out;
+                        uint16_t* base;
+                        if (mat == 0) base = p.q_out + (size_t)c0 * p.n_out;
+                        else base = (mat == 1 ? p.kcache : p.vcache) + (size_t)(p.prefix_len + (p.kv_rows == nullptr ? c0 : 0)) * p.n_out;
 #pragma unroll
-                            for (int it = 0; it < NI; ++it) {
-                                const int nl = (et >> 4) + 8 * it;
-                                if (nl < n_hi) *reinterpret_cast<uint4*>(base + (size_t)nl * p.n_out + feat) = packed[it];
-                            }
-                        } else {
-                            // a subset of the tree: row t of the batch is tree node kv_rows[t]
-                            uint16_t* base = (mat == 1 ? p.kcache : p.vcache) + (size_t)p.prefix_len * p.n_out;
-#pragma unroll
-                            for (int it = 0; it < NI; ++it) {
-                                const int nl = (et >> 4) + 8 * it;
-                                if (nl < n_hi)
-                                    *reinterpret_cast<uint4*>(base + (size_t)__ldg(p.kv_rows + c0 + nl) * p.n_out + feat) = packed[it];
+                        for (int it = 0; it < NI; ++it) {
+                            const int nl = (et >> 4) + 8 * it;
+                            if (nl < n_hi) {
+                                // a subset of the tree: row t of the batch is tree node kv_rows[t] (K and V only)
+                                const size_t row = (mat == 0 || p.kv_rows == nullptr) ? (size_t)nl : (size_t)__ldg(p.kv_rows + c0 + nl);
+                                uint16_t* dst = base + row * p.n_out + row0;
+                                *reinterpret_cast<uint2*>(dst + lo) = plo[it];
+                                *reinterpret_cast<uint2*>(dst + hi) = phi[it];
                             }
                         }
                     }
