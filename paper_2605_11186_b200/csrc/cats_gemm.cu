@@ -148,7 +148,7 @@ __device__ __forceinline__ void st_release(int* p, int v) {
 // CTA's share of one projection that carries its pipeline counters in and out.
 // ---------------------------------------------------------------------------------------------------
 struct CtaRange {
-    long long u0, u1;     // this CTA's units in the phase's unit space (see below)
+    int u0, u1;           // this CTA's units in the phase's unit space (see below; the unit count fits 32 bits, checked by the host)
     int vlen, koff;       // every tile owns vlen consecutive units, unit v of a tile being its K unit koff + v
     bool helper;
 };
@@ -163,25 +163,26 @@ __device__ __forceinline__ CtaRange cta_range(const GemmDev& p, int cta) {
     r.vlen = p.n_ku;
     r.koff = 0;
     r.helper = false;
+    const int total = (int)p.total_units;
     if (p.head_units > 0) {
         if (cta < p.n_tiles) {
             r.vlen = p.head_units;
-            r.u0 = (long long)cta * r.vlen;
+            r.u0 = cta * r.vlen;
             r.u1 = r.u0 + r.vlen;
         } else {
             r.helper = true;
             r.vlen = p.n_ku - p.head_units;
             r.koff = p.head_units;
-            r.u0 = min((long long)p.total_rem, (long long)(cta - p.n_tiles) * p.help_upc);
-            r.u1 = min((long long)p.total_rem, r.u0 + p.help_upc);
+            r.u0 = min(p.total_rem, (cta - p.n_tiles) * p.help_upc);
+            r.u1 = min(p.total_rem, r.u0 + p.help_upc);
         }
     } else if (p.split_s > 0) {
-        const long long t0 = (long long)(cta / p.split_s) * p.n_ku;
-        r.u0 = min(t0 + p.n_ku, t0 + (long long)(cta % p.split_s) * p.units_per_cta);
-        r.u1 = min(t0 + p.n_ku, r.u0 + (long long)p.units_per_cta);
+        const int t0 = (cta / p.split_s) * p.n_ku;
+        r.u0 = min(t0 + p.n_ku, t0 + (cta % p.split_s) * p.units_per_cta);
+        r.u1 = min(t0 + p.n_ku, r.u0 + p.units_per_cta);
     } else {
-        r.u0 = min(p.total_units, (long long)cta * p.units_per_cta);
-        r.u1 = min(p.total_units, r.u0 + (long long)p.units_per_cta);
+        r.u0 = min(total, cta * p.units_per_cta);
+        r.u1 = min(total, r.u0 + p.units_per_cta);
     }
     if (r.u1 < r.u0) r.u1 = r.u0;
     return r;
@@ -203,14 +204,17 @@ struct Pipe {               // the CTA's pipeline resources, the same for every 
 // its size (measured), so the two kinds of copies come from different threads.  i: units issued so far by this CTA
 // over all phases (ring position).  Returns false after an abort.
 __device__ __forceinline__ bool produce_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, bool is_w, uint64_t pol, int& i) {
+    // No division in the loop: the thread that issues the copies is the pace maker of the stream, and an integer
+    // division costs it hundreds of cycles.  (tile, v): the unit's tile and its position among the tile's units;
+    // (s, par): ring stage and the parity of the stage's "empty" phase to wait for.
     const int S = pp.S;
-    const int n_units = (int)(r.u1 - r.u0);
+    const int n_units = r.u1 - r.u0;
+    int tile = r.u0 / r.vlen, v = r.u0 - tile * r.vlen;
+    int s = i % S;
+    uint32_t par = ((uint32_t)(i / S) & 1u) ^ 1u;
     for (int k = 0; k < n_units; ++k, ++i) {
-        if (i >= S && !mbar_wait(&pp.ctrl->empty[i % S], ((i / S) - 1) & 1, pp.abort_flag)) return false;
-        const int s = i % S;
-        const long long u = r.u0 + k;
-        const int tile = (int)(u / r.vlen);
-        const int kb = (r.koff + (int)(u - (long long)tile * r.vlen)) * kUnitKb;
+        if (i >= S && !mbar_wait(&pp.ctrl->empty[s], par, pp.abort_flag)) return false;
+        const int kb = (r.koff + v) * kUnitKb;
         const int nk = min(kUnitKb, p.n_kb - kb);
         uint8_t* stage = pp.stages + (size_t)s * p.stage_bytes;
         if (is_w) {
@@ -222,6 +226,8 @@ __device__ __forceinline__ bool produce_units(const GemmDev& p, const CtaRange& 
             mbar_expect_tx(&pp.ctrl->full[s], bytes);
             bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &pp.ctrl->full[s], pol);
         }
+        if (++s == S) { s = 0; par ^= 1u; }
+        if (++v == r.vlen) { v = 0; ++tile; }
     }
     return true;
 }
@@ -236,22 +242,24 @@ __device__ __forceinline__ void drain_after_abort(const Pipe& pp, int i) {
 __device__ __forceinline__ bool mma_units(const GemmDev& p, const CtaRange& r, const Pipe& pp, int& i, int& seg, int half) {
     const int S = pp.S;
     const uint32_t idesc = umma_idesc_bf16_m128(p.n_pad);
+    const int k_lo = pp.dual ? 2 * half : 0, k_hi = pp.dual ? 2 * half + 2 : 4;
     bool ok = true;
-    for (long long u = r.u0; u < r.u1 && ok; ++seg) {
-        const long long tile_end = (u / r.vlen + 1) * r.vlen;
-        const long long seg_end = min(r.u1, tile_end);
+    // as in produce_units: no division per unit.  v: position of unit u among its tile's units
+    int u = r.u0, v = r.u0 % r.vlen;
+    int s = i % S;
+    uint32_t par = (uint32_t)(i / S) & 1u;
+    while (u < r.u1 && ok) {
+        const int seg_end = min(r.u1, u + (r.vlen - v));
         const int b = seg & 1;
         if (seg >= 2) ok = mbar_wait(&pp.ctrl->acc_empty[b], ((seg >> 1) - 1) & 1, pp.abort_flag);
         tc_fence_after_sync();
         const uint32_t d_addr = pp.tmem_acc + (uint32_t)(b * pp.acc_stride + half * p.n_pad);
-        const int k_lo = pp.dual ? 2 * half : 0, k_hi = pp.dual ? 2 * half + 2 : 4;
         bool first = true;
-        for (; u < seg_end && ok; ++u, ++i) {
-            const int s = i % S;
-            ok = mbar_wait(&pp.ctrl->full[s], (i / S) & 1, pp.abort_flag);
+        for (; u < seg_end && ok; ++u, ++i, ++v) {
+            ok = mbar_wait(&pp.ctrl->full[s], par, pp.abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
-            const int kb = (r.koff + (int)(u % r.vlen)) * kUnitKb;
+            const int kb = (r.koff + v) * kUnitKb;
             const int nk = min(kUnitKb, p.n_kb - kb);
             const uint32_t a_addr = smem_u32(pp.stages + (size_t)s * p.stage_bytes);
             const uint32_t b_addr = a_addr + kUnitKb * kWChunk;
@@ -262,8 +270,11 @@ __device__ __forceinline__ bool mma_units(const GemmDev& p, const CtaRange& r, c
                 first = false;
             }
             umma_commit(&pp.ctrl->empty[s]);
+            if (++s == S) { s = 0; par ^= 1u; }
         }
+        if (v == r.vlen) v = 0;
         umma_commit(&pp.ctrl->acc_full[b]);   // also on abort, so that the epilogue warps wake up
+        ++seg;
     }
     return ok;
 }
@@ -280,11 +291,11 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
     const int et = ew * 32 + lane;         // 0..127 among the group's threads
     float* const acc_s = pp.acc_s + (size_t)group * kStagingCols * 128;
     const int c_first = group * kStagingCols, c_step = kEpiGroups * kStagingCols;
-    for (long long u = r.u0; u < r.u1; ++seg) {
-        const int tile = (int)(u / r.vlen);
-        const long long tile_begin = (long long)tile * r.vlen;
-        const long long tile_end = tile_begin + r.vlen;
-        const long long seg_end = min(r.u1, tile_end);
+    for (int u = r.u0; u < r.u1; ++seg) {
+        const int tile = u / r.vlen;
+        const int tile_begin = tile * r.vlen;
+        const int tile_end = tile_begin + r.vlen;
+        const int seg_end = min(r.u1, tile_end);
         const bool tail = (seg_end == tile_end);
         const bool head = !r.helper && (u == tile_begin);
         u = seg_end;
@@ -294,13 +305,13 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
         if (p.head_units > 0) {
             // the tile's remaining units [tile * R, (tile + 1) * R) are spread over at most two helpers
             const int R = p.n_ku - p.head_units;
-            const int j0 = (int)(((long long)tile * R) / p.help_upc), j1 = (int)(((long long)(tile + 1) * R - 1) / p.help_upc);
+            const int j0 = (tile * R) / p.help_upc, j1 = ((tile + 1) * R - 1) / p.help_upc;
             g_first = 2 * tile;
             g_n = j1 - j0 + 1;
             if (r.helper) my_slot = 2 * tile + ((cta - p.n_tiles) - j0);
         } else {
-            head_cta = (int)(tile_begin / p.units_per_cta);
-            last_cta = (int)((tile_end - 1) / p.units_per_cta);
+            head_cta = tile_begin / p.units_per_cta;
+            last_cta = (tile_end - 1) / p.units_per_cta;
             g_first = cta + 1;
             g_n = (head && !tail) ? last_cta - cta : 0;
         }
@@ -871,6 +882,7 @@ cudaError_t launch_gemm(const GemmProblem& p, cudaStream_t st) {
     const GemmPlan pl = gemm_plan(p);
     GemmDev d;
     const size_t smem = make_gemm_dev(p, pl, pl.units_per_cta, d);
+    if (d.total_units + (long long)kGemmCtas * pl.units_per_cta >= (1ll << 31)) return cudaErrorInvalidValue;   // the kernel counts units in 32 bits
     switch (p.epi) {
         case EPI_PARTIAL: return launch_pdl(k_gemm_sk<EPI_PARTIAL>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
         case EPI_QKV: return launch_pdl(k_gemm_sk<EPI_QKV>, dim3(pl.n_ctas), dim3(kGemmThreads), smem, st, d);
