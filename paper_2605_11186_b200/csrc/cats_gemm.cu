@@ -40,7 +40,10 @@ constexpr int kGemmThreads = 384;      // warps: 0 W producer, 1 and 7 MMA issue
 constexpr int kCtrlBytes = 512;
 constexpr int kMaxStages = 14;
 constexpr int kWChunk = 16384;        // 128 rows x 64 bf16
-constexpr int kUnitKb = 2;            // K blocks per pipeline stage (one bulk copy of W, one of X)
+#ifndef CATS_UNIT_KB
+#define CATS_UNIT_KB 2
+#endif
+constexpr int kUnitKb = CATS_UNIT_KB;   // K blocks per pipeline stage (one bulk copy of W, one of X)
 constexpr int kStagingCols = 32;      // epilogue staging tile: 32 nodes x 128 features fp32
 
 struct GemmDev {
@@ -655,7 +658,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
         }
     } else if (warp == 7) {
         // ---------------- second MMA issuer: the other two K = 16 steps of every K block, into its own accumulator half ----------------
-        if (lane == 0) {
+        if (kGemmDualIssue && lane == 0) {
             int i = 0, seg = 0;
             mma_units(p, r, pp, i, seg, 1);
         }
