@@ -51,6 +51,15 @@ int cats_debug_wait_limit_ns(unsigned long long ns);
  * Set a short wait limit first, or each expiry takes a second. */
 void cats_debug_inject_fault(int which);
 
+/* Measurement: which weights the kernels that leave HBM idle request into L2
+ * for the projections after them.  which: 0 attention -> O projection,
+ * 1 attention -> gate/up, 2 attention -> down, 3 the norm before QKV -> QKV,
+ * 4 the norm before gate/up -> gate/up.  Of the matrix's 32 KB units every
+ * period-th one is requested, starting at unit `phase`; period 0: none,
+ * -1: the built-in choice (default for 1 and 3, the others default to 0).
+ * Changes no result. */
+void cats_debug_l2_warm(int which, int period, int phase);
+
 #ifdef __cplusplus
 }
 #endif

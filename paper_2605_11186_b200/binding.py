@@ -203,6 +203,13 @@ def inject_fault(which: int) -> None:
     lib.cats_debug_inject_fault(C.c_int(which))
 
 
+def l2_warm(which: int, period: int, phase: int = 0) -> None:
+    """cats_debug_l2_warm: which weights the kernels that leave HBM idle request into L2 (0 attention -> O, 1 attention ->
+    gate/up, 2 attention -> down, 3 norm before QKV -> QKV, 4 norm before gate/up -> gate/up); every period-th 32 KB unit
+    from unit ``phase``; period 0 none, -1 the built-in choice."""
+    lib.cats_debug_l2_warm(C.c_int(which), C.c_int(period), C.c_int(phase))
+
+
 def workspace_layout(cfg: ModelCfg, T: int) -> dict:
     """Byte offsets of the intermediate buffers inside the workspace (for tests that inspect them)."""
     out = (C.c_size_t * 8)()

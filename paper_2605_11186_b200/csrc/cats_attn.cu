@@ -68,6 +68,7 @@ struct AttnDev {
     float* part_o;       // n_outer > 1: [nh][n_outer][T_pad][hd] fp32
     float* part_ml;      //              [nh][n_outer][T_pad][2]
     int dbg_skip_q;      // fault injection (tcgen05 kernel): the loader announces Q but never copies it
+    WarmReq warm[3];     // see AttnProblem
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -717,6 +718,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 tma_load_2d(q_s + 128 * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
             }
             for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 1, ld_policy);
+            if (!STREAM) {
+                // a one-block share moves little data: HBM is free to fetch the coming projections' weights meanwhile
+                const unsigned n_cta = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
+#pragma unroll
+                for (int w = 0; w < 3; ++w) l2_warm(p.warm[w], me, n_cta);
+            }
             for (int j = NST; STREAM && j < nb; ++j) {
                 if (!mbar_wait(bar_free + j % NST, (uint32_t)(j / NST - 1) & 1u, wait_expired)) break;
                 mbar_expect_tx(bar_kv + j % NST, (uint32_t)stage_bytes);
@@ -1126,6 +1133,7 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     d.part_o = p.part_o; d.part_ml = p.part_ml;
     d.d_status = p.d_status;
     d.dbg_skip_q = g_debug_fault == 2 ? 1 : 0;
+    for (int w = 0; w < 3; ++w) d.warm[w] = warm_req(p.warm[w].ptr, p.warm[w].bytes, p.warm[w].period, p.warm[w].phase);
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;

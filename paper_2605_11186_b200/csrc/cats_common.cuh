@@ -55,6 +55,32 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // launch_dependents: lets the next kernel in the stream start its prologue.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- requests into L2 ----------------------------------------------------------------------------
+// Weights a later kernel will stream, requested into L2 by a kernel that leaves HBM idle: of the 32 KB units of
+// [ptr, ptr + bytes) every period-th one starting at unit `phase`, so that the later kernel draws on L2 and HBM at once.
+struct WarmReq {
+    const uint8_t* ptr;
+    unsigned long long bytes;     // 0: nothing
+    int period, phase;
+};
+constexpr unsigned kWarmUnit = 32768;
+// Called by ONE thread of each of n_cta CTAs (me: its index): the selected units are dealt out round robin.
+__device__ __forceinline__ void l2_warm(const WarmReq& w, unsigned me, unsigned n_cta) {
+    if (w.bytes == 0) return;
+    const unsigned n_units = (unsigned)(w.bytes / kWarmUnit);
+    for (unsigned u = (unsigned)w.phase + me * (unsigned)w.period; u < n_units; u += n_cta * (unsigned)w.period)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(w.ptr + (size_t)u * kWarmUnit), "r"(kWarmUnit) : "memory");
+}
+inline WarmReq warm_req(const void* ptr, size_t bytes, int period, int phase) {
+    WarmReq w;
+    const bool on = ptr != nullptr && period >= 1 && phase >= 0 && bytes >= kWarmUnit;
+    w.ptr = on ? (const uint8_t*)ptr : nullptr;
+    w.bytes = on ? (unsigned long long)bytes : 0ull;
+    w.period = on ? period : 1;
+    w.phase = on ? phase : 0;
+    return w;
+}
+
 // ---- mbarrier -----------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

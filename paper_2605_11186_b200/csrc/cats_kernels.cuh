@@ -48,7 +48,7 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
                            float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st,
-                           int32_t* d_status = nullptr);
+                           int32_t* d_status = nullptr, const WarmReq* warm = nullptr);   // warm: see WarmReq (register kernel only)
 // Checks a partial-tree node list (strictly ascending, inside [0, T)) and writes a copy clamped into range.
 cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,
@@ -156,6 +156,7 @@ struct AttnProblem {
     int mt_per_cta;     //   query tiles per CTA in that case
     int use_tc;         //   1: the tcgen05 kernel (head_dim 128)
     int32_t* d_status;
+    WarmReq warm[3];    // weights of the projections that follow, to be requested into L2 (tcgen05 kernel, one-block shares)
 };
 // Chooses the KV split; returns bytes of partial storage needed.
 size_t attn_plan(AttnProblem& p);

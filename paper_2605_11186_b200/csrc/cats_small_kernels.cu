@@ -450,7 +450,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
                                                      uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
                                                      const int32_t* __restrict__ nodes, float2* __restrict__ rope, int hd,
                                                      float rope_base, int* zero_flags, int n_flags, int cs,
-                                                     int32_t* d_status) {
+                                                     int32_t* d_status, const WarmReq warm) {
     __shared__ float red[8];
     __shared__ __align__(8) uint64_t xbar;     // completes when the partial sums of squares of all cs CTAs have landed
     __shared__ float slots[4];                 // slots[r]: the partial sum of the cluster's CTA r
@@ -497,6 +497,8 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
             if (s < n_part && cl < cols_cta)
                 pv[j][s] = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + col0 + cl);
     }
+    // weights of the projection that follows, beyond what its own first copies fetch: requested into L2 while HBM is idle
+    if (threadIdx.x == 32) l2_warm(warm, blockIdx.x, gridDim.x);
     // the rotary table of this node (fp64 so that large positions lose no accuracy): computed while the loads are in flight
     if (rope != nullptr && rank == cs - 1) {
         int half = hd / 2;
@@ -615,12 +617,13 @@ cudaError_t launch_embed(const void* E, const int32_t* tokens, int T, int H, int
 cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* part, int n_part, size_t part_stride,
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
                            float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st,
-                           int32_t* d_status) {
+                           int32_t* d_status, const WarmReq* warm_in) {
     const int n_pad = (T + 15) / 16 * 16;
+    const WarmReq warm = warm_in ? warm_req(warm_in->ptr, warm_in->bytes, warm_in->period, warm_in->phase) : warm_req(nullptr, 0, 0, 0);
 #define CATS_NORM_REG(NC)                                                                                                   \
     return launch_cluster_pdl(k_rmsnorm_reg<NC>, dim3(T * cs), dim3(256), cs, st, resid, copy_from, part, n_part, part_stride, \
                               (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, n_pad, pos, nodes, rope, hd, rope_base,    \
-                              zero_flags, n_flags, cs, d_status)
+                              zero_flags, n_flags, cs, d_status, warm)
 #ifndef CATS_NORM_SMEM
     {
         // as many CTAs per row as keep the grid within one wave and leave every CTA at least 256 columns
