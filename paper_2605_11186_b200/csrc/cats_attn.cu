@@ -708,7 +708,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 // the cache rows of the CTAs that start last (measured: the kernel 3.8 us longer).
                 const unsigned n_cta = gridDim.x * gridDim.y, me = blockIdx.y * gridDim.x + blockIdx.x;
 #pragma unroll
-                for (int w = 0; w < 3; ++w) l2_warm(p.warm[w], me, n_cta);
+                for (int w = 0; w < 3; ++w) l2_warm(p.warm[w], me, n_cta, 24);
             }
             if (!STREAM && ok) issue_pv(0);      // one-block share: the same thread issues P V as well
         }

@@ -64,11 +64,14 @@ struct WarmReq {
     int period, phase;
 };
 constexpr unsigned kWarmUnit = 32768;
-// Called by ONE thread of each of n_cta CTAs (me: its index): the selected units are dealt out round robin.
-__device__ __forceinline__ void l2_warm(const WarmReq& w, unsigned me, unsigned n_cta) {
+// Called by n_workers threads (me: the caller's index among them), best one per warp: a request costs its thread
+// 60-120 ns and the lanes of a warp take turns.  The selected units are dealt out round robin, at most max_each per
+// caller (what does not fit is simply not requested).
+__device__ __forceinline__ void l2_warm(const WarmReq& w, unsigned me, unsigned n_workers, int max_each) {
     if (w.bytes == 0) return;
     const unsigned n_units = (unsigned)(w.bytes / kWarmUnit);
-    for (unsigned u = (unsigned)w.phase + me * (unsigned)w.period; u < n_units; u += n_cta * (unsigned)w.period)
+    int n = 0;
+    for (unsigned u = (unsigned)w.phase + me * (unsigned)w.period; u < n_units && n < max_each; u += n_workers * (unsigned)w.period, ++n)
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(w.ptr + (size_t)u * kWarmUnit), "r"(kWarmUnit) : "memory");
 }
 inline WarmReq warm_req(const void* ptr, size_t bytes, int period, int phase) {

@@ -498,7 +498,8 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
                 pv[j][s] = __ldcg(reinterpret_cast<const float4*>(part + (size_t)s * part_stride + (size_t)t * H) + col0 + cl);
     }
     // weights of the projection that follows, beyond what its own first copies fetch: requested into L2 while HBM is idle
-    if (threadIdx.x == 32) l2_warm(warm, blockIdx.x, gridDim.x);
+    // (one thread of every warp, a few requests each, while the loads above are in flight)
+    if ((threadIdx.x & 31) == 0) l2_warm(warm, blockIdx.x * 8 + (threadIdx.x >> 5), gridDim.x * 8, 8);
     // the rotary table of this node (fp64 so that large positions lose no accuracy): computed while the loads are in flight
     if (rope != nullptr && rank == cs - 1) {
         int half = hd / 2;
