@@ -33,9 +33,11 @@ UNIT = "tree tokens/s"
 PREFIX = 512
 SWEEP = (16, 32, 64, 128)
 # dram__bytes_read + dram__bytes_write of the four projection launches of a layer at T=64, from the ncu capture of a
-# 2-layer stack summarised under profiles/ (QKV 101.3+3.2, O 34.1+0.0, gate/up 180.9+6.5, down 91.6+3.2 MB), scaled to the
-# 128 layer launches of a forward; the LM head (not captured) is counted at its packed size.
-NCU_TRAFFIC_PER_LAUNCH = (32 * (104.5e6 + 34.1e6 + 187.4e6 + 94.8e6) + 262.1e6) / 129
+# 2-layer stack summarised under profiles/ (QKV 101.3+3.7, O 34.1+0.0, gate/up 180.9+4.8, down 91.6+3.0 MB), scaled to the
+# 128 layer launches of a forward; the LM head (not captured) is counted at its packed size.  (ncu replays every launch
+# with cold caches; inside a forward part of these bytes has already been requested into L2 by the attention and norm
+# kernels, which is why the timed fraction below comes from a run of the projections alone.)
+NCU_TRAFFIC_PER_LAUNCH = (32 * (105.0e6 + 34.1e6 + 185.7e6 + 94.6e6) + 262.1e6) / 129
 TARGET_FORWARD_FRAC_OF_8TBS = 0.70
 
 
