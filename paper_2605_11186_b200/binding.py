@@ -188,7 +188,8 @@ def stage_mask(mask: int) -> None:
 
 
 def attention_kernel(which: int) -> None:
-    """cats_debug_attention_kernel: -1 by shape (default), 0 the mma.sync kernel, 1 the tcgen05 kernel."""
+    """cats_debug_attention_kernel: -1 by shape (default), 0 the mma.sync kernel, 1 the tcgen05 kernel, 2 the tcgen05
+    kernel with two softmax threads per query row for every tree size."""
     lib.cats_debug_attention_kernel(C.c_int(which))
 
 

@@ -256,7 +256,7 @@ int cats_last_launch_count(void) { return g_launch_count; }
 
 /* Measurement and fault-injection hooks, declared in include/cats_debug.h. */
 void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
-void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which ? 1 : 0); }
+void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which > 2 ? 1 : which); }
 void cats_debug_l2_warm(int which, int period, int phase) { if (which >= 0 && which < 5) { g_warm[which][0] = period; g_warm[which][1] = phase; } }
 void cats_debug_inject_fault(int which) { g_debug_fault = (which == 1 || which == 2) ? which : 0; }
 int cats_debug_wait_limit_ns(unsigned long long ns) {

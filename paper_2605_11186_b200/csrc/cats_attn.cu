@@ -490,6 +490,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1) k_tree_attn(const AttnDev p) 
 // ---------------------------------------------------------------------------------------------------
 constexpr int kTcThreads = 352;       // warps 0-7: softmax; 8: issue of Q K^T, tensor-memory allocation; 9: TMA loads; 10: issue of P V
                                       // (streamed shares only: a one-block share is launched with 320 threads)
+// Trees of at most 64 nodes fill only the tensor-memory lanes 0-63, which only warps with (warp index mod 4) in {0, 1} can
+// reach: the WIDE instances run 14 warps so that eight of them (0, 1, 4, 5, 8, 9, 12, 13) are such warps and FOUR threads
+// share every query row instead of two.  There warp 2 issues Q K^T and allocates, warp 3 loads, warp 6 issues P V.
+constexpr int kTcThreadsWide = 448;
 constexpr int kTcBoxRows = 32;        // rows of one TMA box (64 head-dim elements wide)
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
@@ -536,18 +540,20 @@ __device__ __forceinline__ uint32_t tc_visible16(int g0, int P, int c_end, uint6
     }
     return bits;
 }
-__device__ __forceinline__ void pair_barrier(int quadrant) {     // the two warps that share a lane quadrant
-    asm volatile("bar.sync %0, 64;" ::"r"(quadrant + 1) : "memory");
+template <int NT>
+__device__ __forceinline__ void pair_barrier(int quadrant) {     // the NT threads (two or four warps) that share a lane quadrant
+    asm volatile("bar.sync %0, %1;" ::"r"(quadrant + 1), "n"(NT) : "memory");
 }
+template <int NT>
 __device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     // the same barrier, returning the OR of pred
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, %2, 64, q;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(r)
-        : "r"((uint32_t)pred), "r"(quadrant + 1)
+        : "r"((uint32_t)pred), "r"(quadrant + 1), "n"(NT)
         : "memory");
     return r != 0;
 }
@@ -555,8 +561,8 @@ __device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     /
 // CPT: the most columns of S one softmax thread holds (a block has at most 2 CPT rows); instances for the streamed
 // 64-row blocks and for one-block shares of up to 128, 160 and 192 rows.
 // STREAM: the share is streamed in blocks (otherwise it is one block, and everything that hands blocks on is compiled out).
-template <int CPT, bool STREAM>
-__global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
+template <int CPT, bool STREAM, bool WIDE>
+__global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
                                                                 const __grid_constant__ CUtensorMap tm_k,
                                                                 const __grid_constant__ CUtensorMap tm_v) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
@@ -565,8 +571,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     const int Tpad = p.n_mt * 16;
     uint8_t* q_s = sm;                                                           // [2][128][128 B]
     uint8_t* kv_s = q_s + 128 * 256;                                             // ring of K and V blocks
-    float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][2][128] row maxima (by block parity), [2][128] row sums
-    float* recv = xch + 768;                                                     // [csize][rpr][REC]
+    constexpr int NH = WIDE ? 4 : 2;                                             // softmax threads per query row
+    constexpr int W_ISSUE = WIDE ? 2 : 8, W_LOAD = WIDE ? 3 : 9, W_PV = WIDE ? 6 : 10;
+    float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][NH][128] row maxima (by block parity), [NH][128] row sums
+    float* recv = xch + 3 * NH * 128;                                            // [csize][rpr][REC]
     uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // base of the mbarriers; slot 0 unused
     // Every barrier that a thread may find more than one phase ahead of itself would give a wrong answer to a parity
     // wait, so each one is either indexed by block parity (its next completion needs the waiter's own progress) or by
@@ -586,6 +594,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool softmax_warp = WIDE ? (warp & 2) == 0 : warp < 8;
     const int split = (int)blockIdx.x, h = blockIdx.y;
     const int S = p.P + p.Tk;
     const int c_begin = min(S, split * p.rows_per_split);
@@ -616,7 +625,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     };
 
     pdl_launch_dependents();
-    if (warp == 8) {
+    if (warp == W_ISSUE) {
         tmem_alloc(tmem_slot, kTcCols);
         tmem_relinquish();
         if (lane == 0) {
@@ -630,7 +639,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         }
     }
     uint64_t ld_policy = 0;
-    if (warp == 9 && lane == 0) {
+    if (warp == W_LOAD && lane == 0) {
         // The loader sets up its own barriers and requests the prefix rows of every stage of the ring at once: they depend
         // neither on the previous kernel nor on the rest of the set-up.
         for (int i = 0; i < kTcMaxStages; ++i) { mbar_init(bar_kv + i, 1); mbar_init(bar_free + i, 1); }
@@ -677,7 +686,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         umma_commit(bar_free + b % NST);
         return true;
     };
-    if (warp == 8) {
+    if (warp == W_ISSUE) {
         // ---- issue of S(b) = Q K(b)^T: as soon as block b has landed and the product that read the S / P buffer of
         //      block b - 2 has completed (issuing one tcgen05.mma costs its thread about a hundred cycles, so the two
         //      kinds of products are issued by two threads) ----
@@ -712,12 +721,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             }
             if (!STREAM && ok) issue_pv(0);      // one-block share: the same thread issues P V as well
         }
-    } else if (STREAM && warp == 10) {
+    } else if (STREAM && warp == W_PV) {
         // ---- issue of O += P(b) V(b) for streamed shares (a one-block share is launched without this warp) ----
         if (lane == 0)
             for (int b = 0; b < nb; ++b)
                 if (!issue_pv(b)) break;
-    } else if (warp == 9) {
+    } else if (warp == W_LOAD) {
         // ---- loader: Q and the boxes that depend on the previous kernel, then a refill whenever a P V product frees a stage ----
         if (lane == 0) {
             if (nb > 0) mbar_expect_tx(bar_q, 128u * 256u);
@@ -732,13 +741,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 load_kv(j, j % NST, 2, ld_policy);
             }
         }
-    } else {
-        // ---- warps 0-7: softmax ----
+    } else if (softmax_warp) {
+        // ---- the eight softmax warps: NH of them share a lane quadrant and split the block's columns ----
         const int quad = warp & 3, hf = warp >> 2;
         const int row = quad * 32 + lane;                       // the query row (= TMEM lane) of this thread
         const bool act = quad * 32 < Tpad;                      // the warp owns query rows
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const int ncol = NB / 2, c0 = hf * ncol;                // this thread's columns of a block
+        const int ncol = ((NB / 16 + NH - 1) / NH) * 16, c0 = hf * ncol;   // this thread's columns of a block (whole groups of 16)
         uint64_t mk0 = 0ull, mk1 = 0ull;
         if (row < p.T) {
             const size_t node = p.nodes != nullptr ? p.nodes[row] : row;
@@ -757,13 +766,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
             if (act) {
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16)
-                    if (c < ncol) tmem_ld16_nowait(tS + lane_base + (uint32_t)(c0 + c), v + c);
+                    if (c < ncol && c0 + c < NB) tmem_ld16_nowait(tS + lane_base + (uint32_t)(c0 + c), v + c);
                 tmem_wait_ld<CPT>(v);
                 const int lim = min(p.P, c_end);
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // independent chains
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16) {
-                    if (c < ncol) {
+                    if (c < ncol && c0 + c < NB) {
                         const int g0 = r0 + c0 + c;
                         if (g0 + 16 > lim) {
                             const uint32_t vis = tc_visible16(g0, p.P, c_end, mk0, mk1);
@@ -782,15 +791,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 if (!STREAM) {
                     // the only block: its maximum is the reference (one exchange, whose barrier orders the loads and stores)
                     xch[hf * 128 + row] = mx;
-                    pair_barrier(quad);
-                    m_run = fmaxf(mx, xch[(hf ^ 1) * 128 + row]);
+                    pair_barrier<32 * NH>(quad);
+                    m_run = mx;
+#pragma unroll
+                    for (int k = 1; k < NH; ++k) m_run = fmaxf(m_run, xch[((hf + k) % NH) * 128 + row]);
                     ref = (m_run == -INFINITY) ? 0.f : m_run;
                 } else {
                     const bool want = !(m_run != -INFINITY && mx <= m_run + 8.f);
-                    if (pair_barrier_or(quad, want)) {
-                        xch[((b & 1) * 2 + hf) * 128 + row] = mx;
-                        pair_barrier(quad);
-                        mx = fmaxf(mx, xch[((b & 1) * 2 + (hf ^ 1)) * 128 + row]);
+                    if (pair_barrier_or<32 * NH>(quad, want)) {
+                        xch[((b & 1) * NH + hf) * 128 + row] = mx;
+                        pair_barrier<32 * NH>(quad);
+#pragma unroll
+                        for (int k = 1; k < NH; ++k) mx = fmaxf(mx, xch[((b & 1) * NH + (hf + k) % NH) * 128 + row]);
                         const float mn = (m_run != -INFINITY && mx <= m_run + 8.f) ? m_run : fmaxf(m_run, mx);
                         ref = (mn == -INFINITY) ? 0.f : mn;
                         corr = exp2f(m_run - ref);
@@ -806,12 +818,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 tc_fence_after_sync();
                 {
 #pragma unroll
-                    for (int c = 0; c < HD / 2; c += 16) {
+                    for (int c = 0; c < HD / NH; c += 16) {
                         float o[16];
-                        tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
+                        tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / NH) + c), o);
 #pragma unroll
                         for (int e = 0; e < 16; ++e) o[e] *= corr;
-                        tmem_st16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
+                        tmem_st16(tO + lane_base + (uint32_t)(hf * (HD / NH) + c), o);
                     }
                 }
             }
@@ -819,7 +831,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                 float ls4[4] = {0.f, 0.f, 0.f, 0.f};                      // independent chains, summed in a fixed order
 #pragma unroll
                 for (int c = 0; c < CPT; c += 16) {
-                    if (c < ncol) {
+                    if (c < ncol && c0 + c < NB) {
                         uint32_t hi[8], lo[8];
 #pragma unroll
                         for (int e = 0; e < 16; e += 2) {
@@ -834,7 +846,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                             lo[e >> 1] = __byte_perm(__float_as_uint(l0), __float_as_uint(l1), 0x7632);
                         }
                         tmem_st8(tS + lane_base + (uint32_t)((c0 + c) >> 1), hi);
-                        tmem_st8(tS + lane_base + (uint32_t)(ncol + ((c0 + c) >> 1)), lo);
+                        tmem_st8(tS + lane_base + (uint32_t)(NB / 2 + ((c0 + c) >> 1)), lo);
                     }
                 }
                 l_run = (STREAM ? l_run * corr : 0.f) + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
@@ -854,7 +866,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
         }
         if (p.csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA of the cluster has started
         if (act) {
-            float* xl = xch + 512;                              // [2][128]
+            float* xl = xch + 2 * NH * 128;                     // [NH][128]
             xl[hf * 128 + row] = l_run;
             // the record of (part = this CTA, row): in the merging CTA's recv area, or, for a lone CTA, over the idle ring
             const int dest = p.csize > 1 ? min(row / p.rpr, p.csize - 1) : 0;
@@ -862,10 +874,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
                                            : reinterpret_cast<const float*>(kv_s) + (size_t)row * REC;
             const uint32_t ra = cluster_map(smem_u32(rec), dest);
 #pragma unroll
-            for (int c = 0; c < HD / 2; c += 16) {
+            for (int c = 0; c < HD / NH; c += 16) {
                 float o[16];
                 if (nb > 0) {
-                    tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / 2) + c), o);
+                    tmem_ld16(tO + lane_base + (uint32_t)(hf * (HD / NH) + c), o);
                 } else {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) o[e] = 0.f;
@@ -874,12 +886,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
 #pragma unroll
                     for (int e = 0; e < 16; e += 4)
                         asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
-                                     ::"r"(ra + (uint32_t)(hf * (HD / 2) + c + e) * 4u), "f"(o[e]), "f"(o[e + 1]), "f"(o[e + 2]), "f"(o[e + 3]) : "memory");
+                                     ::"r"(ra + (uint32_t)(hf * (HD / NH) + c + e) * 4u), "f"(o[e]), "f"(o[e + 1]), "f"(o[e + 2]), "f"(o[e + 3]) : "memory");
                 }
             }
-            pair_barrier(quad);
-            if (hf == 0 && row < Tpad)
-                asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra + (uint32_t)HD * 4u), "f"(m_run), "f"(l_run + xl[128 + row]) : "memory");
+            pair_barrier<32 * NH>(quad);
+            if (hf == 0 && row < Tpad) {
+                float l_tot = l_run;
+#pragma unroll
+                for (int k = 1; k < NH; ++k) l_tot += xl[k * 128 + row];
+                asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra + (uint32_t)HD * 4u), "f"(m_run), "f"(l_tot) : "memory");
+            }
         }
     }
     tc_fence_before_sync();
@@ -889,8 +905,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     const float* src_parts = reinterpret_cast<const float*>(kv_s);
     int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
     if (csize > 1) {
-        // warps 0-7 have passed the first phase of the cluster barrier above; the second one publishes the records
-        if (warp >= 8) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        // the softmax warps have passed the first phase of the cluster barrier above; the second one publishes the records
+        if (!softmax_warp) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         row0 = min(Tpad, rank * rpr);
@@ -900,14 +916,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tree_attn_tc(const AttnDev p,
     } else {
         __syncthreads();
     }
-    if (warp == 8) {
+    if (warp == W_ISSUE) {
         tc_fence_after_sync();
         tmem_dealloc(tbase, kTcCols);
     }
     if (threadIdx.x == 0 && *wait_expired) report(p.d_status, CATS_ERR_TIMEOUT);
     // One thread per (query row, 8 output columns): all rows of the CTA are merged at once, every load of a thread is
     // independent of the others (the (m, l) pairs are broadcast reads), and the result leaves as one 16-byte store.
-    for (int it = threadIdx.x; it < n_my * (HD / 8) && warp < 8; it += 256) {
+    for (int it = threadIdx.x; it < n_my * (HD / 8); it += (int)blockDim.x) {
         const int rl = it / (HD / 8), c8 = (it % (HD / 8)) * 8;
         const int grow = row0 + rl;                    // global query row
         if (grow >= p.T) continue;
@@ -1013,7 +1029,7 @@ size_t attn_plan(AttnProblem& p) {
     // against the mma.sync kernel: 3.07 vs 3.07 ms at T = 1, 3.09 vs 3.10 at 8, 3.11 vs 3.13 at 16, 3.15 vs 3.22 at 32,
     // 3.40 vs 3.48 at 64, 3.96 vs 4.14 at 128; alone over 16384 rows: 74 vs 81 us at T = 16, 85 vs 253 us at T = 128).
     p.use_tc = (p.hd == 128 && p.scale > 0.f) ? 1 : 0;
-    if (attn_tc_override() >= 0) p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_override() == 1) ? 1 : 0;
+    if (attn_tc_override() >= 0) p.use_tc = (p.hd == 128 && p.scale > 0.f && attn_tc_override() >= 1) ? 1 : 0;
     const int n_mt = tpad / 16;
     if (!p.use_tc && n_mt >= 4 && S <= 1024) {     // measured at 32 heads: ahead up to about 1000 rows (15.8 vs 17.4 us at 576 rows), behind beyond
         int mpc = 1, groups = n_mt;
@@ -1110,11 +1126,15 @@ static bool attn_tensor_map(const void* ptr, long long cols, long long rows, lon
 static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<48, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -1139,7 +1159,8 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
-    const size_t fixed = 1024 + 128 * 256 + 3072 + recv + 192;     // alignment slack, Q, pair exchange, received partials, barriers
+    const bool wide = tpad <= 64 && g_debug_attn_kernel != 2;        // four softmax threads per query row (see kTcThreadsWide)
+    const size_t fixed = 1024 + 128 * 256 + (wide ? 6144 : 3072) + recv + 192;     // alignment slack, Q, exchange among a row's threads, received partials, barriers
     // the ring: stages of 64 rows of K and V (32 KB each), as many as fit, at least three (which also hold a one-block share)
     int stages = (int)((227 * 1024 - fixed) / (kTcStream * 512));
     if (stages > kTcMaxStages) stages = kTcMaxStages;
@@ -1162,11 +1183,17 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
         return cudaErrorNotSupported;
     cudaError_t e;
     const dim3 one(kTcThreads - 32);      // the warp that issues P V on its own exists for streamed shares only
-    if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<32, true>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else e = launch_cluster(k_tree_attn_tc<96, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    const dim3 wd(kTcThreadsWide);
+    if (wide) {
+        if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<16, true, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<16, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<32, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else e = launch_cluster(k_tree_attn_tc<48, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    } else if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<32, true, false>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else e = launch_cluster(k_tree_attn_tc<96, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
