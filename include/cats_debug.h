@@ -34,7 +34,7 @@ int cats_debug_workspace_layout(const cats_model_cfg *cfg, int32_t T, size_t *ou
 /* Attention kernel used for head_dim 128: -1 (default) chosen by shape, 0 the
  * mma.sync kernel (the fallback when the driver offers no tensor maps), 1 the
  * tcgen05 kernel, 2 the tcgen05 kernel with two softmax threads per query row
- * for every tree size (by default trees of at most 64 nodes get four). */
+ * (by default every tree gets four). */
 void cats_debug_attention_kernel(int which);
 
 /* Limit of every bounded device-side wait, in nanoseconds, on the CURRENT

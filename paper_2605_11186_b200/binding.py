@@ -189,7 +189,7 @@ def stage_mask(mask: int) -> None:
 
 def attention_kernel(which: int) -> None:
     """cats_debug_attention_kernel: -1 by shape (default), 0 the mma.sync kernel, 1 the tcgen05 kernel, 2 the tcgen05
-    kernel with two softmax threads per query row for every tree size."""
+    kernel with two softmax threads per query row instead of four."""
     lib.cats_debug_attention_kernel(C.c_int(which))
 
 

@@ -493,7 +493,11 @@ constexpr int kTcThreads = 352;       // warps 0-7: softmax; 8: issue of Q K^T, 
 // Trees of at most 64 nodes fill only the tensor-memory lanes 0-63, which only warps with (warp index mod 4) in {0, 1} can
 // reach: the WIDE instances run 14 warps so that eight of them (0, 1, 4, 5, 8, 9, 12, 13) are such warps and FOUR threads
 // share every query row instead of two.  There warp 2 issues Q K^T and allocates, warp 3 loads, warp 6 issues P V.
+// Larger trees get four threads per row too, with sixteen softmax warps (0-15; 16 issues Q K^T, 17 loads, 18 issues
+// P V): 19 warps leave 104 registers per thread, enough for every instance (at most 48 columns of S per thread: 87).
 constexpr int kTcThreadsWide = 448;
+constexpr int kTcThreadsWide128 = 608;
+constexpr int tc_threads(int wd) { return wd == 0 ? kTcThreads : (wd == 1 ? kTcThreadsWide : kTcThreadsWide128); }
 constexpr int kTcBoxRows = 32;        // rows of one TMA box (64 head-dim elements wide)
 constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), S1 / P [192,384), O [384,512)
 constexpr int kTcSStride = 192;
@@ -561,8 +565,8 @@ __device__ __forceinline__ bool pair_barrier_or(int quadrant, bool pred) {     /
 // CPT: the most columns of S one softmax thread holds (a block has at most 2 CPT rows); instances for the streamed
 // 64-row blocks and for one-block shares of up to 128, 160 and 192 rows.
 // STREAM: the share is streamed in blocks (otherwise it is one block, and everything that hands blocks on is compiled out).
-template <int CPT, bool STREAM, bool WIDE>
-__global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
+template <int CPT, bool STREAM, int WIDE>      // WIDE: 0 two softmax threads per query row, 1 four (trees of <= 64 nodes), 2 four (any tree)
+__global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const AttnDev p, const __grid_constant__ CUtensorMap tm_q,
                                                                 const __grid_constant__ CUtensorMap tm_k,
                                                                 const __grid_constant__ CUtensorMap tm_v) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
@@ -572,7 +576,8 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) k_tree_
     uint8_t* q_s = sm;                                                           // [2][128][128 B]
     uint8_t* kv_s = q_s + 128 * 256;                                             // ring of K and V blocks
     constexpr int NH = WIDE ? 4 : 2;                                             // softmax threads per query row
-    constexpr int W_ISSUE = WIDE ? 2 : 8, W_LOAD = WIDE ? 3 : 9, W_PV = WIDE ? 6 : 10;
+    constexpr int W_ISSUE = WIDE == 0 ? 8 : (WIDE == 1 ? 2 : 16), W_LOAD = W_ISSUE + 1, W_PV = WIDE == 1 ? 6 : W_ISSUE + 2;
+    constexpr int N_SOFTMAX = WIDE == 2 ? 512 : 256;                             // softmax threads (arrivals per hand-off)
     float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][NH][128] row maxima (by block parity), [NH][128] row sums
     float* recv = xch + 3 * NH * 128;                                            // [csize][rpr][REC]
     uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // base of the mbarriers; slot 0 unused
@@ -594,7 +599,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) k_tree_
     volatile int* wait_expired = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool softmax_warp = WIDE ? (warp & 2) == 0 : warp < 8;
+    const bool softmax_warp = WIDE == 0 ? warp < 8 : (WIDE == 1 ? (warp & 2) == 0 : warp < 16);
     const int split = (int)blockIdx.x, h = blockIdx.y;
     const int S = p.P + p.Tk;
     const int c_begin = min(S, split * p.rows_per_split);
@@ -633,7 +638,7 @@ __global__ void __launch_bounds__(WIDE ? kTcThreadsWide : kTcThreads, 1) k_tree_
             for (int i = 0; i < NSB; ++i) {
                 mbar_init(bar_s + i, 1);
                 mbar_init(bar_o + i, 1);
-                mbar_init(bar_p + i, 256);
+                mbar_init(bar_p + i, N_SOFTMAX);
             }
             mbar_fence_init();
         }
@@ -1126,15 +1131,19 @@ static bool attn_tensor_map(const void* ptr, long long cols, long long rows, lon
 static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<48, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(k_tree_attn_tc<32, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<64, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<80, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<96, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<48, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<16, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<32, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tree_attn_tc<48, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -1159,7 +1168,8 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
-    const bool wide = tpad <= 64 && g_debug_attn_kernel != 2;        // four softmax threads per query row (see kTcThreadsWide)
+    // four softmax threads per query row (see kTcThreadsWide), on 8 softmax warps for trees of <= 64 nodes, else on 16
+    const int wide = g_debug_attn_kernel == 2 ? 0 : (tpad <= 64 ? 1 : 2);
     const size_t fixed = 1024 + 128 * 256 + (wide ? 6144 : 3072) + recv + 192;     // alignment slack, Q, exchange among a row's threads, received partials, barriers
     // the ring: stages of 64 rows of K and V (32 KB each), as many as fit, at least three (which also hold a one-block share)
     int stages = (int)((227 * 1024 - fixed) / (kTcStream * 512));
@@ -1183,17 +1193,22 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
         return cudaErrorNotSupported;
     cudaError_t e;
     const dim3 one(kTcThreads - 32);      // the warp that issues P V on its own exists for streamed shares only
-    const dim3 wd(kTcThreadsWide);
-    if (wide) {
-        if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<16, true, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-        else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<16, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-        else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<32, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-        else e = launch_cluster(k_tree_attn_tc<48, false, true>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    } else if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<32, true, false>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
-    else e = launch_cluster(k_tree_attn_tc<96, false, false>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    const dim3 wd(kTcThreadsWide), wd2(kTcThreadsWide128);
+    if (wide == 2) {
+        if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<16, true, 2>, grid, wd2, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<16, false, 2>, grid, wd2, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<32, false, 2>, grid, wd2, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else e = launch_cluster(k_tree_attn_tc<48, false, 2>, grid, wd2, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    } else if (wide == 1) {
+        if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<16, true, 1>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<16, false, 1>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<32, false, 1>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+        else e = launch_cluster(k_tree_attn_tc<48, false, 1>, grid, wd, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    } else if (d.stages > 1) e = launch_cluster(k_tree_attn_tc<32, true, 0>, grid, dim3(kTcThreads), smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 64) e = launch_cluster(k_tree_attn_tc<32, false, 0>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 128) e = launch_cluster(k_tree_attn_tc<64, false, 0>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else if (d.blk <= 160) e = launch_cluster(k_tree_attn_tc<80, false, 0>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
+    else e = launch_cluster(k_tree_attn_tc<96, false, 0>, grid, one, smem, p.cluster, st, d, tm_q, tm_k, tm_v);
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);

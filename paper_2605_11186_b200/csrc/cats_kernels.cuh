@@ -16,7 +16,7 @@ extern thread_local bool g_call_boundary;
 
 // Measurement / fault-injection state set through the cats_debug_* hooks (include/cats_debug.h); process-wide.
 extern int g_debug_attn_kernel;   // -1: attention kernel chosen by shape; 0: mma.sync kernel; 1: tcgen05 kernel; 2: tcgen05 kernel,
-                                  // two softmax threads per query row for every tree size
+                                  // two softmax threads per query row instead of four
 extern int g_debug_fault;         // 0: none; 1: a helper CTA of a projection never publishes; 2: the attention loader drops Q
 cudaError_t set_wait_limit_gemm(unsigned long long ns);
 cudaError_t set_wait_limit_attn(unsigned long long ns);

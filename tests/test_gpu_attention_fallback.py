@@ -23,11 +23,11 @@ def test_head_dim_128_cases_on_the_mma_sync_kernel():
     assert " passed" in r.stdout and "failed" not in r.stdout
 
 
-def test_small_trees_on_the_two_threads_per_row_instances():
-    """Trees of at most 64 nodes normally run the instances with four softmax threads per query row; the instances with
-    two (the ones trees of 65-128 nodes use) are run on the same cases here."""
+def test_cases_on_the_two_threads_per_row_instances():
+    """By default every tree runs the instances with four softmax threads per query row; the instances with two are run
+    on the same cases here."""
     env = dict(os.environ, CATS_TEST_ATTENTION_KERNEL="2")
-    sel = "test_tree_attention_matches_oracle and (heap64_P256 or heap64_P4096 or chain16 or chain5_P0 or single_P1 or rand40 or rand49_P200_h32 or rand33 or rand17_P700_h40)"
+    sel = "test_tree_attention_matches_oracle and (heap64_P256 or heap64_P4096 or chain16 or chain5_P0 or single_P1 or rand40 or rand49_P200_h32 or rand33 or rand17_P700_h40 or rand128_P256 or rand128_P1024 or rand90_P5000_h32 or rand100_P63)"
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_gpu_parity.py"), "-q", "-x", "-k", sel],
                        env=env, cwd=ROOT, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
