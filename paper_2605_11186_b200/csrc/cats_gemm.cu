@@ -779,12 +779,15 @@ GemmPlan gemm_plan(const GemmProblem& p) {
         //   T = 64:  a = 24 / 25 / 26 / 27 / 28 -> 3.322 / 3.301 / 3.230 / 3.241 / 3.255 ms
         //   T = 128: a = 25 / 26 / 27 / 28      -> 4.072 / 3.955 / 3.976 / 3.979 ms
         // (an owner's SM pulls more once the helpers have finished, so the optimum is flat towards large shares: with
-        // a = 31, next to no help at all, the forward is only 2 % slower.)
+        // a = 31, next to no help at all, the forward is only 2 % slower.)  Measured again with a quarter of the matrix on its
+        // way into L2 when the kernel starts (lead = 7 / 8.5 / 10 / 11.5 / 13 units at T = 16, + 3 at T = 64, + 4.5 at T = 128):
+        //   T = 16: 2.672 / 2.673 / 2.658 / 2.659 / 2.634 ms    T = 64: 2.840 / 2.848 / 2.796 / 2.794 / 2.794 ms
+        //   T = 128: 3.50 / 3.46 / 3.41 / 3.45 / 3.47 ms  ->  13 units up to 64 nodes, 14.5 above.
         const int h = kGemmCtas - tiles;
         const double rho = (double)tiles / h;
         int lg = 0;                                    // log2(n_pad / 16): 0, 1, 2, 3 for trees of up to 16, 32, 64, 128 nodes
         for (int n = ((p.T + 15) / 16) * 16; n > 16; n = (n + 1) / 2) ++lg;
-        const double lead = (10.0 + 1.5 * lg) * n_ku / 32.0;
+        const double lead = (lg <= 2 ? 13.0 : 10.0 + 1.5 * lg) * n_ku / 32.0;
         int a = (int)((rho * n_ku + lead) / (1.0 + rho) + 0.999);
         if (a > n_ku - 1) a = n_ku - 1;
         const int R = n_ku - a;
