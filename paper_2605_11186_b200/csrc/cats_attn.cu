@@ -69,6 +69,7 @@ struct AttnDev {
     float* part_ml;      //              [nh][n_outer][T_pad][2]
     int dbg_skip_q;      // fault injection (tcgen05 kernel): the loader announces Q but never copies it
     WarmReq warm[3];     // see AttnProblem
+    int recv_over_ring;  // tcgen05 kernel: the records deposited by the cluster's CTAs lie over the K/V ring (see the kernel)
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -503,7 +504,7 @@ constexpr int kTcCols = 512;          // tensor-memory columns: S0 / P [0,192), 
 constexpr int kTcSStride = 192;
 constexpr int kTcStream = 64;         // cache rows per block when a share is streamed
 constexpr int kTcOneShot = 192;       // a share of at most this many rows is one block
-constexpr int kTcMaxStages = 4;
+constexpr int kTcMaxStages = 7;
 
 __device__ __forceinline__ void tmem_ld16_nowait(uint32_t taddr, float* v) {
     uint32_t r[16];
@@ -573,14 +574,23 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     constexpr int HD = 128, REC = HD + 4;
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
     const int Tpad = p.n_mt * 16;
-    uint8_t* q_s = sm;                                                           // [2][128][128 B]
-    uint8_t* kv_s = q_s + 128 * 256;                                             // ring of K and V blocks
+    // Q holds only the 32-row boxes that contain rows of the batch; the MMA reads 128 rows per head-dim half all the same
+    // (the rows beyond are whatever follows in shared memory; nobody reads their results).
+    const int q_rows = (Tpad + kTcBoxRows - 1) / kTcBoxRows * kTcBoxRows;
+    uint8_t* q_s = sm;                                                           // [2][q_rows][128 B]
+    uint8_t* kv_s = q_s + (size_t)q_rows * 256;                                  // ring of K and V blocks
     constexpr int NH = WIDE ? 4 : 2;                                             // softmax threads per query row
     constexpr int W_ISSUE = WIDE == 0 ? 8 : (WIDE == 1 ? 2 : 16), W_LOAD = W_ISSUE + 1, W_PV = WIDE == 1 ? 6 : W_ISSUE + 2;
     constexpr int N_SOFTMAX = WIDE == 2 ? 512 : 256;                             // softmax threads (arrivals per hand-off)
     float* xch = reinterpret_cast<float*>(kv_s + p.kv_area);                    // [2][NH][128] row maxima (by block parity), [NH][128] row sums
-    float* recv = xch + 3 * NH * 128;                                            // [csize][rpr][REC]
-    uint64_t* rbar = reinterpret_cast<uint64_t*>(recv + (p.csize > 1 ? (size_t)p.csize * p.rpr * REC : 0));   // base of the mbarriers; slot 0 unused
+    // The records the cluster's CTAs deposit here, [csize][rpr][REC].  Either an area of their own: then nothing but
+    // "that CTA has started" is required before a peer stores into it, and every thread arrives at the cluster barrier
+    // right after the set-up.  Or (recv_over_ring: streamed shares of large trees, where the area would cost two of five
+    // ring stages) they lie over the ring: then every thread arrives only when its part of the streaming is over, which
+    // costs the barrier's latency in front of the deposit.
+    const bool over_ring = p.recv_over_ring != 0;
+    float* recv = over_ring ? reinterpret_cast<float*>(kv_s) : xch + 3 * NH * 128;
+    uint64_t* rbar = reinterpret_cast<uint64_t*>(xch + 3 * NH * 128 + ((p.csize > 1 && !over_ring) ? (size_t)p.csize * p.rpr * REC : 0));   // base of the mbarriers; slot 0 unused
     // Every barrier that a thread may find more than one phase ahead of itself would give a wrong answer to a parity
     // wait, so each one is either indexed by block parity (its next completion needs the waiter's own progress) or by
     // ring stage (the classical full / empty pair).
@@ -659,8 +669,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    // nobody stores into a peer's shared memory before that CTA has started: arrive here, wait just before the deposit
-    if (p.csize > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    if (p.csize > 1 && !over_ring) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_wait();
     const uint32_t tbase = *tmem_slot;
     // tensor-memory columns.  One-block share: S / P [0,192), O [384,512).  Streamed: S / P buffers [64 k, 64 k + 64), k < 4.
@@ -710,7 +719,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
                 const uint64_t da0 = umma_desc_sw128(q_u32), db0 = umma_desc_sw128(ks_u32);      // the address field takes plain additions
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
-                    const uint64_t da = da0 + (uint64_t)(((ks >> 2) * (128 * 128) + (ks & 3) * 32) >> 4);
+                    const uint64_t da = da0 + (uint64_t)(((ks >> 2) * (q_rows * 128) + (ks & 3) * 32) >> 4);
                     const uint64_t db = db0 + (uint64_t)(((uint32_t)(ks >> 2) * half + (uint32_t)(ks & 3) * 32u) >> 4);
                     umma_bf16(tS, da, db, idesc, ks > 0);
                 }
@@ -734,10 +743,10 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     } else if (warp == W_LOAD) {
         // ---- loader: Q and the boxes that depend on the previous kernel, then a refill whenever a P V product frees a stage ----
         if (lane == 0) {
-            if (nb > 0) mbar_expect_tx(bar_q, 128u * 256u);
-            for (int rb = 0; rb < 128 && nb > 0 && !p.dbg_skip_q; rb += kTcBoxRows) {
+            if (nb > 0) mbar_expect_tx(bar_q, (uint32_t)q_rows * 256u);
+            for (int rb = 0; rb < q_rows && nb > 0 && !p.dbg_skip_q; rb += kTcBoxRows) {
                 tma_load_2d(q_s + (size_t)rb * 128, &tm_q, h * HD, rb, bar_q, ld_policy);
-                tma_load_2d(q_s + 128 * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
+                tma_load_2d(q_s + (size_t)q_rows * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
             }
             for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 1, ld_policy);
             for (int j = NST; STREAM && j < nb; ++j) {
@@ -869,7 +878,11 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             if (ok) ok = mbar_wait(bar_o + sbuf(nb - 1), sphase(nb - 1), wait_expired);
             tc_fence_after_sync();
         }
-        if (p.csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every CTA of the cluster has started
+        // Nobody stores into a peer's shared memory before that CTA has started, or, with the records over the ring, is done
+        // with its ring: the first phase of the cluster barrier (over_ring: these warps arrive now that their last product
+        // has completed, the others when they have issued their last copy or MMA).
+        if (p.csize > 1 && over_ring) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (p.csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         if (act) {
             float* xl = xch + 2 * NH * 128;                     // [NH][128]
             xl[hf * 128 + row] = l_run;
@@ -911,6 +924,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     int part_stride = Tpad * REC, row0 = 0, n_my = Tpad;
     if (csize > 1) {
         // the softmax warps have passed the first phase of the cluster barrier above; the second one publishes the records
+        if (!softmax_warp && over_ring) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         if (!softmax_warp) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
         asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -1170,13 +1184,15 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     const size_t recv = p.cluster > 1 ? (size_t)p.cluster * d.rpr * rec * 4 : 0;
     // four softmax threads per query row (see kTcThreadsWide), on 8 softmax warps for trees of <= 64 nodes, else on 16
     const int wide = g_debug_attn_kernel == 2 ? 0 : (tpad <= 64 ? 1 : 2);
-    const size_t fixed = 1024 + 128 * 256 + (wide ? 6144 : 3072) + recv + 192;     // alignment slack, Q, exchange among a row's threads, received partials, barriers
+    const size_t q_bytes = (size_t)((tpad + kTcBoxRows - 1) / kTcBoxRows * kTcBoxRows) * 256;
+    d.recv_over_ring = (p.cluster > 1 && wide == 2 && p.rows_per_split > kTcOneShot) ? 1 : 0;
+    const size_t fixed = 1024 + q_bytes + (wide ? 6144 : 3072) + (d.recv_over_ring ? 0 : recv) + 320;     // alignment slack, Q, exchange among a row's threads, received records, barriers
     // the ring: stages of 64 rows of K and V (32 KB each), as many as fit, at least three (which also hold a one-block share)
     int stages = (int)((227 * 1024 - fixed) / (kTcStream * 512));
     if (stages > kTcMaxStages) stages = kTcMaxStages;
     if (stages < 3) return cudaErrorInvalidConfiguration;
     d.kv_area = stages * kTcStream * 512;
-    if ((size_t)d.kv_area < (size_t)tpad * rec * 4) return cudaErrorInvalidConfiguration;   // the deposit aliases the ring
+    if ((size_t)d.kv_area < (size_t)tpad * rec * 4 || (size_t)d.kv_area < recv) return cudaErrorInvalidConfiguration;   // the deposit lies over the ring
     if (p.rows_per_split <= kTcOneShot) {
         d.blk = (p.rows_per_split + 31) / 32 * 32;
         d.stages = 1;
