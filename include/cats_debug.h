@@ -61,6 +61,17 @@ void cats_debug_inject_fault(int which);
  * Changes no result. */
 void cats_debug_l2_warm(int which, int period, int phase);
 
+/* Time line of the kernels inside a forward.  Only a library built with
+ * -DCATS_TIMELINE records one (paper_2605_11186_b200/timeline.py builds it
+ * beside the normal library and prints the table); the normal build returns
+ * CATS_ERR_UNSUPPORTED.  kernel: 0 the projection kernel (512 launch slots),
+ * 1 the tcgen05 attention kernel (128), 2 the register RMSNorm kernel (256);
+ * a launch slot is [160 CTAs][16 stamps] of 64-bit %globaltimer values (ns),
+ * zero where a CTA or stamp does not exist; the stamps are listed beside each
+ * kernel in the sources.  host == NULL clears the slots and restarts the
+ * numbering; else up to `bytes` bytes are copied to the HOST buffer. */
+int cats_debug_timeline(int kernel, void *host, size_t bytes);
+
 #ifdef __cplusplus
 }
 #endif

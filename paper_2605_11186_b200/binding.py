@@ -13,8 +13,12 @@ from . import build as _build
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcats.so")
-
-if not os.path.exists(LIB_PATH):
+# CATS_LIBRARY: another build of the same library (timeline.py sets it to the measurement build before importing this)
+if os.environ.get("CATS_LIBRARY"):
+    LIB_PATH = os.environ["CATS_LIBRARY"]
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError("CATS_LIBRARY=%s does not exist" % LIB_PATH)
+elif not os.path.exists(LIB_PATH):
     _build.build()
 lib = C.CDLL(LIB_PATH)
 
@@ -209,6 +213,23 @@ def l2_warm(which: int, period: int, phase: int = 0) -> None:
     gate/up, 2 attention -> down, 3 norm before QKV -> QKV, 4 norm before gate/up -> gate/up); every period-th 32 KB unit
     from unit ``phase``; period 0 none, -1 the built-in choice."""
     lib.cats_debug_l2_warm(C.c_int(which), C.c_int(period), C.c_int(phase))
+
+
+TIMELINE_SLOTS = {0: 512, 1: 128, 2: 256}     # launch slots per kernel (projection, tcgen05 attention, register norm)
+
+
+def timeline(kernel: int):
+    """cats_debug_timeline: the stamps of the given kernel as an int64 array [slots][160][16] (ns, zero = not written).
+    Only the measurement build records them (CatsError UNSUPPORTED otherwise)."""
+    import numpy as np
+    a = np.zeros((TIMELINE_SLOTS[kernel], 160, 16), dtype=np.uint64)
+    _check(lib.cats_debug_timeline(C.c_int(kernel), C.c_void_p(a.ctypes.data), C.c_size_t(a.nbytes)), "cats_debug_timeline")
+    return a.astype(np.int64)
+
+
+def timeline_clear() -> None:
+    for k in TIMELINE_SLOTS:
+        _check(lib.cats_debug_timeline(C.c_int(k), None, C.c_size_t(0)), "cats_debug_timeline")
 
 
 def workspace_layout(cfg: ModelCfg, T: int) -> dict:

@@ -11,23 +11,28 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC", "--shared", "-cudart", "static"]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib=LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(os.path.join(CSRC, f)) > t for f in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
+TIMELINE_LIB = os.path.join(HERE, "libcats_timeline.so")
+
+
+def build(force: bool = False, verbose: bool = False, timeline: bool = False) -> str:
+    """timeline: build the measurement variant (``-DCATS_TIMELINE``, see cats_debug_timeline) as libcats_timeline.so."""
+    out = TIMELINE_LIB if timeline else LIB
+    if not force and not _stale(out):
+        return out
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    tmp = out + ".tmp.%d" % os.getpid()
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + (["-DCATS_TIMELINE"] if timeline else []) + \
         [os.path.join(CSRC, f) for f in SOURCES] + ["-ldl", "-o", tmp]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

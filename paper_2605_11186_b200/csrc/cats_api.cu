@@ -258,6 +258,15 @@ int cats_last_launch_count(void) { return g_launch_count; }
 void cats_debug_stage_mask(unsigned mask) { g_stage_mask = mask & 0x7f; }
 void cats_debug_attention_kernel(int which) { g_debug_attn_kernel = which < 0 ? -1 : (which > 2 ? 1 : which); }
 void cats_debug_l2_warm(int which, int period, int phase) { if (which >= 0 && which < 5) { g_warm[which][0] = period; g_warm[which][1] = phase; } }
+int cats_debug_timeline(int kernel, void* host, size_t bytes) {
+    const bool clear = host == nullptr;
+    cudaError_t e = cudaErrorInvalidValue;
+    if (kernel == 0) e = timeline_gemm(host, bytes, clear);
+    else if (kernel == 1) e = timeline_attn(host, bytes, clear);
+    else if (kernel == 2) e = timeline_norm(host, bytes, clear);
+    if (e == cudaErrorNotSupported) return CATS_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? CATS_OK : (e == cudaErrorInvalidValue ? CATS_ERR_INVALID_ARG : CATS_ERR_CUDA);
+}
 void cats_debug_inject_fault(int which) { g_debug_fault = (which == 1 || which == 2) ? which : 0; }
 int cats_debug_wait_limit_ns(unsigned long long ns) {
     if (ns == 0) ns = kWaitLimitNs;

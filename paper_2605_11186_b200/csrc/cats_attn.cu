@@ -70,7 +70,20 @@ struct AttnDev {
     int dbg_skip_q;      // fault injection (tcgen05 kernel): the loader announces Q but never copies it
     WarmReq warm[3];     // see AttnProblem
     int recv_over_ring;  // tcgen05 kernel: the records deposited by the cluster's CTAs lie over the K/V ring (see the kernel)
+#ifdef CATS_TIMELINE
+    unsigned long long* tl;      // this launch's time-line slot
+#endif
 };
+#ifdef CATS_TIMELINE
+#define ATTN_TL(slot) CATS_TL(p.tl, slot)
+static __device__ unsigned long long g_tl_attn[128 * kTlCtas * kTlStamps];
+static int g_tl_attn_next = 0;
+#else
+#define ATTN_TL(slot) do { } while (0)
+#endif
+// time-line stamps of the tcgen05 kernel: 0 CTA entered, 1 set-up done, 2 dependency resolved, 3 dependent copies issued,
+// 4 Q and the first block landed, 5 first Q K^T issued, 6 first S complete, 7 last P written, 8 last P V complete,
+// 9 records deposited, 10 records published (cluster barrier), 11 merged, CTA leaves
 
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -572,6 +585,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
                                                                 const __grid_constant__ CUtensorMap tm_v) {
     extern __shared__ __align__(128) uint8_t sm_raw[];
     constexpr int HD = 128, REC = HD + 4;
+    if (threadIdx.x == 0) ATTN_TL(0);
     uint8_t* sm = sm_raw + ((1024u - (smem_u32(sm_raw) & 1023u)) & 1023u);      // the operand tiles need 1024-byte alignment
     const int Tpad = p.n_mt * 16;
     // Q holds only the 32-row boxes that contain rows of the batch; the MMA reads 128 rows per head-dim half all the same
@@ -669,8 +683,10 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    if (threadIdx.x == 0) ATTN_TL(1);
     if (p.csize > 1 && !over_ring) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     pdl_wait();
+    if (threadIdx.x == 0) ATTN_TL(2);
     const uint32_t tbase = *tmem_slot;
     // tensor-memory columns.  One-block share: S / P [0,192), O [384,512).  Streamed: S / P buffers [64 k, 64 k + 64), k < 4.
     const uint32_t tO = tbase + 384;
@@ -710,6 +726,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
                 ok = mbar_wait(bar_kv + b % NST, (uint32_t)(b / NST) & 1u, wait_expired);
                 if (ok && b >= NSB) ok = mbar_wait(bar_o + sbuf(b), sphase(b - NSB), wait_expired);
                 if (!ok) break;
+                if (b == 0) ATTN_TL(4);
                 tc_fence_after_sync();
                 const int r0 = c_begin + b * NB;
                 const int n16 = min(NB, (c_end - r0 + 15) & ~15);
@@ -724,6 +741,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
                     umma_bf16(tS, da, db, idesc, ks > 0);
                 }
                 umma_commit(bar_s + sbuf(b));
+                if (b == 0) ATTN_TL(5);
             }
             if (!STREAM) {
                 // A one-block share moves little data: HBM is free to fetch the coming projections' weights meanwhile.
@@ -749,6 +767,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
                 tma_load_2d(q_s + (size_t)q_rows * 128 + (size_t)rb * 128, &tm_q, h * HD + 64, rb, bar_q, ld_policy);
             }
             for (int b = 0; b < NST && b < nb; ++b) load_kv(b, b, 1, ld_policy);
+            ATTN_TL(3);
             for (int j = NST; STREAM && j < nb; ++j) {
                 if (!mbar_wait(bar_free + j % NST, (uint32_t)(j / NST - 1) & 1u, wait_expired)) break;
                 mbar_expect_tx(bar_kv + j % NST, (uint32_t)stage_bytes);
@@ -776,6 +795,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             float v[CPT];
             float corr = 1.f, ref = 0.f;
             if (ok) ok = mbar_wait(bar_s + sbuf(b), sphase(b), wait_expired);
+            if (threadIdx.x == 0 && b == 0) ATTN_TL(6);
             tc_fence_after_sync();
             if (act) {
 #pragma unroll
@@ -871,6 +891,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             // before every thread has arrived for the buffer's previous block (S(b) is issued only after that block's
             // P V has completed, which needed all of its P).
             mbar_arrive(bar_p + sbuf(b));
+            if (threadIdx.x == 0 && b == nb - 1) ATTN_TL(7);
         }
         // ---- this thread's half of the row's O, and the row's (m, l), go straight into the shared memory of the CTA
         //      that merges the row: stores through distributed shared memory, made visible by the cluster barrier ----
@@ -878,6 +899,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             if (ok) ok = mbar_wait(bar_o + sbuf(nb - 1), sphase(nb - 1), wait_expired);
             tc_fence_after_sync();
         }
+        if (threadIdx.x == 0) ATTN_TL(8);
         // Nobody stores into a peer's shared memory before that CTA has started, or, with the records over the ring, is done
         // with its ring: the first phase of the cluster barrier (over_ring: these warps arrive now that their last product
         // has completed, the others when they have issued their last copy or MMA).
@@ -916,6 +938,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             }
         }
     }
+    if (threadIdx.x == 0) ATTN_TL(9);
     tc_fence_before_sync();
     const int csize = p.csize, rpr = p.rpr;
     const int rank = split % csize, outer = split / csize;
@@ -935,6 +958,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
     } else {
         __syncthreads();
     }
+    if (threadIdx.x == 0) ATTN_TL(10);
     if (warp == W_ISSUE) {
         tc_fence_after_sync();
         tmem_dealloc(tbase, kTcCols);
@@ -988,6 +1012,7 @@ __global__ void __launch_bounds__(tc_threads(WIDE), 1) k_tree_attn_tc(const Attn
             if (c8 == 0) { p.part_ml[gbase * 2] = M; p.part_ml[gbase * 2 + 1] = L; }
         }
     }
+    if (threadIdx.x == 0) ATTN_TL(11);
 }
 
 // out[t][h][:] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s over the clusters of a head.  One CTA per (node, head).
@@ -1178,6 +1203,13 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     d.part_o = p.part_o; d.part_ml = p.part_ml;
     d.d_status = p.d_status;
     d.dbg_skip_q = g_debug_fault == 2 ? 1 : 0;
+#ifdef CATS_TIMELINE
+    {
+        unsigned long long* base = nullptr;
+        cudaGetSymbolAddress((void**)&base, g_tl_attn);
+        d.tl = base + (size_t)(g_tl_attn_next++ % 128) * kTlCtas * kTlStamps;
+    }
+#endif
     for (int w = 0; w < 3; ++w) d.warm[w] = warm_req(p.warm[w].ptr, p.warm[w].bytes, p.warm[w].period, p.warm[w].phase);
     const int tpad = d.n_mt * 16, rec = p.hd + 4;
     d.rpr = (((tpad + p.cluster - 1) / p.cluster) + 1) / 2 * 2;
@@ -1228,6 +1260,22 @@ static cudaError_t launch_tree_attention_tc(const AttnProblem& p, cudaStream_t s
     if (e != cudaSuccess || p.n_splits == 1) return e;
     return launch_pdl(k_attn_combine, dim3(p.T, p.nh), dim3(128), 0, st, (const float*)p.part_o, (const float*)p.part_ml,
                       p.n_splits, tpad, p.nh, p.hd, (uint16_t*)p.out, p.out_packed_npad);
+}
+
+// Time line of the tcgen05 attention launches (measurement builds): copies the stamps to the host, or clears them.
+cudaError_t timeline_attn(void* host, size_t bytes, bool clear) {
+#ifdef CATS_TIMELINE
+    if (clear) {
+        void* b = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&b, g_tl_attn);
+        g_tl_attn_next = 0;
+        return e != cudaSuccess ? e : cudaMemset(b, 0, sizeof(g_tl_attn));
+    }
+    return cudaMemcpyFromSymbol(host, g_tl_attn, bytes < sizeof(g_tl_attn) ? bytes : sizeof(g_tl_attn));
+#else
+    (void)host; (void)bytes; (void)clear;
+    return cudaErrorNotSupported;
+#endif
 }
 
 cudaError_t launch_tree_attention(const AttnProblem& p, cudaStream_t st) {

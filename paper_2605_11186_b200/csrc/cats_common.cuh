@@ -55,6 +55,16 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // launch_dependents: lets the next kernel in the stream start its prologue.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- time line (measurement builds only: -DCATS_TIMELINE) ---------------------------------------
+// Every launch of the projection, attention and norm kernels gets a slot of [kTlCtas][kTlStamps] 64-bit words; a CTA's
+// role threads store %globaltimer there at the points named in timeline.py.  Nothing of this exists in a normal build.
+constexpr int kTlCtas = 160, kTlStamps = 16;
+#ifdef CATS_TIMELINE
+#define CATS_TL(base, slot) do { (base)[(size_t)(blockIdx.y * gridDim.x + blockIdx.x) * kTlStamps + (slot)] = globaltimer_ns(); } while (0)
+#else
+#define CATS_TL(base, slot) do { } while (0)
+#endif
+
 // ---- requests into L2 ----------------------------------------------------------------------------
 // Weights a later kernel will stream, requested into L2 by a kernel that leaves HBM idle: of the 32 KB units of
 // [ptr, ptr + bytes) every period-th one starting at unit `phase`, so that the later kernel draws on L2 and HBM at once.

@@ -72,8 +72,22 @@ struct GemmDev {
     const int32_t *tree_parent, *tree_tokens;   //   [T]
     float* cand;                  //   [T]: logit of every node's own token at its parent
     int32_t* d_status;
+#ifdef CATS_TIMELINE
+    unsigned long long* tl;      // this launch's time-line slot
+#endif
     int dbg_skip_publish;        // fault injection: contributors of shared tiles keep their flags to themselves
 };
+
+#ifdef CATS_TIMELINE
+#define GEMM_TL(slot) CATS_TL(p.tl, slot)
+static __device__ unsigned long long g_tl_gemm[512 * kTlCtas * kTlStamps];
+static int g_tl_gemm_next = 0;
+#else
+#define GEMM_TL(slot) do { } while (0)
+#endif
+// time-line stamps of this kernel: 0 CTA entered, 1 set-up done, 2 first weight copy issued, 3 first stage landed,
+// 4 dependency resolved, 5 last weight copy issued, 6 last stage landed, 7 last accumulator complete, 8 epilogue done
+// (group 0; 12: group 1), 9 CTA leaves, 10 the SM's id, 11 first activation copy issued
 
 struct GemmCtrl {
     uint64_t full[kMaxStages];
@@ -224,10 +238,13 @@ __device__ __forceinline__ bool produce_units(const GemmDev& p, const CtaRange& 
             const uint32_t bytes = (uint32_t)nk * kWChunk;
             mbar_expect_tx(&pp.ctrl->full[s], bytes);
             bulk_load(stage, p.Wp + ((size_t)tile * p.n_kb + kb) * kWChunk, bytes, &pp.ctrl->full[s], pol);
+            if (k == 0) GEMM_TL(2);
+            if (k == n_units - 1) GEMM_TL(5);
         } else {
             const uint32_t bytes = (uint32_t)nk * p.x_chunk_bytes;
             mbar_expect_tx(&pp.ctrl->full[s], bytes);
             bulk_load(stage + kUnitKb * kWChunk, p.Xp + (size_t)kb * p.x_chunk_bytes, bytes, &pp.ctrl->full[s], pol);
+            if (k == 0) GEMM_TL(11);
         }
         if (++s == S) { s = 0; par ^= 1u; }
         if (++v == r.vlen) { v = 0; ++tile; }
@@ -261,6 +278,8 @@ __device__ __forceinline__ bool mma_units(const GemmDev& p, const CtaRange& r, c
         for (; u < seg_end && ok; ++u, ++i, ++v) {
             ok = mbar_wait(&pp.ctrl->full[s], par, pp.abort_flag);
             if (!ok) break;
+            if (half == 0 && u == r.u0) GEMM_TL(3);
+            if (half == 0 && u == r.u1 - 1) GEMM_TL(6);
             tc_fence_after_sync();
             const int kb = (r.koff + v) * kUnitKb;
             const int nk = min(kUnitKb, p.n_kb - kb);
@@ -371,6 +390,7 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
         }
         if (ok) ok = mbar_wait(&pp.ctrl->acc_full[b], (seg >> 1) & 1, pp.abort_flag);
         ok = ok && !*pp.abort_flag;
+        if (et == 0 && group == 0 && u >= r.u1) GEMM_TL(7);
         tc_fence_after_sync();
         const uint32_t taddr = pp.tmem_acc + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(b * pp.acc_stride);
         const uint32_t dual = pp.dual ? (uint32_t)p.n_pad : 0u;
@@ -570,6 +590,7 @@ __device__ __forceinline__ void epilogue_units(const GemmDev& p, const CtaRange&
         }
         tc_fence_before_sync();
         mbar_arrive(&pp.ctrl->acc_empty[b]);
+        if (et == 0 && u >= r.u1) GEMM_TL(8 + group * 4);
     }
 }
 
@@ -633,7 +654,16 @@ template <int EPI>
 __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     Pipe pp;
+#ifdef CATS_TIMELINE
+    if (threadIdx.x == 0) {
+        GEMM_TL(0);
+        unsigned sm;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
+        p.tl[(size_t)blockIdx.x * kTlStamps + 10] = sm;
+    }
+#endif
     if (!pipe_setup(pp, smem_raw, p.n_stages, p.stage_bytes, p.tmem_cols, p.n_pad, p.d_status)) return;
+    if (threadIdx.x == 0) GEMM_TL(1);
     pdl_launch_dependents();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -645,7 +675,10 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
         if (lane == 0) {
             const bool is_w = (warp == 0);
             const uint64_t pol = is_w ? l2_policy_evict_first() : l2_policy_evict_last();
-            if (!is_w) pdl_wait();    // activations come from the previous kernel; weights never do
+            if (!is_w) {
+                pdl_wait();    // activations come from the previous kernel; weights never do
+                GEMM_TL(4);
+            }
             int i = 0;
             produce_units(p, r, pp, is_w, pol, i);
             if (*pp.abort_flag) drain_after_abort(pp, i);
@@ -670,6 +703,7 @@ __global__ void __maxnreg__(CATS_GEMM_MAXREG) k_gemm_sk(const GemmDev p) {
         epilogue_units<EPI>(p, r, pp, cta, warp, lane, warp < 6 ? 0 : 1, seg, ok);
     }
     pipe_teardown(pp, p.tmem_cols, p.d_status);
+    if (threadIdx.x == 0) GEMM_TL(9);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -734,6 +768,22 @@ cudaError_t launch_pack_weights(const void* const* src, int n_src, int layout, i
 // ---------------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------------
+// Time line of the projection launches (measurement builds): copies the stamps to the host, or clears them.
+cudaError_t timeline_gemm(void* host, size_t bytes, bool clear) {
+#ifdef CATS_TIMELINE
+    if (clear) {
+        void* b = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&b, g_tl_gemm);
+        g_tl_gemm_next = 0;
+        return e != cudaSuccess ? e : cudaMemset(b, 0, sizeof(g_tl_gemm));
+    }
+    return cudaMemcpyFromSymbol(host, g_tl_gemm, bytes < sizeof(g_tl_gemm) ? bytes : sizeof(g_tl_gemm));
+#else
+    (void)host; (void)bytes; (void)clear;
+    return cudaErrorNotSupported;
+#endif
+}
+
 cudaError_t set_wait_limit_gemm(unsigned long long ns) { return cudaMemcpyToSymbol(g_wait_limit_ns, &ns, sizeof(ns)); }
 
 int gemm_num_tiles(const GemmProblem& p) {
@@ -871,6 +921,13 @@ size_t make_gemm_dev(const GemmProblem& p, const GemmPlan& pl, int max_stages, G
     d.cand = p.cand;
     d.d_status = p.d_status;
     d.dbg_skip_publish = g_debug_fault == 1 ? 1 : 0;
+#ifdef CATS_TIMELINE
+    {
+        unsigned long long* base = nullptr;
+        cudaGetSymbolAddress((void**)&base, g_tl_gemm);
+        d.tl = base + (size_t)(g_tl_gemm_next++ % 512) * kTlCtas * kTlStamps;
+    }
+#endif
     return (size_t)stages * d.stage_bytes + kStagingBytes + kCtrlBytes;
 }
 }  // namespace

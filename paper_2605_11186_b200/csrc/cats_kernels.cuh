@@ -50,6 +50,11 @@ cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* pa
                            const void* gain, int T, int H, float eps, void* xn_packed, const int32_t* pos, const int32_t* nodes,
                            float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st,
                            int32_t* d_status = nullptr, const WarmReq* warm = nullptr);   // warm: see WarmReq (register kernel only)
+// Time lines (builds with -DCATS_TIMELINE; cudaErrorNotSupported otherwise): every launch of the kernel writes a slot of
+// [kTlCtas][kTlStamps] 64-bit words, the stamps being %globaltimer values at points listed beside each kernel.
+cudaError_t timeline_gemm(void* host, size_t bytes, bool clear);    // 512 slots
+cudaError_t timeline_attn(void* host, size_t bytes, bool clear);    // 128 slots (tcgen05 kernel)
+cudaError_t timeline_norm(void* host, size_t bytes, bool clear);    // 256 slots (k_rmsnorm_reg)
 // Checks a partial-tree node list (strictly ascending, inside [0, T)) and writes a copy clamped into range.
 cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st);
 cudaError_t launch_argmax_reduce(const float* pmax, const int32_t* pidx, int n_tiles, int t_stride, int T, int32_t* amax,

@@ -443,6 +443,16 @@ cudaError_t set_wait_limit_small(unsigned long long ns) { return cudaMemcpyToSym
 // Footprint: a CTA of this kernel fits on an SM beside a resident CTA of the projection kernel, so the projection that
 // follows can already be resident and stream its first weight stages while the norm runs.  Thread pairs (even, odd
 // lane) hold the two halves of one 16-byte group of the packed output.
+#ifdef CATS_TIMELINE
+static __device__ unsigned long long g_tl_norm[256 * kTlCtas * kTlStamps];
+static int g_tl_norm_next = 0;
+#define NORM_TL(slot) CATS_TL(tl, slot)
+#define NORM_TL_PARAM , unsigned long long* tl
+#else
+#define NORM_TL(slot) do { } while (0)
+#define NORM_TL_PARAM
+#endif
+// time-line stamps of k_rmsnorm_reg: 0 CTA entered, 2 dependency resolved, 3 row and partial sums summed, 9 CTA leaves
 template <int NC>
 __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, const float* __restrict__ copy_from,
                                                      const float* __restrict__ part, int n_part, size_t part_stride,
@@ -450,11 +460,12 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
                                                      uint8_t* __restrict__ xn, int n_pad, const int32_t* __restrict__ pos,
                                                      const int32_t* __restrict__ nodes, float2* __restrict__ rope, int hd,
                                                      float rope_base, int* zero_flags, int n_flags, int cs,
-                                                     int32_t* d_status, const WarmReq warm) {
+                                                     int32_t* d_status, const WarmReq warm NORM_TL_PARAM) {
     __shared__ float red[8];
     __shared__ __align__(8) uint64_t xbar;     // completes when the partial sums of squares of all cs CTAs have landed
     __shared__ float slots[4];                 // slots[r]: the partial sum of the cluster's CTA r
     __shared__ int wait_expired;
+    if (threadIdx.x == 0) NORM_TL(0);
     pdl_launch_dependents();
     const int t = blockIdx.x / cs, rank = blockIdx.x - t * cs;
     const int cols_cta = H / 4 / cs;          // float4 columns of this CTA
@@ -477,6 +488,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
         if (xn != nullptr && cl < cols_cta) g[j] = __ldg(reinterpret_cast<const uint2*>(gain) + col0 + cl);
     }
     pdl_wait();
+    if (threadIdx.x == 0) NORM_TL(2);
     if (zero_flags != nullptr && blockIdx.x == 0)
         for (int i = threadIdx.x; i < n_flags; i += blockDim.x) zero_flags[i] = 0;
     const float4* r4 = reinterpret_cast<const float4*>((copy_from ? copy_from : resid) + (size_t)t * H);
@@ -531,6 +543,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
+    if (threadIdx.x == 0) NORM_TL(3);
     float tot = 0.f;
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
@@ -575,6 +588,7 @@ __global__ void __launch_bounds__(256) k_rmsnorm_reg(float* __restrict__ resid, 
             *reinterpret_cast<uint2*>(xn + packed_act_offset(t, c >> 1, n_pad) + (size_t)(c & 1) * 8) = o;
         }
     }
+    if (threadIdx.x == 0) NORM_TL(9);
 }
 
 template <typename Kern, typename... Args>
@@ -620,11 +634,19 @@ cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* pa
                            float2* rope, int hd, float rope_base, int* zero_flags, int n_flags, cudaStream_t st,
                            int32_t* d_status, const WarmReq* warm_in) {
     const int n_pad = (T + 15) / 16 * 16;
+#ifdef CATS_TIMELINE
+    unsigned long long* tl_ptr = nullptr;
+    cudaGetSymbolAddress((void**)&tl_ptr, g_tl_norm);
+    tl_ptr += (size_t)(g_tl_norm_next++ % 256) * kTlCtas * kTlStamps;
+#define NORM_TL_ARG , tl_ptr
+#else
+#define NORM_TL_ARG
+#endif
     const WarmReq warm = warm_in ? warm_req(warm_in->ptr, warm_in->bytes, warm_in->period, warm_in->phase) : warm_req(nullptr, 0, 0, 0);
 #define CATS_NORM_REG(NC)                                                                                                   \
     return launch_cluster_pdl(k_rmsnorm_reg<NC>, dim3(T * cs), dim3(256), cs, st, resid, copy_from, part, n_part, part_stride, \
                               (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, n_pad, pos, nodes, rope, hd, rope_base,    \
-                              zero_flags, n_flags, cs, d_status, warm)
+                              zero_flags, n_flags, cs, d_status, warm NORM_TL_ARG)
 #ifndef CATS_NORM_SMEM
     {
         // as many CTAs per row as keep the grid within one wave and leave every CTA at least 256 columns
@@ -644,6 +666,22 @@ cudaError_t launch_rmsnorm(float* resid, const float* copy_from, const float* pa
     return launch_pdl(k_rmsnorm, dim3(T), dim3(256), (size_t)H * sizeof(float), st, resid, copy_from, part, n_part,
                       part_stride, (const uint16_t*)gain, H, eps, (uint8_t*)xn_packed, n_pad, pos, nodes, rope,
                       hd, rope_base, zero_flags, n_flags);
+}
+
+// Time line of the k_rmsnorm_reg launches (measurement builds): copies the stamps to the host, or clears them.
+cudaError_t timeline_norm(void* host, size_t bytes, bool clear) {
+#ifdef CATS_TIMELINE
+    if (clear) {
+        void* b = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&b, g_tl_norm);
+        g_tl_norm_next = 0;
+        return e != cudaSuccess ? e : cudaMemset(b, 0, sizeof(g_tl_norm));
+    }
+    return cudaMemcpyFromSymbol(host, g_tl_norm, bytes < sizeof(g_tl_norm) ? bytes : sizeof(g_tl_norm));
+#else
+    (void)host; (void)bytes; (void)clear;
+    return cudaErrorNotSupported;
+#endif
 }
 
 cudaError_t launch_check_nodes(const int32_t* nodes, int m, int T, int32_t* clamped, int32_t* d_status, cudaStream_t st) {
